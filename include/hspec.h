@@ -1,0 +1,205 @@
+/*
+ * hspec.h — C ABI of the H-Spec block-parallel draft step on one B200 (sm_100a).
+ *
+ * One call of hspec_draft_block runs, for B concurrent requests, one forward pass of
+ * the hybrid Mamba-attention drafter of the paper (Sec. 3.3, App. B.1):
+ *   last-position target hidden state -> Proj_r -> Proj_dS -> S_init   (Sec. 3.3.1, eq. for S_init)
+ *   k block rows (last token, then mask tokens; no positional embedding) (Sec. 3.3.1, "Input-dependent selectivity")
+ *   per layer: Mamba-2 mixer scanned over the k rows from S_init          (Sec. 3.3.1)
+ *              attention whose keys/values are the target model's own paged KV cache, read
+ *              in place, plus the block's causal keys/values              (Sec. 3.3.2)
+ *              SwiGLU MLP                                                 (App. B.1 "MLP")
+ *   final norm, the target's LM head, arg-max -> k draft tokens           (App. B.2 "Pruned drafter vocabulary": LM head is the target's)
+ * No drafter-side KV cache exists: the library never writes the KV pools (Sec. 3.2).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
+ *     ordinary host memory.  No torch / C++ types cross this boundary.
+ *   - All matrices are row-major [out_features, in_features] bf16; vectors are fp32.
+ *   - Every function returns HSPEC_OK (0) or a negative hspec_status; nothing throws or aborts.
+ *     hspec_last_error() returns a static or per-handle message for the last failure.
+ *   - Work is enqueued on the caller's stream; hspec_draft_block performs no host synchronisation.
+ *     Asynchronous device faults surface through the CUDA runtime on the caller's next sync;
+ *     bounded in-kernel waits that give up set a device status word readable with hspec_get_stats.
+ *   - A library built without a usable CUDA device fails loudly (HSPEC_ERR_CUDA): there is no CPU path.
+ */
+#ifndef HSPEC_H_
+#define HSPEC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define HSPEC_MAX_LAYERS 16
+#define HSPEC_MAX_SLOTS 16
+#define HSPEC_MAX_K 32            /* block positions per step */
+
+typedef enum {
+  HSPEC_OK = 0,
+  HSPEC_ERR_INVALID_ARG = -1,        /* NULL pointer, bad handle, B/k out of range */
+  HSPEC_ERR_BAD_SHAPE = -2,          /* config or tensor shape the kernels cannot take */
+  HSPEC_ERR_NOT_LOADED = -3,         /* a required weight tensor was never loaded */
+  HSPEC_ERR_WORKSPACE_TOO_SMALL = -4,
+  HSPEC_ERR_PAGE_OUT_OF_RANGE = -5,  /* host-side validation of a page table found a bad id */
+  HSPEC_ERR_CUDA = -6,               /* a CUDA runtime / driver call failed (message has the text) */
+  HSPEC_ERR_TIMEOUT = -7             /* a bounded in-kernel wait gave up (status word) */
+} hspec_status;
+
+typedef enum { HSPEC_BF16 = 0, HSPEC_F32 = 1, HSPEC_I32 = 2 } hspec_dtype;
+
+/* Shapes of the drafter (App. B.1).  H = Di / P Mamba heads; d_S = H * P * N. */
+typedef struct {
+  int32_t D;                 /* hidden size of target and drafter */
+  int32_t n_fuse;            /* number of target layers whose last-position hidden states are concatenated */
+  int32_t r;                 /* fusion rank of Proj_r (the paper sets it to D) */
+  int32_t L;                 /* drafter layers, <= HSPEC_MAX_LAYERS */
+  int32_t has_attn[HSPEC_MAX_LAYERS]; /* 1: Mamba-attention-MLP layer, 0: Mamba-MLP layer */
+  int32_t kv_slot[HSPEC_MAX_LAYERS];  /* which target-layer KV pool layer l's attention reads (layer-wise KV mapping) */
+  int32_t n_slots;           /* number of distinct target KV pools passed per step */
+  int32_t Di, P, N, G;       /* Mamba-2: inner width, head dim, state dim, B/C groups */
+  int32_t d_conv;            /* depthwise conv width (<= 4) */
+  int32_t dt_rank;           /* 0: dt projected directly to H; >0: through a rank-dt_rank bottleneck */
+  int32_t Hq, Hkv, dh;       /* attention heads (= the target's), head dim (64 or 128) */
+  float rope_theta;          /* the target's RoPE base */
+  int32_t window;            /* sliding window in tokens, 0 = full context */
+  int32_t qk_norm;           /* 1: per-head RMSNorm on q and the block's k before RoPE */
+  int32_t F;                 /* SwiGLU width */
+  int32_t V;                 /* vocabulary (rows of the LM head) */
+  int32_t mask_id;           /* token id whose embedding fills block rows 1..k-1 */
+  float rms_eps;
+  int32_t page_size;         /* tokens per KV page (16) */
+  int32_t max_batch;         /* largest B a step may carry */
+  int32_t max_k;             /* largest k a step may carry, <= HSPEC_MAX_K */
+  int32_t max_pages_per_req; /* largest page-table row length (bounds the context) */
+} hspec_config;
+
+/* A named tensor in DEVICE memory.  The library borrows the pointer: it must stay valid and
+ * unchanged until hspec_destroy.  Names (l = layer index):
+ *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D]
+ *   layers.l.mamba.{norm [D], in_proj [Di + (Di+2GN) + (dt_rank or H), D] (rows z | xBC | dt),
+ *                   dt_up [H, dt_rank] (only if dt_rank>0), conv_w [Di+2GN, d_conv], conv_b [Di+2GN],
+ *                   dt_bias [H], A_log [H], Dskip [H], gnorm [Di], out_proj [D, Di]}
+ *   layers.l.attn.{norm [D], wqkv [(Hq+2Hkv)*dh, D] (rows q | k | v), q_norm [dh], k_norm [dh], wo [D, Hq*dh]}
+ *   layers.l.mlp.{norm [D], w_gate_up [2F, D] (rows gate | up), w_down [D, F]}
+ * Matrices must be HSPEC_BF16 with a 16-byte aligned base; vectors HSPEC_F32. */
+typedef struct {
+  const char* name;      /* host, NUL-terminated */
+  const void* data;      /* device */
+  int32_t dtype;         /* hspec_dtype */
+  int32_t ndim;          /* 1 or 2 */
+  int64_t shape[2];
+} hspec_tensor;
+
+/* Inputs of one step (the paper's drafter inputs: last-position hidden states, the target's KV
+ * cache in place, the last sampled token; Sec. 3.2 / 3.3). */
+typedef struct {
+  int32_t B;                     /* requests, 1..max_batch */
+  int32_t k;                     /* block positions = draft tokens emitted, 1..max_k */
+  const int32_t* page_table;     /* device int32 [B, page_table_stride]: logical page j of request b -> physical page.
+                                    Entries at or past ceil(ctx/page_size) are never read. */
+  int32_t page_table_stride;     /* row pitch in elements, <= max_pages_per_req */
+  const int32_t* ctx_lens;       /* device int32 [B]: tokens of request b already in the target cache (>= 0) */
+  int32_t max_ctx;               /* host: an upper bound on every ctx_lens[b]; 0 = page_table_stride*page_size.
+                                    Only used to size the split of long contexts; a loose bound costs idle CTAs. */
+  const void* last_hidden;       /* device bf16 [B, n_fuse*D]: target hidden state(s) at the last input position */
+  const int32_t* last_token;     /* device int32 [B]: last accepted token id (block row 0) */
+  const void* const* k_pools;    /* HOST array of n_slots device pointers, each bf16 [num_pages, page_size, Hkv, dh];
+                                    keys are stored already rotated by the target.  Never written. */
+  const void* const* v_pools;    /* same for values */
+  int64_t num_pages;             /* pages in each pool */
+  void* stream;                  /* cudaStream_t (0 = default stream) */
+  void* workspace;               /* device scratch, >= hspec_workspace_bytes(cfg), 1024-byte aligned; owned by the caller,
+                                    contents undefined between calls */
+  size_t workspace_bytes;
+} hspec_step;
+
+/* Outputs of one step, device memory owned by the caller. */
+typedef struct {
+  int32_t* draft_ids;   /* int32 [B, k], required: arg-max of the logits, lowest index on ties */
+  float* logits;        /* fp32 [B, k, V] or NULL (then the logits are never materialised) */
+  float* hidden;        /* fp32 [B, k, D] or NULL: the residual stream before the final norm */
+} hspec_out;
+
+typedef struct hspec_handle hspec_handle;
+
+typedef struct {
+  uint64_t kernel_launches;   /* kernels this handle enqueued since it was created */
+  uint32_t device_status;     /* 0, or a code written by a bounded in-kernel wait that gave up
+                                 (reading it synchronises the handle's last stream) */
+  uint32_t launches_last_step;
+} hspec_stats;
+
+/* Validates the config, creates the handle (host memory only; no weights yet).  Sec. 3.3 / App. B.1. */
+int hspec_init(const hspec_config* cfg, hspec_handle** out);
+/* Device scratch bytes a step of up to (max_batch, max_k, max_pages_per_req) needs. */
+size_t hspec_workspace_bytes(const hspec_config* cfg);
+/* Registers n named device tensors (may be called several times).  Shapes are checked against the config. */
+int hspec_load_weights(hspec_handle* h, const hspec_tensor* tensors, int32_t n);
+/* Enqueues one block-parallel draft step (Sec. 3.3) on in->stream.  Needs every tensor loaded. */
+int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* out);
+/* Frees the handle.  Borrowed tensors, pools and the workspace stay the caller's. */
+int hspec_destroy(hspec_handle* h);
+/* Message of the last failure on this handle (or of the last failed hspec_init if h is NULL). */
+const char* hspec_last_error(const hspec_handle* h);
+int hspec_get_stats(hspec_handle* h, hspec_stats* out);
+
+/* ------------------------------------------------------------------------------------------------
+ * Single-operation entry points: the same kernels the step uses, exposed one at a time so that each
+ * can be checked against its definition.  All pointers are DEVICE pointers unless stated; all calls
+ * enqueue on `stream` and do not synchronise.
+ * ---------------------------------------------------------------------------------------------- */
+
+/* y[M, n_out] = x[M, K] W[n_out, K]^T, x and W bf16, fp32 accumulation (every linear map of Sec. 3.3).
+ * out_dtype HSPEC_F32 or HSPEC_BF16; ldy = row pitch of y in elements.  accumulate != 0 (fp32 only):
+ * y += result (the residual form).  splits <= 0 lets the library choose how many K-slices to use;
+ * `workspace` (>= hspec_gemm_workspace_bytes) is needed when more than one slice is used.
+ * Needs K % 8 == 0, 16-byte aligned x and W. */
+int hspec_op_gemm(const void* x, const void* W, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,
+                  int32_t out_dtype, int32_t accumulate, int32_t splits, void* workspace, size_t workspace_bytes,
+                  void* stream);
+size_t hspec_gemm_workspace_bytes(int32_t M, int32_t n_out, int32_t K);
+/* LM head fused with arg-max (App. B.2): ids[m] = lowest index of max_v x[m,:] . W[v,:]; logits fp32 [M, V] or NULL. */
+int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t* ids, float* logits, int32_t M, int32_t V,
+                            int32_t K, void* workspace, size_t workspace_bytes, void* stream);
+/* RMSNorm over the last axis: y bf16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
+int hspec_op_rmsnorm(const float* x, const float* w, void* y_bf16, int32_t M, int32_t n, float eps, void* stream);
+/* Mamba-2 mixer core for B requests x k rows (Sec. 3.3.1): causal depthwise conv + SiLU on xBC (zero left
+ * context), dt = softplus(dt_raw + dt_bias), decay exp(dt * -exp(A_log)), the selective recurrence over the
+ * k rows started from s_init, the D skip, and the SiLU(z) gate.
+ *   zxbcdt fp32 [B*k, ld_in]: columns z [Di] | xBC [Di + 2GN] (| dt [H] when dt_raw is NULL)
+ *   dt_raw fp32 [B*k, H] or NULL;  s_init bf16 [B, H, P, N] or NULL (zero state)
+ *   y_gated fp32 [B*k, Di] = (scan output) * SiLU(z). */
+int hspec_op_mamba_scan(const float* zxbcdt, int64_t ld_in, const float* dt_raw, const void* s_init,
+                        const float* conv_w, const float* conv_b, const float* dt_bias, const float* A_log,
+                        const float* Dskip, float* y_gated, int32_t B, int32_t k, int32_t Di, int32_t P,
+                        int32_t N, int32_t G, int32_t d_conv, void* stream);
+/* Per-head RMSNorm (optional) + rotate-half RoPE at positions ctx_lens[b] + i (Sec. 3.3.2, positional alignment).
+ * qkv fp32 [B*k, (Hq+2Hkv)*dh] (q | k | v) -> q bf16 [B*k, Hq, dh], kb bf16 [B*k, Hkv, dh], vb bf16 [B*k, Hkv, dh]. */
+int hspec_op_qk_norm_rope(const float* qkv, const float* q_norm_w, const float* k_norm_w, const int32_t* ctx_lens,
+                          void* q, void* kb, void* vb, int32_t B, int32_t k, int32_t Hq, int32_t Hkv, int32_t dh,
+                          float theta, float eps, int32_t qk_norm, void* stream);
+/* Block-query GQA attention over the target's paged KV (read in place) plus the block's causal keys (Sec. 3.3.2).
+ * q/kb/vb as produced by hspec_op_qk_norm_rope; k_pool/v_pool bf16 [num_pages, page_size, Hkv, dh];
+ * o bf16 [B*k, Hq*dh].  window 0 = full.  max_ctx: host upper bound on ctx_lens (0 = stride*page_size).
+ * chunk_tokens <= 0 lets the library pick the context split. */
+int hspec_op_attention(const void* q, const void* kb, const void* vb, const void* k_pool, const void* v_pool,
+                       const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens,
+                       int32_t max_ctx, void* o, int32_t B, int32_t k, int32_t Hq, int32_t Hkv, int32_t dh,
+                       int32_t page_size, int32_t window, int32_t chunk_tokens, void* workspace,
+                       size_t workspace_bytes, void* stream);
+size_t hspec_attention_workspace_bytes(int32_t B, int32_t k, int32_t Hq, int32_t Hkv, int32_t dh, int32_t max_ctx,
+                                       int32_t window, int32_t chunk_tokens);
+/* Contiguous copy of one request's prefix out of a paged pool: dst bf16 [ctx_len, Hkv, dh] (pure data movement,
+ * bit-exact; used to check the page-table addressing of the attention kernel, Sec. 3.3.2). */
+int hspec_debug_gather_kv(const void* pool, const int32_t* page_table_row, int32_t ctx_len, int32_t page_size,
+                          int32_t Hkv, int32_t dh, void* dst, void* stream);
+/* h bf16 [M, F] = SiLU(gu[:, :F]) * gu[:, F:], gu fp32 [M, 2F] (App. B.1 "MLP"). */
+int hspec_op_swiglu(const float* gu, void* h_bf16, int32_t M, int32_t F, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HSPEC_H_ */

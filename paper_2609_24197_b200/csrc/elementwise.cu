@@ -1,0 +1,165 @@
+// Row-wise and element-wise kernels of the draft step (all fp32 math; bf16 only where a tensor-core
+// operand is produced).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace hspec {
+
+namespace {
+
+// Block rows: row 0 of each request is the embedding of its last token, rows 1..k-1 the mask-token
+// embedding; no positional embedding is added (paper Sec. 3.3.1).
+__global__ void embed_rows_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ last_token,
+                                  int mask_id, float* __restrict__ X, int k, int D) {
+  const int m = blockIdx.x;
+  const int b = m / k, i = m % k;
+  const int tok = (i == 0) ? last_token[b] : mask_id;
+  const __nv_bfloat16* src = embed + size_t(tok) * D;
+  float* dst = X + size_t(m) * D;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = __bfloat162float(src[d]);
+}
+
+__device__ __forceinline__ float block_sum(float v, float* red) {
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+  const int warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  if ((threadIdx.x & 31) == 0) red[warp] = v;
+  __syncthreads();
+  float t = (threadIdx.x < nw) ? red[threadIdx.x] : 0.f;
+  if (warp == 0) {
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    if (threadIdx.x == 0) red[0] = t;
+  }
+  __syncthreads();
+  const float r = red[0];
+  __syncthreads();
+  return r;
+}
+
+// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, bf16 out.
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __nv_bfloat16* __restrict__ y,
+                               int n, float eps) {
+  __shared__ float red[32];
+  const float* xr = x + size_t(blockIdx.x) * n;
+  float ss = 0.f;
+  for (int d = threadIdx.x; d < n; d += blockDim.x) { const float v = xr[d]; ss += v * v; }
+  const float tot = block_sum(ss, red);
+  const float inv = rsqrtf(tot / float(n) + eps);
+  __nv_bfloat16* yr = y + size_t(blockIdx.x) * n;
+  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = __float2bfloat16_rn(xr[d] * inv * w[d]);
+}
+
+// Per (row, head): optional RMSNorm over dh, then rotate-half RoPE at position ctx_len + i.
+// The angle is one fp32 product pos * inv_freq[j]; sin/cos are the accurate library versions.
+// blockIdx.x = row m, blockIdx.y = head index over q heads then k heads then v heads (v is only converted).
+__global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* __restrict__ qw,
+                                    const float* __restrict__ kw, const float* __restrict__ inv_freq,
+                                    const int32_t* __restrict__ ctx_lens, __nv_bfloat16* __restrict__ q,
+                                    __nv_bfloat16* __restrict__ kb, __nv_bfloat16* __restrict__ vb, int k, int Hq,
+                                    int Hkv, int dh, float eps, int qk_norm) {
+  const int m = blockIdx.x, hh = blockIdx.y;
+  const int lane = threadIdx.x;                       // one warp per (row, head)
+  const float* src = qkv + size_t(m) * (Hq + 2 * Hkv) * dh + size_t(hh) * dh;
+  const int half = dh / 2;
+  if (hh >= Hq + Hkv) {                               // values: plain conversion
+    __nv_bfloat16* dst = vb + (size_t(m) * Hkv + (hh - Hq - Hkv)) * dh;
+    for (int d = lane; d < dh; d += 32) dst[d] = __float2bfloat16_rn(src[d]);
+    return;
+  }
+  const bool is_q = hh < Hq;
+  const float* w = is_q ? qw : kw;
+  float inv = 1.f;
+  if (qk_norm) {
+    float ss = 0.f;
+    for (int d = lane; d < dh; d += 32) { const float v = src[d]; ss += v * v; }
+    for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    inv = rsqrtf(ss / float(dh) + eps);
+  }
+  const float pos = float(ctx_lens[m / k] + m % k);
+  __nv_bfloat16* dst = is_q ? q + (size_t(m) * Hq + hh) * dh : kb + (size_t(m) * Hkv + (hh - Hq)) * dh;
+  for (int j = lane; j < half; j += 32) {
+    float v1 = src[j] * inv, v2 = src[j + half] * inv;
+    if (qk_norm) { v1 *= w[j]; v2 *= w[j + half]; }
+    float sn, cs;
+    sincosf(pos * inv_freq[j], &sn, &cs);
+    dst[j] = __float2bfloat16_rn(v1 * cs - v2 * sn);
+    dst[j + half] = __float2bfloat16_rn(v2 * cs + v1 * sn);
+  }
+}
+
+__global__ void swiglu_kernel(const float* __restrict__ gu, __nv_bfloat16* __restrict__ h, int M, int F) {
+  const long long total = (long long)M * F;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int m = int(idx / F), f = int(idx % F);
+    const float gte = gu[size_t(m) * 2 * F + f], up = gu[size_t(m) * 2 * F + F + f];
+    h[idx] = __float2bfloat16_rn(silu_f(gte) * up);
+  }
+}
+
+__global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, size_t n) {
+  for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x)
+    dst[i] = src[i];
+}
+
+// inv_freq table per (theta, dh): theta^(-2j/dh) evaluated in double, rounded to fp32, kept on the device.
+struct RopeTable { float theta; int dh; float* dev; };
+RopeTable g_rope[8];
+int g_n_rope = 0;
+
+const float* rope_table(float theta, int dh, cudaStream_t stream) {
+  for (int i = 0; i < g_n_rope; ++i)
+    if (g_rope[i].theta == theta && g_rope[i].dh == dh) return g_rope[i].dev;
+  if (g_n_rope == 8) return nullptr;
+  float host[128];
+  const int half = dh / 2;
+  for (int j = 0; j < half; ++j) host[j] = float(pow(double(theta), -2.0 * double(j) / double(dh)));
+  float* dev = nullptr;
+  if (cudaMalloc(&dev, sizeof(float) * half) != cudaSuccess) return nullptr;
+  if (cudaMemcpy(dev, host, sizeof(float) * half, cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
+  (void)stream;
+  g_rope[g_n_rope++] = RopeTable{theta, dh, dev};
+  return dev;
+}
+
+int grid_for(long long total, int threads) {
+  long long b = (total + threads - 1) / threads;
+  return int(b > 148 * 16 ? 148 * 16 : (b < 1 ? 1 : b));
+}
+
+}  // namespace
+
+cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
+                              int D, cudaStream_t stream) {
+  embed_rows_kernel<<<B * k, 256, 0, stream>>>((const __nv_bfloat16*)embed_bf16, last_token, mask_id, X, k, D);
+  return cudaGetLastError();
+}
+
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_bf16, int M, int n, float eps, cudaStream_t stream) {
+  const int threads = n >= 2048 ? 512 : 256;
+  rmsnorm_kernel<<<M, threads, 0, stream>>>(x, w, (__nv_bfloat16*)y_bf16, n, eps);
+  return cudaGetLastError();
+}
+
+cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
+                                void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
+                                int qk_norm, cudaStream_t stream) {
+  if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
+  const float* tab = rope_table(theta, dh, stream);
+  if (!tab) return cudaErrorMemoryAllocation;
+  dim3 grid(B * k, Hq + 2 * Hkv);
+  qk_norm_rope_kernel<<<grid, 32, 0, stream>>>(qkv, qw, kw, tab, ctx_lens, (__nv_bfloat16*)q, (__nv_bfloat16*)kb,
+                                               (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps, qk_norm);
+  return cudaGetLastError();
+}
+
+cudaError_t swiglu_launch(const float* gu, void* h_bf16, int M, int F, cudaStream_t stream) {
+  swiglu_kernel<<<grid_for((long long)M * F, 256), 256, 0, stream>>>(gu, (__nv_bfloat16*)h_bf16, M, F);
+  return cudaGetLastError();
+}
+
+cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream) {
+  copy_f32_kernel<<<grid_for((long long)n, 256), 256, 0, stream>>>(src, dst, n);
+  return cudaGetLastError();
+}
+
+}  // namespace hspec

@@ -1,0 +1,386 @@
+// bf16 GEMM y = x W^T on the 5th-generation tensor cores (tcgen05 + TMEM + TMA), sm_100a.
+//
+// Every dense map of the draft step is "few activation rows times a tall weight matrix".  The
+// weight rows therefore sit on the MMA's M side (128 output features per CTA = 128 TMEM lanes) and
+// the activation rows on its N side (BN = 16..256 rows = BN TMEM columns), so a step with one
+// request and a step with 256 requests run the same kernel: the accumulator tile is y^T.
+//
+//   warp 0 : TMA producer  (weights [128 x 64] and activations [BN x 64] per stage, 128-byte swizzle)
+//   warp 1 : allocates TMEM, issues tcgen05.mma (one elected thread), commits stages back
+//   warps 2..5 : epilogue, one TMEM lane quarter each: tcgen05.ld -> registers -> global
+//
+// Epilogues: fp32 / bf16 store, fp32 accumulate-into (residual), fp32 K-slice partial, and the
+// LM-head form that reduces each activation row's (max, index) over the CTA's 128 vocabulary rows.
+#include "common.cuh"
+#include "kernels.h"
+
+#include <cuda.h>
+
+namespace hspec {
+
+namespace {
+
+constexpr int TILE_W = 128;       // weight rows per CTA (UMMA M)
+constexpr int TILE_K = 64;        // bf16 elements per stage along K = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr uint32_t A_STAGE_BYTES = TILE_W * TILE_K * 2;   // 16 KiB
+
+struct __align__(8) GemmSmemTail {
+  uint64_t full[GEMM_MAX_STAGES];
+  uint64_t empty[GEMM_MAX_STAGES];
+  uint64_t tmem_full;
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+  float red_val[4][256];   // LM-head epilogue: per lane-quarter (max, index) of each activation row
+  int red_idx[4][256];
+};
+
+__global__ void __launch_bounds__(192, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g) {
+  extern __shared__ uint8_t smem_raw[];
+  // 128-byte swizzle needs 1024-byte aligned tiles
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t b_stage_bytes = g.BN * TILE_K * 2;
+  const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  GemmSmemTail* tail = reinterpret_cast<GemmSmemTail*>(smem + size_t(g.stages) * stage_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile_m = blockIdx.x;            // activation-row tile (fastest: CTAs sharing a weight tile run together)
+  const int tile_n = blockIdx.y;            // weight-row tile
+  const int split = blockIdx.z;
+  const int kt_begin = split * g.k_tiles_per_split;
+  const int kt_end = min(g.k_tiles_total, kt_begin + g.k_tiles_per_split);
+  const int n_kt = kt_end - kt_begin;       // >= 1 by construction of the grid
+  const uint32_t tmem_cols = g.tmem_cols;
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    for (int s = 0; s < g.stages; ++s) {
+      mbar_init(smem_u32(&tail->full[s]), 1);
+      mbar_init(smem_u32(&tail->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&tail->tmem_full), 1);
+    tail->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&tail->tmem_base), tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_acc = tail->tmem_base;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first();   // weights are streamed once per step
+      const uint64_t pol_x = policy_evict_last();    // activations are re-read by every weight tile
+      for (int i = 0; i < n_kt; ++i) {
+        const int s = i % g.stages;
+        const uint32_t round = i / g.stages;
+        if (round > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (round - 1) & 1)) {
+          atomicExch(g.status, STATUS_TIMEOUT_PRODUCER);
+          atomicExch(&tail->abort_flag, 1u);
+          break;
+        }
+        const uint32_t full = smem_u32(&tail->full[s]);
+        mbar_expect_tx(full, stage_bytes);
+        uint8_t* sa = smem + size_t(s) * stage_bytes;
+        tma_load_2d(smem_u32(sa), &tmA, (kt_begin + i) * TILE_K, tile_n * TILE_W, full, pol_w);
+        tma_load_2d(smem_u32(sa + A_STAGE_BYTES), &tmB, (kt_begin + i) * TILE_K, tile_m * g.BN, full, pol_x);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16_m128(g.BN);
+      bool ok = true;
+      for (int i = 0; i < n_kt && ok; ++i) {
+        const int s = i % g.stages;
+        const uint32_t round = i / g.stages;
+        if (!mbar_wait(smem_u32(&tail->full[s]), round & 1)) {
+          atomicExch(g.status, STATUS_TIMEOUT_MMA);
+          atomicExch(&tail->abort_flag, 1u);
+          ok = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes);
+        const uint64_t da = umma_desc_kmajor_sw128(sa);
+        const uint64_t db = umma_desc_kmajor_sw128(sa + A_STAGE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < TILE_K / UMMA_K; ++kk) {
+          // advancing K inside the swizzle row: +32 bytes = +2 in the descriptor's 16-byte units
+          umma_bf16(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&tail->empty[s]));   // stage reusable once these MMAs have read it
+      }
+      // accumulator complete (or aborted: release the epilogue either way)
+      if (ok) umma_commit(smem_u32(&tail->tmem_full));
+      else mbar_arrive(smem_u32(&tail->tmem_full));
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;                         // TMEM lane quarter this warp may read
+    bool ok = mbar_wait(smem_u32(&tail->tmem_full), 0);
+    if (!ok) atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
+    tc_fence_after();
+    if (*reinterpret_cast<volatile uint32_t*>(&tail->abort_flag)) ok = false;
+    const int n = tile_n * TILE_W + q * 32 + lane;  // output feature (weight row) of this thread
+    const bool n_ok = n < g.N_out;
+    const int m0 = tile_m * g.BN;
+    for (int c0 = 0; c0 < g.BN && ok; c0 += 16) {
+      uint32_t r[16];
+      tmem_ld16(tmem_acc + (uint32_t(q * 32) << 16) + uint32_t(c0), r);
+      tmem_ld_wait();
+      if (g.mode == EPI_STORE_F32 || g.mode == EPI_PARTIAL_F32) {
+        float* out = reinterpret_cast<float*>(g.out) + (g.mode == EPI_PARTIAL_F32 ? size_t(split) * g.M * g.ldo : 0);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __uint_as_float(r[j]);
+        }
+      } else if (g.mode == EPI_ACCUM_F32) {
+        float* out = reinterpret_cast<float*>(g.out);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] += __uint_as_float(r[j]);
+        }
+      } else if (g.mode == EPI_STORE_BF16) {
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(g.out);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
+        }
+      } else {  // EPI_ARGMAX: logits optional, (max, lowest index) over this warp's 32 vocabulary rows
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          float v = n_ok ? __uint_as_float(r[j]) : -INFINITY;
+          if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v;
+          int idx = n;
+#pragma unroll
+          for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+            if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+          }
+          if (lane == 0) { tail->red_val[q][c0 + j] = v; tail->red_idx[q][c0 + j] = idx; }
+        }
+      }
+    }
+    if (g.mode == EPI_ARGMAX) {
+      asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
+      const int t = threadIdx.x - 64;                     // 0..127
+      for (int c = t; c < g.BN; c += 128) {
+        const int m = m0 + c;
+        if (m >= g.M) continue;
+        float v = tail->red_val[0][c];
+        int idx = tail->red_idx[0][c];
+#pragma unroll
+        for (int qq = 1; qq < 4; ++qq) {
+          const float ov = tail->red_val[qq][c];
+          const int oi = tail->red_idx[qq][c];
+          if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+        }
+        if (!ok) { v = -INFINITY; idx = 0x7fffffff; }
+        g.part_val[size_t(tile_n) * g.M + m] = v;
+        g.part_idx[size_t(tile_n) * g.M + m] = idx;
+      }
+    }
+    tc_fence_before();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_acc, tmem_cols);
+  }
+}
+
+// Sum the K-slice partials in slice order (deterministic) and apply the final store.
+__global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, int M, int N, void* out,
+                                     long long ldo, int mode) {
+  const long long total = (long long)M * N;
+  for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int m = int(i / N), n = int(i % N);
+    float acc = 0.f;
+    for (int s = 0; s < splits; ++s) acc += part[(size_t(s) * M + m) * N + n];
+    if (mode == EPI_STORE_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] = acc;
+    else if (mode == EPI_ACCUM_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] += acc;
+    else reinterpret_cast<__nv_bfloat16*>(out)[size_t(m) * ldo + n] = __float2bfloat16_rn(acc);
+  }
+}
+
+// ids[m] = lowest index among the per-tile maxima (tiles are in ascending vocabulary order).
+__global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
+                                     int* __restrict__ ids) {
+  const int m = blockIdx.x;
+  float v = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
+    const float ov = pv[size_t(t) * M + m];
+    const int oi = pi[size_t(t) * M + m];
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = v; si[threadIdx.x >> 5] = idx; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int nw = blockDim.x >> 5;
+    v = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+    idx = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+    }
+    if (threadIdx.x == 0) ids[m] = idx;
+  }
+}
+
+// ------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+int g_smem_optin = -1;
+
+}  // namespace
+
+// 2-D bf16 row-major [rows, cols] tensor, box [box_rows x 64 columns], 128-byte swizzle, zero fill.
+bool make_tmap_bf16_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
+                       int box_rows, std::string* err) {
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { if (err) *err = "cuTensorMapEncodeTiled is not available from the CUDA driver"; return false; }
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || ((ld_elems * 2) & 15)) {
+    if (err) *err = "TMA operand needs a 16-byte aligned base and row pitch";
+    return false;
+  }
+  cuuint64_t dims[2] = {cuuint64_t(cols), cuuint64_t(rows)};
+  cuuint64_t strides[1] = {cuuint64_t(ld_elems) * 2};
+  cuuint32_t box[2] = {cuuint32_t(TILE_K), cuuint32_t(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    if (err) *err = "cuTensorMapEncodeTiled failed with CUresult " + std::to_string(int(r));
+    return false;
+  }
+  return true;
+}
+
+int gemm_pick_bn(int M) {
+  if (M >= 256) return 256;
+  return ((M + 15) / 16) * 16;
+}
+
+int gemm_pick_splits(int M, int n_out, int K, int num_sms) {
+  // Weight streaming (few rows): keep every SM fed.  Many rows: one slice (tensor-bound, no reduction pass).
+  const int k_tiles = (K + TILE_K - 1) / TILE_K;
+  const int tiles = ((n_out + TILE_W - 1) / TILE_W) * ((M + 255) / 256);
+  if (tiles >= num_sms || k_tiles < 8) return 1;
+  int want = (2 * num_sms + tiles - 1) / tiles;
+  int max_by_k = k_tiles / 4;               // at least 4 K-tiles per slice
+  int s = want < max_by_k ? want : max_by_k;
+  if (s > 16) s = 16;
+  return s < 1 ? 1 : s;
+}
+
+size_t gemm_splitk_bytes(int M, int n_out, int splits) {
+  return splits > 1 ? size_t(splits) * M * n_out * sizeof(float) : 0;
+}
+
+// Launches y = x W^T.  tmW must describe W with box rows 128; x is described here (box rows BN).
+cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launches, std::string* err) {
+  if (g_smem_optin < 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         g_smem_optin);
+    if (e != cudaSuccess) return e;
+  }
+  GemmArgs g{};
+  g.M = c.M; g.N_out = c.n_out; g.K = c.K;
+  g.BN = gemm_pick_bn(c.M);
+  g.k_tiles_total = (c.K + TILE_K - 1) / TILE_K;
+  int splits = c.splits < 1 ? 1 : c.splits;
+  if (splits > g.k_tiles_total) splits = g.k_tiles_total;
+  g.k_tiles_per_split = (g.k_tiles_total + splits - 1) / splits;
+  splits = (g.k_tiles_total + g.k_tiles_per_split - 1) / g.k_tiles_per_split;   // no empty slice
+  uint32_t cols = 32;
+  while (cols < uint32_t(g.BN)) cols <<= 1;
+  g.tmem_cols = cols;
+  const size_t stage_bytes = A_STAGE_BYTES + size_t(g.BN) * TILE_K * 2;
+  const size_t fixed = sizeof(GemmSmemTail) + 1024;
+  int stages = int((size_t(g_smem_optin) - fixed) / stage_bytes);
+  if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
+  if (stages > g.k_tiles_per_split) stages = g.k_tiles_per_split < 2 ? 2 : g.k_tiles_per_split;
+  if (stages < 2) { if (err) *err = "shared memory too small for the GEMM pipeline"; return cudaErrorInvalidValue; }
+  g.stages = stages;
+  g.status = c.status;
+  g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx;
+  g.ldo = c.ldo;
+  if (splits > 1) {
+    if (c.mode == EPI_ARGMAX) { if (err) *err = "LM-head epilogue cannot be K-sliced"; return cudaErrorInvalidValue; }
+    if (c.splitk_ws == nullptr || c.splitk_ws_bytes < gemm_splitk_bytes(c.M, c.n_out, splits)) {
+      if (err) *err = "K-slice workspace too small";
+      return cudaErrorInvalidValue;
+    }
+    g.mode = EPI_PARTIAL_F32; g.out = c.splitk_ws; g.ldo = c.n_out;
+  } else {
+    g.mode = c.mode; g.out = c.out;
+  }
+  CUtensorMap tmB;
+  if (!make_tmap_bf16_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BN, err)) return cudaErrorInvalidValue;
+  dim3 grid((c.M + g.BN - 1) / g.BN, (c.n_out + TILE_W - 1) / TILE_W, splits);
+  const size_t smem = size_t(stages) * stage_bytes + fixed;
+  gemm_tcgen05_kernel<<<grid, 192, smem, stream>>>(*c.tmW, tmB, g);
+  if (launches) ++*launches;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  if (splits > 1) {
+    const long long total = (long long)c.M * c.n_out;
+    int blocks = int((total + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M,
+                                                     c.n_out, c.out, c.ldo, c.mode);
+    if (launches) ++*launches;
+    e = cudaGetLastError();
+  }
+  return e;
+}
+
+cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
+                                 uint64_t* launches) {
+  argmax_reduce_kernel<<<M, 256, 0, stream>>>(pv, pi, n_tiles, M, ids);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace hspec

@@ -1,0 +1,103 @@
+// Internal interfaces between the kernel files and the C ABI layer (not exported).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+
+namespace hspec {
+
+constexpr int GEMM_MAX_STAGES = 8;
+
+enum GemmEpilogue : int {
+  EPI_STORE_F32 = 0,    // y fp32 = acc
+  EPI_STORE_BF16 = 1,   // y bf16 = acc
+  EPI_ACCUM_F32 = 2,    // y fp32 += acc   (residual)
+  EPI_PARTIAL_F32 = 3,  // K-slice partial (internal)
+  EPI_ARGMAX = 4,       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
+};
+
+struct GemmArgs {       // kernel argument block
+  int M, N_out, K;
+  int BN;               // activation rows per CTA = UMMA N (multiple of 16, <= 256)
+  int k_tiles_total, k_tiles_per_split;
+  int stages;
+  uint32_t tmem_cols;
+  int mode;
+  void* out;
+  long long ldo;
+  float* logits;
+  float* part_val;
+  int* part_idx;
+  uint32_t* status;
+};
+
+struct GemmCall {       // host-side description of one y = x W^T
+  const CUtensorMap* tmW;   // weights [n_out, K], box 128 x 64
+  const void* x;            // bf16 [M, K], row pitch ldx elements
+  long long ldx;
+  int M, n_out, K;
+  int mode;                 // EPI_STORE_F32 / EPI_STORE_BF16 / EPI_ACCUM_F32 / EPI_ARGMAX
+  void* out;
+  long long ldo;
+  int splits;
+  void* splitk_ws;
+  size_t splitk_ws_bytes;
+  float* logits;            // EPI_ARGMAX only (may be null)
+  float* part_val;
+  int* part_idx;
+  uint32_t* status;
+};
+
+bool make_tmap_bf16_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
+                       int box_rows, std::string* err);
+int gemm_pick_bn(int M);
+int gemm_pick_splits(int M, int n_out, int K, int num_sms);
+size_t gemm_splitk_bytes(int M, int n_out, int splits);
+cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
+                                 uint64_t* launches);
+
+// ---- attention (attention.cu)
+struct AttnCall {
+  const void *q, *kb, *vb;          // bf16 [B*k, Hq, dh], [B*k, Hkv, dh] x2
+  const void *k_pool, *v_pool;      // bf16 [num_pages, page, Hkv, dh]
+  const int32_t* page_table;
+  int page_table_stride;
+  const int32_t* ctx_lens;
+  int max_ctx;                      // host bound on ctx_lens
+  void* o;                          // bf16 [B*k, Hq*dh]
+  int B, k, Hq, Hkv, dh, page_size, window;
+  int chunk_tokens;                 // <= 0: choose
+  void* ws;
+  size_t ws_bytes;
+};
+int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms);
+size_t attn_workspace_bytes(int B, int k, int Hq, int Hkv, int dh, int max_ctx, int window, int chunk_tokens);
+cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+cudaError_t gather_kv_launch(const void* pool, const int32_t* row, int ctx_len, int page_size, int Hkv, int dh,
+                             void* dst, cudaStream_t stream);
+
+// ---- scan (scan.cu)
+struct ScanCall {
+  const float* zxbcdt; long long ld_in;
+  const float* dt_raw;              // [B*k, H] or null (then the dt columns of zxbcdt)
+  const void* s_init;               // bf16 [B, H, P, N] or null
+  const float *conv_w, *conv_b, *dt_bias, *A_log, *Dskip;
+  float* y_gated;                   // [B*k, Di]
+  int B, k, Di, P, N, G, d_conv;
+};
+cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+
+// ---- element-wise kernels (elementwise.cu)
+cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
+                              int D, cudaStream_t stream);
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_bf16, int M, int n, float eps, cudaStream_t stream);
+cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
+                                void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
+                                int qk_norm, cudaStream_t stream);
+cudaError_t swiglu_launch(const float* gu, void* h_bf16, int M, int F, cudaStream_t stream);
+cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream);
+
+}  // namespace hspec

@@ -1,0 +1,172 @@
+// Mamba-2 mixer core over the k block rows, started from the injected state (paper Sec. 3.3.1).
+//
+// One CTA per (request, head).  Because the recurrence S_i = a_i S_{i-1} + dt_i x_i B_i^T is linear,
+// all k positions are evaluated in one pass without carrying the state:
+//   y_t = exp(c_t) * (S_init C_t)  +  sum_{s<=t} exp(c_t - c_s) dt_s (C_t . B_s) x_s  +  D x_t,
+//   c_t = sum_{r<=t} dt_r A   (inclusive prefix sum over the block positions, one warp shuffle scan).
+// S_init (bf16 [P, N] per head) is read from HBM exactly once with 16-byte loads; it is the only
+// large operand, so the kernel is bound by that read.  The causal depthwise conv + SiLU of x, B, C
+// (zero left context), softplus(dt), the D skip and the SiLU(z) gate are fused around it.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace hspec {
+
+namespace {
+
+constexpr int SCAN_THREADS = 128;
+constexpr int KMAX = 32;
+
+struct ScanArgs {
+  const float* zxbcdt; long long ld_in;
+  const float* dt_raw;
+  const __nv_bfloat16* s_init;
+  const float *conv_w, *conv_b, *dt_bias, *A_log, *Dskip;
+  float* y;
+  int B, k, Di, P, N, G, H, d_conv, d_xBC;
+  int NP;          // padded N (row pitch of the staged state in floats)
+};
+
+__device__ __forceinline__ float softplus_f(float v) { return v > 20.f ? v : log1pf(expf(v)); }
+
+__global__ void __launch_bounds__(SCAN_THREADS)
+mamba_scan_kernel(ScanArgs a) {
+  extern __shared__ __align__(16) float sm[];
+  const int tid = threadIdx.x;
+  const int h = blockIdx.x, b = blockIdx.y;
+  const int g = h / (a.H / a.G);
+  const int k = a.k, P = a.P, N = a.N;
+  float* xs = sm;                    // [k][P]
+  float* Bs = xs + KMAX * P;         // [k][N]
+  float* Cs = Bs + KMAX * N;         // [k][N]
+  float* Wm = Cs + KMAX * N;         // [k][k]  exp(c_t - c_s) dt_s (C_t . B_s), s <= t
+  float* dec = Wm + KMAX * KMAX;     // [k]     exp(c_t)
+  float* dts = dec + KMAX;           // [k]
+  float* cum = dts + KMAX;           // [k]
+  float* Ss = cum + KMAX;            // [P][NP] staged S_init (fp32)
+  const size_t row0 = size_t(b) * k;
+
+  // ---- conv + SiLU for this head's x channels and its group's B, C channels
+  const int n_ch = P + 2 * N;
+  for (int idx = tid; idx < k * n_ch; idx += SCAN_THREADS) {
+    const int i = idx / n_ch, cc = idx % n_ch;
+    int ch;                          // channel inside xBC
+    if (cc < P) ch = h * P + cc;
+    else if (cc < P + N) ch = a.Di + g * N + (cc - P);
+    else ch = a.Di + a.G * N + g * N + (cc - P - N);
+    float acc = a.conv_b[ch];
+    for (int j = 0; j < a.d_conv; ++j) {
+      const int src = i - (a.d_conv - 1) + j;
+      if (src >= 0) acc += a.conv_w[ch * a.d_conv + j] * a.zxbcdt[(row0 + src) * a.ld_in + a.Di + ch];
+    }
+    const float v = silu_f(acc);
+    if (cc < P) xs[i * P + cc] = v;
+    else if (cc < P + N) Bs[i * N + (cc - P)] = v;
+    else Cs[i * N + (cc - P - N)] = v;
+  }
+  // ---- dt, cumulative log-decay (warp 0: inclusive shuffle scan over the k <= 32 positions)
+  if (tid < 32) {
+    float dt = 0.f, dA = 0.f;
+    if (tid < k) {
+      const float raw = a.dt_raw ? a.dt_raw[(row0 + tid) * a.H + h]
+                                 : a.zxbcdt[(row0 + tid) * a.ld_in + a.Di + a.d_xBC + h];
+      dt = softplus_f(raw + a.dt_bias[h]);
+      dA = dt * (-expf(a.A_log[h]));
+    }
+    float c = dA;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const float up = __shfl_up_sync(0xffffffffu, c, off);
+      if (tid >= off) c += up;
+    }
+    if (tid < k) { dts[tid] = dt; cum[tid] = c; dec[tid] = expf(c); }
+  }
+  // ---- stage S_init[b, h] (bf16 -> fp32), 16-byte loads
+  if (a.s_init != nullptr) {
+    const __nv_bfloat16* src = a.s_init + (size_t(b) * a.H + h) * P * N;
+    if ((N & 7) == 0) {
+      const int vec = P * N / 8;
+      for (int idx = tid; idx < vec; idx += SCAN_THREADS) {
+        const uint4 raw = reinterpret_cast<const uint4*>(src)[idx];
+        const int p = (idx * 8) / N, n = (idx * 8) % N;
+        float* d = Ss + p * a.NP + n;
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          d[2 * e] = __uint_as_float(w[e] << 16);
+          d[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+        }
+      }
+    } else {
+      for (int idx = tid; idx < P * N; idx += SCAN_THREADS)
+        Ss[(idx / N) * a.NP + idx % N] = __bfloat162float(src[idx]);
+    }
+  }
+  __syncthreads();
+  // ---- W[t][s] = exp(c_t - c_s) dt_s (C_t . B_s) for s <= t
+  for (int idx = tid; idx < k * k; idx += SCAN_THREADS) {
+    const int t = idx / k, s = idx % k;
+    float w = 0.f;
+    if (s <= t) {
+      float dot = 0.f;
+      for (int n = 0; n < N; ++n) dot += Cs[t * N + n] * Bs[s * N + n];
+      w = expf(cum[t] - cum[s]) * dts[s] * dot;
+    }
+    Wm[t * KMAX + s] = w;
+  }
+  __syncthreads();
+  // ---- outputs: thread owns head channel p for all k positions
+  const float Dh = a.Dskip[h];
+  for (int p = tid; p < P; p += SCAN_THREADS) {
+    float acc[KMAX];
+#pragma unroll
+    for (int t = 0; t < KMAX; ++t) acc[t] = 0.f;
+    if (a.s_init != nullptr) {
+      const float* srow = Ss + p * a.NP;
+      for (int n = 0; n < N; ++n) {
+        const float sv = srow[n];
+#pragma unroll
+        for (int t = 0; t < KMAX; ++t)
+          if (t < k) acc[t] += Cs[t * N + n] * sv;
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < KMAX; ++t) {
+      if (t < k) {
+        float y = dec[t] * acc[t] + Dh * xs[t * P + p];
+        for (int s = 0; s <= t; ++s) y += Wm[t * KMAX + s] * xs[s * P + p];
+        const size_t row = row0 + t;
+        const float z = a.zxbcdt[row * a.ld_in + h * P + p];
+        a.y[row * a.Di + h * P + p] = y * silu_f(z);
+      }
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launches, std::string* err) {
+  if (c.k < 1 || c.k > KMAX) { if (err) *err = "scan: k out of range"; return cudaErrorInvalidValue; }
+  if (c.Di % c.P) { if (err) *err = "scan: Di must be a multiple of P"; return cudaErrorInvalidValue; }
+  ScanArgs a{};
+  a.zxbcdt = c.zxbcdt; a.ld_in = c.ld_in; a.dt_raw = c.dt_raw; a.s_init = (const __nv_bfloat16*)c.s_init;
+  a.conv_w = c.conv_w; a.conv_b = c.conv_b; a.dt_bias = c.dt_bias; a.A_log = c.A_log; a.Dskip = c.Dskip;
+  a.y = c.y_gated; a.B = c.B; a.k = c.k; a.Di = c.Di; a.P = c.P; a.N = c.N; a.G = c.G; a.H = c.Di / c.P;
+  a.d_conv = c.d_conv; a.d_xBC = c.Di + 2 * c.G * c.N;
+  a.NP = c.N + 1;                                    // odd pitch: threads of a warp own consecutive p
+  if (a.H % c.G) { if (err) *err = "scan: heads must divide into groups"; return cudaErrorInvalidValue; }
+  const size_t smem = sizeof(float) * (size_t(KMAX) * c.P + 2 * size_t(KMAX) * c.N + KMAX * KMAX + 3 * KMAX +
+                                       size_t(c.P) * a.NP);
+  static size_t smem_set = 0;
+  if (smem > 48 * 1024 && smem > smem_set) {
+    cudaError_t e = cudaFuncSetAttribute(mamba_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    if (e != cudaSuccess) { if (err) *err = "scan: state tile does not fit in shared memory"; return e; }
+    smem_set = smem;
+  }
+  dim3 grid(a.H, c.B);
+  mamba_scan_kernel<<<grid, SCAN_THREADS, smem, stream>>>(a);
+  if (launches) ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace hspec

@@ -1,0 +1,260 @@
+"""Parity of each CUDA kernel, called through the C ABI, against the oracle's definition of the op."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import hspec_oracle as O
+from conftest import to_np
+from harness import assert_close, bf16_round
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def hs():
+    import paper_2609_24197_b200 as m
+    from paper_2609_24197_b200 import build
+    build.build()
+    m.load_library()
+    return m
+
+
+def _randn(shape, seed, std=1.0, dtype=torch.float32):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std).to(dtype)
+
+
+# ------------------------------------------------------------------------------ page gather
+@pytest.mark.parametrize("ctx", [0, 1, 15, 16, 17, 40, 1000])
+def test_gather_kv_bit_exact(hs, ctx):
+    Hkv, dh = 2, 64
+    n_pages = (ctx + 15) // 16 + 3
+    g = torch.Generator().manual_seed(ctx)
+    pool = torch.randint(0, 65536, (n_pages, 16, Hkv, dh), generator=g, dtype=torch.int32).to(torch.uint16)
+    row = torch.randperm(n_pages, generator=g)[:max(1, (ctx + 15) // 16)].to(torch.int32)
+    dst = torch.zeros((max(ctx, 1), Hkv, dh), dtype=torch.bfloat16, device="cuda")
+    hs.hspec_debug_gather_kv(pool.view(torch.bfloat16).cuda(), row.cuda(), ctx, dst)
+    torch.cuda.synchronize()
+    ref = O.gather_kv(pool.numpy(), row.numpy(), ctx)
+    np.testing.assert_array_equal(dst[:ctx].cpu().view(torch.uint16).numpy(), ref)
+
+
+# ------------------------------------------------------------------------------ GEMM
+GEMM_CASES = [
+    (1, 256, 64), (8, 1064, 256), (16, 1024, 256), (48, 300, 16), (5, 128, 4096), (200, 384, 4096),
+    (256, 640, 128), (257, 130, 1024), (513, 256, 320), (33, 17536 // 8, 520),
+]
+
+
+@pytest.mark.parametrize("M,n_out,K", GEMM_CASES)
+@pytest.mark.parametrize("mode", ["f32", "bf16", "accum", "split3"])
+def test_gemm(hs, M, n_out, K, mode):
+    x = _randn((M, K), 1, 1.0, torch.bfloat16)
+    W = _randn((n_out, K), 2, 0.05, torch.bfloat16)
+    ref = O.gemm(to_np(x), to_np(W))
+    ws = torch.empty(hs.hspec_gemm_workspace_bytes(M, n_out, K), dtype=torch.uint8, device="cuda")
+    if mode == "bf16":
+        y = torch.full((M, n_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+        hs.hspec_op_gemm(x, W, y, workspace=ws)
+    elif mode == "accum":
+        y0 = _randn((M, n_out), 3)
+        y = y0.clone()
+        hs.hspec_op_gemm(x, W, y, accumulate=True, workspace=ws)
+        ref = ref + y0.cpu().numpy().astype(np.float64)
+    else:
+        y = torch.full((M, n_out), float("nan"), dtype=torch.float32, device="cuda")
+        hs.hspec_op_gemm(x, W, y, splits=3 if mode == "split3" else 0, workspace=ws)
+    torch.cuda.synchronize()
+    assert_close(y.float().cpu().numpy(), ref, f"gemm {M}x{n_out}x{K} {mode}", tol=1e-2 if mode == "bf16" else 2e-3)
+
+
+def test_gemm_strided_output_and_exact_small_integers(hs):
+    # integer-valued operands: fp32 accumulation is exact, so the result must be bit-exact
+    M, n_out, K = 20, 260, 192
+    g = torch.Generator().manual_seed(5)
+    x = torch.randint(-3, 4, (M, K), generator=g).to(torch.bfloat16).cuda()
+    W = torch.randint(-3, 4, (n_out, K), generator=g).to(torch.bfloat16).cuda()
+    big = torch.full((M, n_out + 7), -1.0, dtype=torch.float32, device="cuda")
+    y = big[:, :n_out]
+    import ctypes as C
+    lib = hs.load_library()
+    rc = lib.hspec_op_gemm(C.c_void_p(x.data_ptr()), C.c_void_p(W.data_ptr()), C.c_void_p(big.data_ptr()), M, n_out, K,
+                           n_out + 7, hs.HSPEC_F32, 0, 1, None, 0, C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    assert rc == 0
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(y.cpu().numpy(), O.gemm(to_np(x), to_np(W)).astype(np.float32))
+    assert (big[:, n_out:] == -1.0).all()
+
+
+@pytest.mark.parametrize("M,V,K", [(8, 1024, 256), (40, 1000, 256), (300, 2500, 128)])
+def test_lm_head_argmax(hs, M, V, K):
+    x = _randn((M, K), 7, 1.0, torch.bfloat16)
+    W = _randn((V, K), 8, 0.05, torch.bfloat16)
+    W[V - 3] = W[5]                    # exact ties between rows 5 and V-3: the lower index must win
+    x[0] = W[5] * 40                   # make row 0 point at the tied pair
+    ids = torch.full((M,), -1, dtype=torch.int32, device="cuda")
+    logits = torch.empty((M, V), dtype=torch.float32, device="cuda")
+    ws = torch.empty(hs.hspec_gemm_workspace_bytes(M, V, K), dtype=torch.uint8, device="cuda")
+    hs.hspec_op_lm_head_argmax(x, W, ids, logits, ws)
+    torch.cuda.synchronize()
+    ref = O.gemm(to_np(x), to_np(W))
+    assert_close(logits.cpu().numpy(), ref, "lm-head logits", tol=2e-3)
+    lg = logits.cpu().numpy()
+    np.testing.assert_array_equal(ids.cpu().numpy(), np.argmax(lg, axis=-1))     # first index of the maximum
+    assert ids[0].item() == 5 and lg[0, 5] == lg[0, V - 3]
+    ref_ids, margin = O.argmax_margin(ref)
+    sure = margin > 1e-3
+    np.testing.assert_array_equal(ids.cpu().numpy()[sure], ref_ids[sure])
+    # without materialising the logits the ids are the same
+    ids2 = torch.full((M,), -1, dtype=torch.int32, device="cuda")
+    hs.hspec_op_lm_head_argmax(x, W, ids2, None, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(ids, ids2)
+
+
+# ------------------------------------------------------------------------------ row-wise ops
+@pytest.mark.parametrize("M,n", [(3, 256), (17, 4096), (5, 10240)])
+def test_rmsnorm(hs, M, n):
+    x, w = _randn((M, n), 11, 3.0), 1 + _randn((n,), 12, 0.02)
+    y = torch.empty((M, n), dtype=torch.bfloat16, device="cuda")
+    hs.hspec_op_rmsnorm(x, w, y, 1e-6)
+    torch.cuda.synchronize()
+    assert_close(y.float().cpu().numpy(), O.rmsnorm(x.cpu().numpy().astype(np.float64), w.cpu().numpy().astype(np.float64), 1e-6),
+                 "rmsnorm", tol=1.2e-2)     # output is rounded to bf16: 2^-9 of the largest element (~3 RMS)
+
+
+def test_swiglu(hs):
+    M, F = 7, 1000
+    gu = _randn((M, 2 * F), 13, 2.0)
+    h = torch.empty((M, F), dtype=torch.bfloat16, device="cuda")
+    hs.hspec_op_swiglu(gu, h)
+    torch.cuda.synchronize()
+    g = gu.cpu().numpy().astype(np.float64)
+    assert_close(h.float().cpu().numpy(), O.silu(g[:, :F]) * g[:, F:], "swiglu", tol=2e-2)
+
+
+@pytest.mark.parametrize("dh,Hq,Hkv,theta,qk_norm", [(64, 4, 2, 1e4, 1), (128, 8, 2, 1e6, 1), (128, 4, 4, 1e6, 0)])
+def test_qk_norm_rope(hs, dh, Hq, Hkv, theta, qk_norm):
+    B, k = 3, 5
+    ctx = torch.tensor([0, 2047, 32760], dtype=torch.int32, device="cuda")
+    qkv = _randn((B * k, (Hq + 2 * Hkv) * dh), 21, 2.0)
+    qw, kw = 1 + _randn((dh,), 22, 0.1), 1 + _randn((dh,), 23, 0.1)
+    q = torch.empty((B * k, Hq, dh), dtype=torch.bfloat16, device="cuda")
+    kb = torch.empty((B * k, Hkv, dh), dtype=torch.bfloat16, device="cuda")
+    vb = torch.empty((B * k, Hkv, dh), dtype=torch.bfloat16, device="cuda")
+    hs.hspec_op_qk_norm_rope(qkv, qw, kw, ctx, q, kb, vb, B, k, Hq, Hkv, dh, theta, 1e-6, qk_norm)
+    torch.cuda.synchronize()
+    a = qkv.cpu().numpy().astype(np.float64).reshape(B * k, Hq + 2 * Hkv, dh)
+    qr, kr = a[:, :Hq], a[:, Hq:Hq + Hkv]
+    if qk_norm:
+        qr = O.rmsnorm(qr, qw.cpu().numpy().astype(np.float64), 1e-6)
+        kr = O.rmsnorm(kr, kw.cpu().numpy().astype(np.float64), 1e-6)
+    for m in range(B * k):
+        pos = int(ctx[m // k]) + m % k
+        assert_close(q[m].float().cpu().numpy(), O.rope(qr[m], pos, theta), f"q row {m}", tol=1.5e-2)
+        assert_close(kb[m].float().cpu().numpy(), O.rope(kr[m], pos, theta), f"k row {m}", tol=1.5e-2)
+    np.testing.assert_array_equal(vb.float().cpu().numpy().reshape(B * k, Hkv, dh), bf16_round(a[:, Hq + Hkv:]))
+
+
+# ------------------------------------------------------------------------------ Mamba-2 mixer core
+@pytest.mark.parametrize("B,k,Di,P,N,G,dtr,zero_state", [
+    (2, 8, 512, 64, 16, 1, True, False), (3, 5, 256, 64, 128, 2, False, False), (1, 16, 8192, 64, 128, 4, False, False),
+    (2, 1, 128, 64, 128, 1, False, False), (2, 32, 192, 64, 4, 1, False, False), (2, 7, 128, 32, 24, 2, False, True),
+])
+def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state):
+    H, d_conv = Di // P, 4
+    d_xBC = Di + 2 * G * N
+    ld = Di + d_xBC + (0 if dtr else H)
+    zx = _randn((B * k, ld), 31, 1.0)
+    dt_raw = _randn((B * k, H), 32, 1.0) if dtr else None
+    s_init = None if zero_state else _randn((B, H, P, N), 33, 1.5, torch.bfloat16)
+    conv_w = (torch.rand((d_xBC, d_conv), device="cuda", generator=torch.Generator(device="cuda").manual_seed(34)) - 0.5)
+    conv_b = _randn((d_xBC,), 35, 0.02)
+    A_log = torch.rand((H,), device="cuda", generator=torch.Generator(device="cuda").manual_seed(36)) * 2
+    dt_bias = _randn((H,), 37, 1.0) - 4.0
+    Dskip = 1 + _randn((H,), 38, 0.1)
+    y = torch.full((B * k, Di), float("nan"), dtype=torch.float32, device="cuda")
+    hs.hspec_op_mamba_scan(zx, dt_raw, s_init, conv_w, conv_b, dt_bias, A_log, Dskip, y, B, k, Di, P, N, G, d_conv)
+    torch.cuda.synchronize()
+    f64 = lambda t: t.cpu().numpy().astype(np.float64)
+    zxn = f64(zx)
+    for b in range(B):
+        rows = zxn[b * k:(b + 1) * k]
+        z, raw = rows[:, :Di], rows[:, Di:Di + d_xBC]
+        dtr_b = f64(dt_raw)[b * k:(b + 1) * k] if dtr else rows[:, Di + d_xBC:]
+        xBC = O.conv_silu(raw, f64(conv_w), f64(conv_b))
+        x = xBC[:, :Di].reshape(k, H, P)
+        Bm, Cm = xBC[:, Di:Di + G * N].reshape(k, G, N), xBC[:, Di + G * N:].reshape(k, G, N)
+        dt, a = O.discretise(dtr_b, f64(dt_bias), f64(A_log))
+        S0 = np.zeros((H, P, N)) if zero_state else O.widen(to_np(s_init[b]))
+        yy, _ = O.scan_sequential(S0, x, Bm, Cm, dt, a, f64(Dskip))
+        ref = yy.reshape(k, Di) * O.silu(z)
+        assert_close(y[b * k:(b + 1) * k].cpu().numpy(), ref, f"scan request {b}", tol=2e-3)
+
+
+# ------------------------------------------------------------------------------ attention
+def _attn_case(hs, B, k, Hq, Hkv, dh, ctxs, window, chunk, seed=0, poison=True):
+    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
+    batch = synth.make_request_batch(cfg, ctx_lens=ctxs, device="cuda", poison_tail=poison, extra_pages=3,
+                                     seed_offset=seed)
+    M = B * k
+    q = _randn((M, Hq, dh), 41 + seed, 1.0, torch.bfloat16)
+    kb = _randn((M, Hkv, dh), 42 + seed, 1.0, torch.bfloat16)
+    vb = _randn((M, Hkv, dh), 43 + seed, 1.0, torch.bfloat16)
+    o = torch.full((M, Hq * dh), float("nan"), dtype=torch.bfloat16, device="cuda")
+    max_ctx = max(ctxs + [1])
+    ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, max_ctx, window, chunk), dtype=torch.uint8,
+                     device="cuda")
+    hs.hspec_op_attention(q, kb, vb, batch["k_pools"][0], batch["v_pools"][0], batch["page_table"], batch["ctx_lens"],
+                          max_ctx, o, B, k, Hq, Hkv, dh, 16, window, chunk, ws)
+    torch.cuda.synchronize()
+    got = o.float().cpu().numpy().reshape(B, k, Hq, dh)
+    kp, vp, pt = to_np(batch["k_pools"][0]), to_np(batch["v_pools"][0]), to_np(batch["page_table"])
+    worst = 0.0
+    for b in range(B):
+        sl = slice(b * k, (b + 1) * k)
+        ref = O.attention_paged(to_np(q[sl]), kp, vp, pt[b], ctxs[b], to_np(kb[sl]), to_np(vb[sl]), window=window)
+        worst = max(worst, assert_close(got[b], ref, f"attention request {b} ctx {ctxs[b]}", tol=1.5e-2))
+    return worst
+
+
+@pytest.mark.parametrize("window", [0, 1, 7, 64, 2048])
+@pytest.mark.parametrize("chunk", [64, 256, 0])
+def test_attention_small_heads(hs, window, chunk):
+    _attn_case(hs, 6, 5, 4, 2, 64, [0, 1, 15, 16, 17, 40], window, chunk)
+
+
+@pytest.mark.parametrize("k,Hq,Hkv,dh", [(8, 4, 2, 64), (16, 32, 8, 128), (16, 16, 2, 128), (32, 8, 1, 128), (3, 8, 8, 128)])
+def test_attention_shapes_and_long_contexts(hs, k, Hq, Hkv, dh):
+    # rows per KV head: 16, 64, 128, 256 (two row tiles), 3; contexts span several chunks and a ragged tail
+    _attn_case(hs, 4, k, Hq, Hkv, dh, [300, 1000, 4099, 63], 0, 0, seed=1)
+    _attn_case(hs, 4, k, Hq, Hkv, dh, [300, 1000, 4099, 63], 0, 512, seed=2)
+    _attn_case(hs, 4, k, Hq, Hkv, dh, [300, 1000, 4099, 2047], 2048, 0, seed=3)
+
+
+def test_attention_page_permutation_is_bit_exact(hs):
+    B, k, Hq, Hkv, dh = 2, 4, 8, 2, 128
+    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
+    batch = synth.make_request_batch(cfg, ctx_lens=[200, 77], device="cuda", extra_pages=4)
+    q = _randn((B * k, Hq, dh), 51, 1.0, torch.bfloat16)
+    kb, vb = _randn((B * k, Hkv, dh), 52, 1.0, torch.bfloat16), _randn((B * k, Hkv, dh), 53, 1.0, torch.bfloat16)
+    ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, 200, 0, 64), dtype=torch.uint8, device="cuda")
+
+    def run(bt):
+        o = torch.empty((B * k, Hq * dh), dtype=torch.bfloat16, device="cuda")
+        hs.hspec_op_attention(q, kb, vb, bt["k_pools"][0], bt["v_pools"][0], bt["page_table"], bt["ctx_lens"], 200, o,
+                              B, k, Hq, Hkv, dh, 16, 0, 64, ws)
+        torch.cuda.synchronize()
+        return o
+    base = run(batch)
+    n = batch["num_pages"]
+    perm = torch.randperm(n, generator=torch.Generator().manual_seed(3)).cuda()
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(n, device="cuda")
+    pt = batch["page_table"].clone()
+    valid = pt >= 0
+    pt[valid] = perm[pt[valid].long()].to(torch.int32)
+    moved = dict(batch, page_table=pt, k_pools=[batch["k_pools"][0][inv]], v_pools=[batch["v_pools"][0][inv]])
+    assert torch.equal(run(moved).view(torch.int16), base.view(torch.int16))
+    assert torch.equal(run(batch).view(torch.int16), base.view(torch.int16))     # run-twice reproducibility

@@ -1,0 +1,122 @@
+"""Parity of the whole draft step (hspec_draft_block) against the oracle, plus the properties that hold
+at any size: request independence, page-permutation invariance (bit-exact), causal k-prefix, determinism."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from harness import check_step, cuda_setup, oracle_step, assert_close, MARGIN
+
+pytestmark = pytest.mark.gpu
+
+MID = dict(D=512, n_fuse=2, r=512, L=2, has_attn=[1, 1], kv_slot=[1, 0], n_slots=2, Di=1024, P=64, N=128, G=4,
+           d_conv=4, dt_rank=0, Hq=8, Hkv=2, dh=128, rope_theta=1.0e6, window=0, qk_norm=1, F=1536, V=2000,
+           rms_eps=1e-6, page_size=16, name="mid", B=5, k=16, ctx=("uniform", 0, 3000))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    from paper_2609_24197_b200 import build
+    build.build()
+
+
+def test_tiny_config_full_parity():
+    cfg = synth.get_config("tiny")
+    drafter, w, batch = cuda_setup(cfg)
+    r = check_step(cfg, drafter, w, batch, cfg["k"], what="tiny")
+    assert r["ids_compared"] >= 4
+    drafter.close()
+
+
+@pytest.mark.parametrize("k", [1, 5, 16, 32])
+def test_mid_config_ragged_contexts(k):
+    cfg = synth.derived(dict(MID, k=k))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[0, 1, 17, 1000, 2999], max_k=32)
+    check_step(cfg, drafter, w, batch, k, what=f"mid k={k}")
+    drafter.close()
+
+
+def test_mid_config_window_and_attentionless_layer():
+    cfg = synth.derived(dict(MID, window=256, has_attn=[1, 0], kv_slot=[1, -1], B=3))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[100, 255, 700])
+    check_step(cfg, drafter, w, batch, 7, what="mid window")
+    drafter.close()
+
+
+def test_properties_bit_exact():
+    cfg = synth.derived(dict(MID))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[33, 700, 16, 2100])
+    k = 8
+    mc = 2100
+
+    def run(bt, kk=k):
+        ids, logits, _ = drafter.draft(bt, kk, want_logits=True, max_ctx=mc)
+        torch.cuda.synchronize()
+        return ids.clone(), logits.clone()
+    ids0, lg0 = run(batch)
+    ids1, lg1 = run(batch)
+    assert torch.equal(lg0, lg1) and torch.equal(ids0, ids1)                     # deterministic
+    # page permutation: any physical placement with the table updated gives identical bits
+    n = batch["num_pages"]
+    perm = torch.randperm(n, generator=torch.Generator().manual_seed(11)).cuda()
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(n, device="cuda")
+    pt = batch["page_table"].clone()
+    valid = pt >= 0
+    pt[valid] = perm[pt[valid].long()].to(torch.int32)
+    moved = dict(batch, page_table=pt, k_pools=[t[inv] for t in batch["k_pools"]], v_pools=[t[inv] for t in batch["v_pools"]])
+    ids2, lg2 = run(moved)
+    assert torch.equal(lg0, lg2) and torch.equal(ids0, ids2)
+    # the KV pools are never written
+    kp_before = [t.clone() for t in batch["k_pools"]]
+    run(batch)
+    for a, b in zip(kp_before, batch["k_pools"]):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    # causal over block positions: the first j rows of a k-step are a j-step (same kernels, other launch shapes)
+    ids3, lg3 = run(batch, 3)
+    ref = lg0[:, :3].cpu().numpy()
+    assert_close(lg3.cpu().numpy(), ref, "k-prefix", tol=5e-3)
+    drafter.close()
+
+
+def test_request_independence_across_batch_sizes():
+    cfg = synth.derived(dict(MID))
+    w = synth.make_weights(cfg, device="cuda")
+    ctxs = [500, 40, 1300]
+    d3, _, batch3 = cuda_setup(cfg, ctx_lens=ctxs, weights=w)
+    _, lg3, _ = d3.draft(batch3, 6, want_logits=True, max_ctx=1300)
+    torch.cuda.synchronize()
+    # request 1 alone, with its own pages
+    one = dict(batch3, ctx_lens=batch3["ctx_lens"][1:2].contiguous(), page_table=batch3["page_table"][1:2].contiguous(),
+               last_hidden=batch3["last_hidden"][1:2].contiguous(), last_token=batch3["last_token"][1:2].contiguous(),
+               ctx_lens_host=[40])
+    _, lg1, _ = d3.draft(one, 6, want_logits=True, max_ctx=1300)
+    torch.cuda.synchronize()
+    assert_close(lg1[0].cpu().numpy(), lg3[1].cpu().numpy(), "request independence", tol=5e-3)
+    d3.close()
+
+
+def _full_size(name, n_check, **over):
+    cfg = synth.get_config(name, **over)
+    drafter, w, batch = cuda_setup(cfg, poison_tail=False, extra_pages=0)
+    B = cfg["B"]
+    # longest, shortest and (if asked) a seeded random request
+    order = np.argsort(batch["ctx_lens_host"])
+    pick = sorted(set([int(order[-1]), int(order[0])][:n_check]))
+    r = check_step(cfg, drafter, w, batch, cfg["k"], requests=pick, dtype=np.float32, what=name)
+    drafter.close()
+    del w, batch
+    torch.cuda.empty_cache()
+    return r
+
+
+def test_latency_8b_full_size():
+    _full_size("latency_8b", 1)
+
+
+def test_serving_8b_full_size_sampled_requests():
+    _full_size("serving_8b", 2)
+
+
+def test_conc128_32b_full_size_sampled_request():
+    _full_size("conc128_32b", 1)
