@@ -12,6 +12,17 @@
  *   final norm, the target's LM head, arg-max -> k draft tokens           (App. B.2 "Pruned drafter vocabulary": LM head is the target's)
  * No drafter-side KV cache exists: the library never writes the KV pools (Sec. 3.2).
  *
+ * Precision
+ *   Weights arrive as bf16.  hspec_load_weights keeps its own device copy of every tensor; matrices that feed
+ *   a tensor-core GEMM are widened once to fp16 (bf16 has 8 significant bits, fp16 has 11: the conversion is
+ *   exact for 2^-17 <= |w| <= 65504 and loses at most 2^-25 below that).  Activations the library produces
+ *   and feeds to a GEMM (norm outputs, the gated SSM output, the attention output, the SwiGLU product, the
+ *   fusion vector, S_init) are fp16 as well, because the MMA needs both operands in one 16-bit type and
+ *   bf16 activations (8 bits) put the step's rounding noise at ~3e-2 of the output RMS over a full logits
+ *   tensor, above the 2e-2 parity bound.  Accumulation is fp32; the residual stream, scan and softmax are
+ *   fp32.  The target's KV pools are read in place as bf16, so q, the block's k/v and the softmax weights
+ *   enter the attention MMAs as bf16.  fp16 saturates at 65504: hidden states beyond that are out of range.
+ *
  * Conventions
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
  *     ordinary host memory.  No torch / C++ types cross this boundary.
@@ -48,7 +59,7 @@ typedef enum {
   HSPEC_ERR_TIMEOUT = -7             /* a bounded in-kernel wait gave up (status word) */
 } hspec_status;
 
-typedef enum { HSPEC_BF16 = 0, HSPEC_F32 = 1, HSPEC_I32 = 2 } hspec_dtype;
+typedef enum { HSPEC_BF16 = 0, HSPEC_F32 = 1, HSPEC_I32 = 2, HSPEC_F16 = 3 } hspec_dtype;
 
 /* Shapes of the drafter (App. B.1).  H = Di / P Mamba heads; d_S = H * P * N. */
 typedef struct {
@@ -76,8 +87,8 @@ typedef struct {
   int32_t max_pages_per_req; /* largest page-table row length (bounds the context) */
 } hspec_config;
 
-/* A named tensor in DEVICE memory.  The library borrows the pointer: it must stay valid and
- * unchanged until hspec_destroy.  Names (l = layer index):
+/* A named tensor in DEVICE memory.  hspec_load_weights copies it (converting GEMM matrices to fp16), so
+ * the caller may free or reuse it afterwards.  Names (l = layer index):
  *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D]
  *   layers.l.mamba.{norm [D], in_proj [Di + (Di+2GN) + (dt_rank or H), D] (rows z | xBC | dt),
  *                   dt_up [H, dt_rank] (only if dt_rank>0), conv_w [Di+2GN, d_conv], conv_b [Di+2GN],
@@ -136,11 +147,12 @@ typedef struct {
 int hspec_init(const hspec_config* cfg, hspec_handle** out);
 /* Device scratch bytes a step of up to (max_batch, max_k, max_pages_per_req) needs. */
 size_t hspec_workspace_bytes(const hspec_config* cfg);
-/* Registers n named device tensors (may be called several times).  Shapes are checked against the config. */
+/* Copies n named device tensors into library-owned device memory (may be called several times; synchronises the
+ * device).  Shapes are checked against the config. */
 int hspec_load_weights(hspec_handle* h, const hspec_tensor* tensors, int32_t n);
 /* Enqueues one block-parallel draft step (Sec. 3.3) on in->stream.  Needs every tensor loaded. */
 int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* out);
-/* Frees the handle.  Borrowed tensors, pools and the workspace stay the caller's. */
+/* Frees the handle and its weight copies.  Pools and the workspace stay the caller's. */
 int hspec_destroy(hspec_handle* h);
 /* Message of the last failure on this handle (or of the last failed hspec_init if h is NULL). */
 const char* hspec_last_error(const hspec_handle* h);
@@ -152,25 +164,26 @@ int hspec_get_stats(hspec_handle* h, hspec_stats* out);
  * enqueue on `stream` and do not synchronise.
  * ---------------------------------------------------------------------------------------------- */
 
-/* y[M, n_out] = x[M, K] W[n_out, K]^T, x and W bf16, fp32 accumulation (every linear map of Sec. 3.3).
- * out_dtype HSPEC_F32 or HSPEC_BF16; ldy = row pitch of y in elements.  accumulate != 0 (fp32 only):
+/* y[M, n_out] = x[M, K] W[n_out, K]^T, x and W both bf16 or both fp16 (in_dtype), fp32 accumulation (every linear
+ * map of Sec. 3.3).  out_dtype HSPEC_F32, HSPEC_BF16 or HSPEC_F16; ldy = row pitch of y in elements.  accumulate != 0 (fp32 only):
  * y += result (the residual form).  splits <= 0 lets the library choose how many K-slices to use;
  * `workspace` (>= hspec_gemm_workspace_bytes) is needed when more than one slice is used.
  * Needs K % 8 == 0, 16-byte aligned x and W. */
-int hspec_op_gemm(const void* x, const void* W, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,
+int hspec_op_gemm(const void* x, const void* W, int32_t in_dtype, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,
                   int32_t out_dtype, int32_t accumulate, int32_t splits, void* workspace, size_t workspace_bytes,
                   void* stream);
 size_t hspec_gemm_workspace_bytes(int32_t M, int32_t n_out, int32_t K);
-/* LM head fused with arg-max (App. B.2): ids[m] = lowest index of max_v x[m,:] . W[v,:]; logits fp32 [M, V] or NULL. */
-int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t* ids, float* logits, int32_t M, int32_t V,
+/* LM head fused with arg-max (App. B.2): ids[m] = lowest index of max_v x[m,:] . W[v,:]; logits fp32 [M, V] or NULL.
+ * x and W are both bf16 or both fp16 (in_dtype). */
+int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M, int32_t V,
                             int32_t K, void* workspace, size_t workspace_bytes, void* stream);
-/* RMSNorm over the last axis: y bf16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
-int hspec_op_rmsnorm(const float* x, const float* w, void* y_bf16, int32_t M, int32_t n, float eps, void* stream);
+/* RMSNorm over the last axis: y fp16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
+int hspec_op_rmsnorm(const float* x, const float* w, void* y_f16, int32_t M, int32_t n, float eps, void* stream);
 /* Mamba-2 mixer core for B requests x k rows (Sec. 3.3.1): causal depthwise conv + SiLU on xBC (zero left
  * context), dt = softplus(dt_raw + dt_bias), decay exp(dt * -exp(A_log)), the selective recurrence over the
  * k rows started from s_init, the D skip, and the SiLU(z) gate.
  *   zxbcdt fp32 [B*k, ld_in]: columns z [Di] | xBC [Di + 2GN] (| dt [H] when dt_raw is NULL)
- *   dt_raw fp32 [B*k, H] or NULL;  s_init bf16 [B, H, P, N] or NULL (zero state)
+ *   dt_raw fp32 [B*k, H] or NULL;  s_init fp16 [B, H, P, N] or NULL (zero state)
  *   y_gated fp32 [B*k, Di] = (scan output) * SiLU(z). */
 int hspec_op_mamba_scan(const float* zxbcdt, int64_t ld_in, const float* dt_raw, const void* s_init,
                         const float* conv_w, const float* conv_b, const float* dt_bias, const float* A_log,
@@ -183,7 +196,7 @@ int hspec_op_qk_norm_rope(const float* qkv, const float* q_norm_w, const float* 
                           float theta, float eps, int32_t qk_norm, void* stream);
 /* Block-query GQA attention over the target's paged KV (read in place) plus the block's causal keys (Sec. 3.3.2).
  * q/kb/vb as produced by hspec_op_qk_norm_rope; k_pool/v_pool bf16 [num_pages, page_size, Hkv, dh];
- * o bf16 [B*k, Hq*dh].  window 0 = full.  max_ctx: host upper bound on ctx_lens (0 = stride*page_size).
+ * o fp16 [B*k, Hq*dh].  window 0 = full.  max_ctx: host upper bound on ctx_lens (0 = stride*page_size).
  * chunk_tokens <= 0 lets the library pick the context split. */
 int hspec_op_attention(const void* q, const void* kb, const void* vb, const void* k_pool, const void* v_pool,
                        const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens,
@@ -196,8 +209,8 @@ size_t hspec_attention_workspace_bytes(int32_t B, int32_t k, int32_t Hq, int32_t
  * bit-exact; used to check the page-table addressing of the attention kernel, Sec. 3.3.2). */
 int hspec_debug_gather_kv(const void* pool, const int32_t* page_table_row, int32_t ctx_len, int32_t page_size,
                           int32_t Hkv, int32_t dh, void* dst, void* stream);
-/* h bf16 [M, F] = SiLU(gu[:, :F]) * gu[:, F:], gu fp32 [M, 2F] (App. B.1 "MLP"). */
-int hspec_op_swiglu(const float* gu, void* h_bf16, int32_t M, int32_t F, void* stream);
+/* h fp16 [M, F] = SiLU(gu[:, :F]) * gu[:, F:], gu fp32 [M, 2F] (App. B.1 "MLP"). */
+int hspec_op_swiglu(const float* gu, void* h_f16, int32_t M, int32_t F, void* stream);
 
 #ifdef __cplusplus
 }

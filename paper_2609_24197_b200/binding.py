@@ -13,7 +13,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhspec.so")
 
 HSPEC_MAX_LAYERS = 16
-HSPEC_BF16, HSPEC_F32, HSPEC_I32 = 0, 1, 2
+HSPEC_BF16, HSPEC_F32, HSPEC_I32, HSPEC_F16 = 0, 1, 2, 3
+_DT = {torch.bfloat16: 0, torch.float32: 1, torch.int32: 2, torch.float16: 3}
 
 EXPORTS = [
     "hspec_init", "hspec_workspace_bytes", "hspec_load_weights", "hspec_draft_block", "hspec_destroy",
@@ -84,10 +85,10 @@ def load_library(path=None):
     lib.hspec_last_error.restype = C.c_char_p
     lib.hspec_get_stats.argtypes = [C.c_void_p, C.POINTER(hspec_stats)]
     vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
-    lib.hspec_op_gemm.argtypes = [vp, vp, vp, i32, i32, i32, i64, i32, i32, i32, vp, sz, vp]
+    lib.hspec_op_gemm.argtypes = [vp, vp, i32, vp, i32, i32, i32, i64, i32, i32, i32, vp, sz, vp]
     lib.hspec_gemm_workspace_bytes.argtypes = [i32, i32, i32]
     lib.hspec_gemm_workspace_bytes.restype = sz
-    lib.hspec_op_lm_head_argmax.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, sz, vp]
+    lib.hspec_op_lm_head_argmax.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp, sz, vp]
     lib.hspec_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, f32, vp]
     lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
     lib.hspec_op_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, vp]
@@ -216,28 +217,28 @@ def hspec_op_gemm(x, W, y, accumulate=False, splits=0, workspace=None):
     n_out = W.shape[0]
     ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
     _check(load_library().hspec_op_gemm(
-        _ptr(x, torch.bfloat16), _ptr(W, torch.bfloat16), _ptr(y), M, n_out, K, y.stride(0),
-        HSPEC_BF16 if y.dtype == torch.bfloat16 else HSPEC_F32, int(accumulate), int(splits),
+        _ptr(x), _ptr(W, x.dtype), _DT[x.dtype], _ptr(y), M, n_out, K, y.stride(0),
+        _DT[y.dtype], int(accumulate), int(splits),
         _ptr(workspace), ws_bytes, _stream()), None, "hspec_op_gemm")
 
 
 def hspec_op_lm_head_argmax(x, W, ids, logits, workspace):
     M, K = x.shape
     _check(load_library().hspec_op_lm_head_argmax(
-        _ptr(x, torch.bfloat16), _ptr(W, torch.bfloat16), _ptr(ids, torch.int32), _ptr(logits, torch.float32),
+        _ptr(x), _ptr(W, x.dtype), _DT[x.dtype], _ptr(ids, torch.int32), _ptr(logits, torch.float32),
         M, W.shape[0], K, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
         None, "hspec_op_lm_head_argmax")
 
 
 def hspec_op_rmsnorm(x, w, y, eps):
-    _check(load_library().hspec_op_rmsnorm(_ptr(x, torch.float32), _ptr(w, torch.float32), _ptr(y, torch.bfloat16),
+    _check(load_library().hspec_op_rmsnorm(_ptr(x, torch.float32), _ptr(w, torch.float32), _ptr(y, torch.float16),
                                            x.shape[0], x.shape[1], float(eps), _stream()), None, "hspec_op_rmsnorm")
 
 
 def hspec_op_mamba_scan(zxbcdt, dt_raw, s_init, conv_w, conv_b, dt_bias, A_log, Dskip, y_gated, B, k, Di, P, N, G,
                         d_conv):
     _check(load_library().hspec_op_mamba_scan(
-        _ptr(zxbcdt, torch.float32), zxbcdt.stride(0), _ptr(dt_raw, torch.float32), _ptr(s_init, torch.bfloat16),
+        _ptr(zxbcdt, torch.float32), zxbcdt.stride(0), _ptr(dt_raw, torch.float32), _ptr(s_init, torch.float16),
         _ptr(conv_w, torch.float32), _ptr(conv_b, torch.float32), _ptr(dt_bias, torch.float32),
         _ptr(A_log, torch.float32), _ptr(Dskip, torch.float32), _ptr(y_gated, torch.float32),
         B, k, Di, P, N, G, d_conv, _stream()), None, "hspec_op_mamba_scan")
@@ -259,7 +260,7 @@ def hspec_op_attention(q, kb, vb, k_pool, v_pool, page_table, ctx_lens, max_ctx,
     _check(load_library().hspec_op_attention(
         _ptr(q, torch.bfloat16), _ptr(kb, torch.bfloat16), _ptr(vb, torch.bfloat16), _ptr(k_pool, torch.bfloat16),
         _ptr(v_pool, torch.bfloat16), _ptr(page_table, torch.int32), int(page_table.shape[1]),
-        _ptr(ctx_lens, torch.int32), int(max_ctx), _ptr(o, torch.bfloat16), B, k, Hq, Hkv, dh, page_size, window,
+        _ptr(ctx_lens, torch.int32), int(max_ctx), _ptr(o, torch.float16), B, k, Hq, Hkv, dh, page_size, window,
         chunk_tokens, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
         None, "hspec_op_attention")
 
@@ -272,7 +273,7 @@ def hspec_debug_gather_kv(pool, page_table_row, ctx_len, dst):
 
 
 def hspec_op_swiglu(gu, h):
-    _check(load_library().hspec_op_swiglu(_ptr(gu, torch.float32), _ptr(h, torch.bfloat16), gu.shape[0], h.shape[1],
+    _check(load_library().hspec_op_swiglu(_ptr(gu, torch.float32), _ptr(h, torch.float16), gu.shape[0], h.shape[1],
                                           _stream()), None, "hspec_op_swiglu")
 
 
@@ -289,7 +290,6 @@ class Drafter:
         self.max_pages = max(1, (max_ctx + ps - 1) // ps)
         self.config = make_config(cfg, max_batch, max_k, self.max_pages)
         self.handle = hspec_init(self.config)
-        self.weights = weights                       # keep the borrowed tensors alive
         hspec_load_weights(self.handle, weights)
         nbytes = hspec_workspace_bytes(self.config)
         self.workspace = torch.empty(nbytes + 1024, dtype=torch.uint8, device="cuda")

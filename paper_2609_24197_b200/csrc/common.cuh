@@ -1,6 +1,7 @@
 // Shared device helpers for the H-Spec draft-step kernels (sm_100a only).
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -153,9 +154,11 @@ __device__ __forceinline__ uint64_t umma_desc_kmajor_sw128(uint32_t smem_addr) {
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n.
-__device__ __forceinline__ uint32_t umma_idesc_bf16_m128(uint32_t n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+// Instruction descriptor: fp32 accumulator, A and B both fp16 or both bf16 (the hardware rejects a mixed
+// pair as an illegal instruction), both K-major, M = 128, N = n.
+__device__ __forceinline__ uint32_t umma_idesc_m128(uint32_t n, bool f16) {
+  const uint32_t fmt = f16 ? 0u : 1u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 // ------------------------------------------------------------------ warp-level mma (attention)

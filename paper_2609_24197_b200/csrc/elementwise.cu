@@ -35,8 +35,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return r;
 }
 
-// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, bf16 out.
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __nv_bfloat16* __restrict__ y,
+// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 out.
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __half* __restrict__ y,
                                int n, float eps) {
   __shared__ float red[32];
   const float* xr = x + size_t(blockIdx.x) * n;
@@ -44,8 +44,8 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   for (int d = threadIdx.x; d < n; d += blockDim.x) { const float v = xr[d]; ss += v * v; }
   const float tot = block_sum(ss, red);
   const float inv = rsqrtf(tot / float(n) + eps);
-  __nv_bfloat16* yr = y + size_t(blockIdx.x) * n;
-  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = __float2bfloat16_rn(xr[d] * inv * w[d]);
+  __half* yr = y + size_t(blockIdx.x) * n;
+  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = __float2half_rn(xr[d] * inv * w[d]);
 }
 
 // Per (row, head): optional RMSNorm over dh, then rotate-half RoPE at position ctx_len + i.
@@ -86,13 +86,13 @@ __global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* 
   }
 }
 
-__global__ void swiglu_kernel(const float* __restrict__ gu, __nv_bfloat16* __restrict__ h, int M, int F) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F) {
   const long long total = (long long)M * F;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
     const int m = int(idx / F), f = int(idx % F);
     const float gte = gu[size_t(m) * 2 * F + f], up = gu[size_t(m) * 2 * F + F + f];
-    h[idx] = __float2bfloat16_rn(silu_f(gte) * up);
+    h[idx] = __float2half_rn(silu_f(gte) * up);
   }
 }
 
@@ -134,9 +134,9 @@ cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token,
   return cudaGetLastError();
 }
 
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_bf16, int M, int n, float eps, cudaStream_t stream) {
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream) {
   const int threads = n >= 2048 ? 512 : 256;
-  rmsnorm_kernel<<<M, threads, 0, stream>>>(x, w, (__nv_bfloat16*)y_bf16, n, eps);
+  rmsnorm_kernel<<<M, threads, 0, stream>>>(x, w, (__half*)y_f16, n, eps);
   return cudaGetLastError();
 }
 
@@ -152,8 +152,8 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
   return cudaGetLastError();
 }
 
-cudaError_t swiglu_launch(const float* gu, void* h_bf16, int M, int F, cudaStream_t stream) {
-  swiglu_kernel<<<grid_for((long long)M * F, 256), 256, 0, stream>>>(gu, (__nv_bfloat16*)h_bf16, M, F);
+cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream) {
+  swiglu_kernel<<<grid_for((long long)M * F, 256), 256, 0, stream>>>(gu, (__half*)h_f16, M, F);
   return cudaGetLastError();
 }
 

@@ -94,7 +94,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16_m128(g.BN);
+      const uint32_t idesc = umma_idesc_m128(g.BN, g.f16 != 0);
       bool ok = true;
       for (int i = 0; i < n_kt && ok; ++i) {
         const int s = i % g.stages;
@@ -155,6 +155,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const int m = m0 + c0 + j;
           if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
         }
+      } else if (g.mode == EPI_STORE_F16) {
+        __half* out = reinterpret_cast<__half*>(g.out);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2half_rn(__uint_as_float(r[j]));
+        }
       } else {  // EPI_ARGMAX: logits optional, (max, lowest index) over this warp's 32 vocabulary rows
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
@@ -211,6 +218,7 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
     for (int s = 0; s < splits; ++s) acc += part[(size_t(s) * M + m) * N + n];
     if (mode == EPI_STORE_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] = acc;
     else if (mode == EPI_ACCUM_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] += acc;
+    else if (mode == EPI_STORE_F16) reinterpret_cast<__half*>(out)[size_t(m) * ldo + n] = __float2half_rn(acc);
     else reinterpret_cast<__nv_bfloat16*>(out)[size_t(m) * ldo + n] = __float2bfloat16_rn(acc);
   }
 }
@@ -271,9 +279,9 @@ int g_smem_optin = -1;
 
 }  // namespace
 
-// 2-D bf16 row-major [rows, cols] tensor, box [box_rows x 64 columns], 128-byte swizzle, zero fill.
-bool make_tmap_bf16_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
-                       int box_rows, std::string* err) {
+// 2-D bf16/fp16 row-major [rows, cols] tensor, box [box_rows x 64 columns], 128-byte swizzle, zero fill.
+bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
+                        int box_rows, bool f16, std::string* err) {
   EncodeTiledFn enc = get_encode();
   if (!enc) { if (err) *err = "cuTensorMapEncodeTiled is not available from the CUDA driver"; return false; }
   if ((reinterpret_cast<uintptr_t>(base) & 15) || ((ld_elems * 2) & 15)) {
@@ -284,7 +292,7 @@ bool make_tmap_bf16_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t 
   cuuint64_t strides[1] = {cuuint64_t(ld_elems) * 2};
   cuuint32_t box[2] = {cuuint32_t(TILE_K), cuuint32_t(box_rows)};
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  CUresult r = enc(tm, f16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
@@ -344,6 +352,7 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launch
   if (stages < 2) { if (err) *err = "shared memory too small for the GEMM pipeline"; return cudaErrorInvalidValue; }
   g.stages = stages;
   g.status = c.status;
+  g.f16 = c.f16 ? 1 : 0;
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx;
   g.ldo = c.ldo;
   if (splits > 1) {
@@ -357,7 +366,7 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launch
     g.mode = c.mode; g.out = c.out;
   }
   CUtensorMap tmB;
-  if (!make_tmap_bf16_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BN, err)) return cudaErrorInvalidValue;
+  if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BN, c.f16, err)) return cudaErrorInvalidValue;
   dim3 grid((c.M + g.BN - 1) / g.BN, (c.n_out + TILE_W - 1) / TILE_W, splits);
   const size_t smem = size_t(stages) * stage_bytes + fixed;
   gemm_tcgen05_kernel<<<grid, 192, smem, stream>>>(*c.tmW, tmB, g);

@@ -2,7 +2,9 @@
 #include "../../include/hspec.h"
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -20,7 +22,7 @@ constexpr int kNumSMs = 148;   // B200; only used to size grids and K-slices
 thread_local std::string g_err;
 
 struct Weight {
-  const void* data = nullptr;
+  void* data = nullptr;      // library-owned device copy (GEMM matrices as fp16, everything else as given)
   int dtype = 0;
   int64_t rows = 0, cols = 0;
   bool has_tm = false;
@@ -47,7 +49,7 @@ int imax(int a, int b) { return a > b ? a : b; }
 
 // Offsets of the step's scratch buffers inside the caller's workspace.
 struct Plan {
-  size_t X, U, BIG, Fv, SINIT, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
+  size_t X, U, BIG, LH, Fv, SINIT, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
   size_t att_bytes, splitk_bytes;
   int attn_chunk, max_ctx;
 };
@@ -65,6 +67,7 @@ Plan make_plan(const hspec_config& c, int B, int k, int max_ctx) {
   p.X = take(M * c.D * 4);
   p.U = take(M * size_t(imax(imax(c.D, c.Di), imax(c.Hq * c.dh, c.F))) * 2);
   p.BIG = take(M * size_t(imax(imax(d.d_in_proj, d.d_qkv), 2 * c.F)) * 4);
+  p.LH = take(size_t(B) * c.n_fuse * c.D * 2);
   p.Fv = take(size_t(B) * c.r * 2);
   p.SINIT = take(size_t(B) * d.d_S * 2);
   p.DTL = take(M * size_t(imax(c.dt_rank, 8)) * 2);
@@ -210,11 +213,16 @@ std::vector<std::string> required_names(const hspec_config& c) {
   return n;
 }
 
-__global__ void cvt_cols_bf16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
-                                     __nv_bfloat16* __restrict__ dst) {
+__global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n) {
+  for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x)
+    dst[i] = __float2half_rn(__bfloat162float(src[i]));
+}
+
+__global__ void cvt_cols_f16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
+                                    __half* __restrict__ dst) {
   const int total = M * ncols;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x)
-    dst[i] = __float2bfloat16_rn(src[size_t(i / ncols) * ld + col0 + i % ncols]);
+    dst[i] = __float2half_rn(src[size_t(i / ncols) * ld + col0 + i % ncols]);
 }
 
 }  // namespace
@@ -262,21 +270,37 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
     if (t[i].dtype != dtype || got_r != rows || got_c != cols || t[i].ndim != (cols ? 2 : 1))
       return fail(h, HSPEC_ERR_BAD_SHAPE, "hspec_load_weights: '" + name + "' has the wrong shape or dtype (expected [" +
                                               std::to_string(rows) + (cols ? "," + std::to_string(cols) : "") + "])");
+    auto old = h->w.find(name);
+    if (old != h->w.end()) { cudaFree(old->second.data); h->w.erase(old); }
     Weight w;
-    w.data = t[i].data; w.dtype = dtype; w.rows = rows; w.cols = cols;
+    w.dtype = dtype; w.rows = rows; w.cols = cols;
+    const size_t count = size_t(rows) * size_t(cols ? cols : 1);
+    const size_t bytes = count * (dtype == HSPEC_F32 ? 4 : 2);
+    CUDA_TRY(h, cudaMalloc(&w.data, bytes));
     if (gemm) {
-      if (!make_tmap_bf16_2d(&w.tm, w.data, rows, cols, cols, 128, &errtxt))
+      // bf16 -> fp16: exact for every value with |w| in [2^-17, 65504]; smaller ones lose at most 2^-25
+      const int blocks = int(std::min<size_t>((count + 255) / 256, 148 * 32));
+      bf16_to_f16_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
+                                          reinterpret_cast<__half*>(w.data), count);
+      CUDA_TRY(h, cudaGetLastError());
+      if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, true, &errtxt)) {
+        cudaFree(w.data);
         return fail(h, HSPEC_ERR_BAD_SHAPE, "hspec_load_weights: '" + name + "': " + errtxt);
+      }
       w.has_tm = true;
+    } else {
+      CUDA_TRY(h, cudaMemcpy(w.data, t[i].data, bytes, cudaMemcpyDeviceToDevice));
     }
     h->w[name] = w;
   }
+  CUDA_TRY(h, cudaDeviceSynchronize());
   return HSPEC_OK;
 }
 
 int hspec_destroy(hspec_handle* h) {
   if (!h) return HSPEC_ERR_INVALID_ARG;
   if (h->d_status) cudaFree(h->d_status);
+  for (auto& kv : h->w) cudaFree(kv.second.data);
   delete h;
   return HSPEC_OK;
 }
@@ -345,6 +369,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   float* X = reinterpret_cast<float*>(ws + p.X);
   void* U = ws + p.U;
   float* BIG = reinterpret_cast<float*>(ws + p.BIG);
+  void* LH = ws + p.LH;
   void* Fv = ws + p.Fv;
   void* SINIT = ws + p.SINIT;
   void* DTL = ws + p.DTL;
@@ -358,7 +383,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   auto gemm = [&](const std::string& wname, const void* x, int rows, int mode, void* o, long long ldo) -> cudaError_t {
     const Weight& w = W(wname);
     GemmCall g{};
-    g.tmW = &w.tm; g.x = x; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
+    g.tmW = &w.tm; g.x = x; g.f16 = true; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
     g.mode = mode; g.out = o; g.ldo = ldo;
     g.splits = gemm_pick_splits(rows, g.n_out, g.K, kNumSMs);
     g.splitk_ws = ws + p.SPLITK; g.splitk_ws_bytes = p.splitk_bytes;
@@ -368,8 +393,15 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
 
   CUDA_TRY(h, embed_rows_launch(W("embed").data, in->last_token, c.mask_id, X, B, k, c.D, st)); ++h->launches;
   // S_init = Proj_dS(Proj_r(concat h)): once per step, shared by all layers
-  CUDA_TRY(h, gemm("proj_r", in->last_hidden, B, EPI_STORE_BF16, Fv, c.r));
-  CUDA_TRY(h, gemm("proj_ds", Fv, B, EPI_STORE_BF16, SINIT, d.d_S));
+  {
+    const size_t n_lh = size_t(B) * c.n_fuse * c.D;
+    bf16_to_f16_kernel<<<int(std::min<size_t>((n_lh + 255) / 256, 148 * 8)), 256, 0, st>>>(
+        reinterpret_cast<const __nv_bfloat16*>(in->last_hidden), reinterpret_cast<__half*>(LH), n_lh);
+    ++h->launches;
+    CUDA_TRY(h, cudaGetLastError());
+  }
+  CUDA_TRY(h, gemm("proj_r", LH, B, EPI_STORE_F16, Fv, c.r));
+  CUDA_TRY(h, gemm("proj_ds", Fv, B, EPI_STORE_F16, SINIT, d.d_S));
 
   for (int l = 0; l < c.L; ++l) {
     const std::string pre = "layers." + std::to_string(l) + ".";
@@ -378,8 +410,8 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     CUDA_TRY(h, gemm(pre + "mamba.in_proj", U, M, EPI_STORE_F32, BIG, d.d_in_proj));
     const float* dt_raw = nullptr;
     if (c.dt_rank > 0) {
-      cvt_cols_bf16_kernel<<<(M * c.dt_rank + 255) / 256, 256, 0, st>>>(BIG, d.d_in_proj, c.Di + d.d_xBC, c.dt_rank, M,
-                                                                      reinterpret_cast<__nv_bfloat16*>(DTL));
+      cvt_cols_f16_kernel<<<(M * c.dt_rank + 255) / 256, 256, 0, st>>>(BIG, d.d_in_proj, c.Di + d.d_xBC, c.dt_rank, M,
+                                                                     reinterpret_cast<__half*>(DTL));
       ++h->launches;
       CUDA_TRY(h, cudaGetLastError());
       CUDA_TRY(h, gemm(pre + "mamba.dt_up", DTL, M, EPI_STORE_F32, DT, d.H));
@@ -421,7 +453,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   {
     const Weight& w = W("lm_head");
     GemmCall g{};
-    g.tmW = &w.tm; g.x = U; g.ldx = c.D; g.M = M; g.n_out = c.V; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
+    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = c.V; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
     g.logits = out->logits; g.ldo = c.V;
     g.part_val = reinterpret_cast<float*>(ws + p.AMAXV); g.part_idx = reinterpret_cast<int*>(ws + p.AMAXI);
     g.status = h->d_status;
@@ -445,17 +477,18 @@ size_t hspec_gemm_workspace_bytes(int32_t M, int32_t n_out, int32_t K) {
   return gemm_splitk_bytes(M, n_out, 16) + size_t((n_out + 127) / 128) * M * 8 + 2048;
 }
 
-int hspec_op_gemm(const void* x, const void* Wt, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,
+int hspec_op_gemm(const void* x, const void* Wt, int32_t in_dtype, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,
                   int32_t out_dtype, int32_t accumulate, int32_t splits, void* workspace, size_t workspace_bytes,
                   void* stream) {
   if (!x || !Wt || !y || M < 1 || n_out < 1 || K < 8 || K % 8) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_gemm: bad argument");
   if (accumulate && out_dtype != HSPEC_F32) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_gemm: accumulate needs fp32 output");
   std::string errtxt;
   CUtensorMap tm;
-  if (!make_tmap_bf16_2d(&tm, Wt, n_out, K, K, 128, &errtxt)) return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_gemm: " + errtxt);
+  if (in_dtype != HSPEC_BF16 && in_dtype != HSPEC_F16) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_gemm: x and W must both be bf16 or both fp16");
+  if (!make_tmap_16bit_2d(&tm, Wt, n_out, K, K, 128, in_dtype == HSPEC_F16, &errtxt)) return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_gemm: " + errtxt);
   GemmCall g{};
-  g.tmW = &tm; g.x = x; g.ldx = K; g.M = M; g.n_out = n_out; g.K = K;
-  g.mode = accumulate ? EPI_ACCUM_F32 : (out_dtype == HSPEC_BF16 ? EPI_STORE_BF16 : EPI_STORE_F32);
+  g.tmW = &tm; g.x = x; g.f16 = (in_dtype == HSPEC_F16); g.ldx = K; g.M = M; g.n_out = n_out; g.K = K;
+  g.mode = accumulate ? EPI_ACCUM_F32 : (out_dtype == HSPEC_BF16 ? EPI_STORE_BF16 : out_dtype == HSPEC_F16 ? EPI_STORE_F16 : EPI_STORE_F32);
   g.out = y; g.ldo = ldy;
   g.splits = splits > 0 ? splits : gemm_pick_splits(M, n_out, K, kNumSMs);
   g.splitk_ws = workspace; g.splitk_ws_bytes = workspace_bytes;
@@ -465,7 +498,7 @@ int hspec_op_gemm(const void* x, const void* Wt, void* y, int32_t M, int32_t n_o
   return HSPEC_OK;
 }
 
-int hspec_op_lm_head_argmax(const void* x, const void* Wt, int32_t* ids, float* logits, int32_t M, int32_t V, int32_t K,
+int hspec_op_lm_head_argmax(const void* x, const void* Wt, int32_t in_dtype, int32_t* ids, float* logits, int32_t M, int32_t V, int32_t K,
                             void* workspace, size_t workspace_bytes, void* stream) {
   if (!x || !Wt || !ids || !workspace || M < 1 || V < 1 || K < 8 || K % 8)
     return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_lm_head_argmax: bad argument");
@@ -473,9 +506,9 @@ int hspec_op_lm_head_argmax(const void* x, const void* Wt, int32_t* ids, float* 
   if (workspace_bytes < vt * M * 8 + 1024) return fail(nullptr, HSPEC_ERR_WORKSPACE_TOO_SMALL, "hspec_op_lm_head_argmax: workspace too small");
   std::string errtxt;
   CUtensorMap tm;
-  if (!make_tmap_bf16_2d(&tm, Wt, V, K, K, 128, &errtxt)) return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_lm_head_argmax: " + errtxt);
+  if (!make_tmap_16bit_2d(&tm, Wt, V, K, K, 128, in_dtype == HSPEC_F16, &errtxt)) return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_lm_head_argmax: " + errtxt);
   GemmCall g{};
-  g.tmW = &tm; g.x = x; g.ldx = K; g.M = M; g.n_out = V; g.K = K; g.mode = EPI_ARGMAX; g.splits = 1;
+  g.tmW = &tm; g.x = x; g.f16 = (in_dtype == HSPEC_F16); g.ldx = K; g.M = M; g.n_out = V; g.K = K; g.mode = EPI_ARGMAX; g.splits = 1;
   g.logits = logits; g.ldo = V;
   g.part_val = reinterpret_cast<float*>(workspace);
   g.part_idx = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(workspace) + align_up(vt * M * 4, 256));
@@ -558,10 +591,10 @@ int hspec_debug_gather_kv(const void* pool, const int32_t* page_table_row, int32
   return HSPEC_OK;
 }
 
-int hspec_op_swiglu(const float* gu, void* h_bf16, int32_t M, int32_t F, void* stream) {
-  if (!gu || !h_bf16 || M < 1 || F < 1) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_swiglu: bad argument");
+int hspec_op_swiglu(const float* gu, void* h_f16, int32_t M, int32_t F, void* stream) {
+  if (!gu || !h_f16 || M < 1 || F < 1) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_swiglu: bad argument");
   std::string errtxt;
-  OP_TRY(swiglu_launch(gu, h_bf16, M, F, reinterpret_cast<cudaStream_t>(stream)));
+  OP_TRY(swiglu_launch(gu, h_f16, M, F, reinterpret_cast<cudaStream_t>(stream)));
   return HSPEC_OK;
 }
 

@@ -15,7 +15,8 @@ enum GemmEpilogue : int {
   EPI_STORE_BF16 = 1,   // y bf16 = acc
   EPI_ACCUM_F32 = 2,    // y fp32 += acc   (residual)
   EPI_PARTIAL_F32 = 3,  // K-slice partial (internal)
-  EPI_ARGMAX = 4,       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
+  EPI_ARGMAX = 4,
+  EPI_STORE_F16 = 5,    // y fp16 = acc       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
 };
 
 struct GemmArgs {       // kernel argument block
@@ -24,6 +25,7 @@ struct GemmArgs {       // kernel argument block
   int k_tiles_total, k_tiles_per_split;
   int stages;
   uint32_t tmem_cols;
+  int f16;              // both operands fp16 (else both bf16)
   int mode;
   void* out;
   long long ldo;
@@ -35,8 +37,9 @@ struct GemmArgs {       // kernel argument block
 
 struct GemmCall {       // host-side description of one y = x W^T
   const CUtensorMap* tmW;   // weights [n_out, K], box 128 x 64
-  const void* x;            // bf16 [M, K], row pitch ldx elements
+  const void* x;            // [M, K] in the same 16-bit type as the weights, row pitch ldx elements
   long long ldx;
+  bool f16;                 // operands are fp16 (else bf16)
   int M, n_out, K;
   int mode;                 // EPI_STORE_F32 / EPI_STORE_BF16 / EPI_ACCUM_F32 / EPI_ARGMAX
   void* out;
@@ -50,8 +53,8 @@ struct GemmCall {       // host-side description of one y = x W^T
   uint32_t* status;
 };
 
-bool make_tmap_bf16_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
-                       int box_rows, std::string* err);
+bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
+                       int box_rows, bool f16, std::string* err);
 int gemm_pick_bn(int M);
 int gemm_pick_splits(int M, int n_out, int K, int num_sms);
 size_t gemm_splitk_bytes(int M, int n_out, int splits);
@@ -67,7 +70,7 @@ struct AttnCall {
   int page_table_stride;
   const int32_t* ctx_lens;
   int max_ctx;                      // host bound on ctx_lens
-  void* o;                          // bf16 [B*k, Hq*dh]
+  void* o;                          // fp16 [B*k, Hq*dh]
   int B, k, Hq, Hkv, dh, page_size, window;
   int chunk_tokens;                 // <= 0: choose
   void* ws;
@@ -83,7 +86,7 @@ cudaError_t gather_kv_launch(const void* pool, const int32_t* row, int ctx_len, 
 struct ScanCall {
   const float* zxbcdt; long long ld_in;
   const float* dt_raw;              // [B*k, H] or null (then the dt columns of zxbcdt)
-  const void* s_init;               // bf16 [B, H, P, N] or null
+  const void* s_init;               // fp16 [B, H, P, N] or null
   const float *conv_w, *conv_b, *dt_bias, *A_log, *Dskip;
   float* y_gated;                   // [B*k, Di]
   int B, k, Di, P, N, G, d_conv;
@@ -93,11 +96,11 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launch
 // ---- element-wise kernels (elementwise.cu)
 cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
                               int D, cudaStream_t stream);
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_bf16, int M, int n, float eps, cudaStream_t stream);
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream);
 cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
                                 void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
                                 int qk_norm, cudaStream_t stream);
-cudaError_t swiglu_launch(const float* gu, void* h_bf16, int M, int F, cudaStream_t stream);
+cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream);
 cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream);
 
 }  // namespace hspec

@@ -24,6 +24,25 @@ def assert_close(got, ref, what, tol=TOL):
     return e
 
 
+def rms_err(got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    return float(np.sqrt(np.mean((got - ref) ** 2))) / max(float(np.sqrt(np.mean(ref * ref))), 1e-30)
+
+
+def assert_bf16_close(got, ref, what, ulps=2, floor=1e-3):
+    """For an op whose OUTPUT is stored in bf16: every element within `ulps` bf16 steps (2^-8 relative each) of the
+    reference, plus `floor` x RMS for elements that cancel to near zero."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    assert np.isfinite(got).all(), f"{what}: non-finite output"
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    bound = ulps * 2.0 ** -8 * np.abs(ref) + floor * rms
+    bad = np.abs(got - ref) > bound
+    assert not bad.any(), f"{what}: {int(bad.sum())} elements off by more than {ulps} bf16 steps; worst " \
+                          f"{float(np.max(np.abs(got - ref) / bound)):.2f}x the bound"
+
+
 def bf16_round(a):
     """float array -> values representable in bf16 (as float32), via torch's round-to-nearest-even."""
     return torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16).float().numpy()
