@@ -1,0 +1,458 @@
+#!/usr/bin/env python
+"""Benchmark of the H-Spec block-parallel draft step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" = one call of hspec_draft_block (the whole hot path) over one batch of seeded synthetic requests.
+The headline workload is the concurrency-128 configuration (32B-class shapes, B = 128, k = 16, contexts
+log-uniform in [1024, 32768]); the concurrency-1 and concurrency-32 configurations are measured in the same run
+and reported under "by_concurrency".  Prints ONE JSON line (rank 0).
+
+Multi-GPU: the step has no exchange between requests, so N > 1 runs N independent replicas (one process per
+GPU, different requests per rank, no data-path collective); time is the max over ranks.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+METRIC = "draft tokens/s per B200 at concurrency 1/32/128; % of HBM roofline"
+HEADLINE = "conc128_32b"
+BY_CONCURRENCY = {"1": "latency_8b", "32": "serving_8b", "128": "conc128_32b"}
+FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
+
+
+# ----------------------------------------------------------------------------- helpers
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(FALLBACK_PEAKS, source="fallback")
+
+
+def workload_accounting(cfg, ctx_lens, B, k):
+    """Algorithmic bytes and flops of one step (weights read once, visible target-KV bytes, dense contractions)."""
+    M = B * k
+    mats = [(n, s) for n, (s, kind) in synth.weight_shapes(cfg).items() if kind == "mat" and n != "embed"]
+    weight_bytes = sum(2 * s[0] * s[1] for _, s in mats)
+    flops = 0.0
+    for n, s in mats:
+        rows = B if n in ("proj_r", "proj_ds") else M
+        flops += 2.0 * rows * s[0] * s[1]
+    n_attn = sum(cfg["has_attn"])
+    W = cfg["window"]
+    vis = [min(c, W - 1) if W > 0 else c for c in ctx_lens]
+    kv_bytes_layer = sum(vis) * cfg["Hkv"] * cfg["dh"] * 2 * 2
+    attn_flops_layer = sum(4.0 * k * cfg["Hq"] * cfg["dh"] * (v + (k + 1) / 2) for v in vis)
+    return dict(weight_bytes=weight_bytes, kv_bytes=kv_bytes_layer * n_attn, kv_bytes_per_layer=kv_bytes_layer,
+                gemm_flops=flops, attn_flops=attn_flops_layer * n_attn,
+                s_init_bytes=B * cfg["d_S"] * 2 * (1 + cfg["L"]),
+                drafter_kv_bytes_avoided=sum(ctx_lens) * n_attn * 2 * cfg["Hkv"] * cfg["dh"] * 2)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        for ts, line in self.lines:
+            if t0 is not None and not (t0 <= ts <= t1 + 0.2):
+                continue
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples in the timed region"], samples=0)
+        return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+
+
+def to_np(t):
+    t = t.detach().cpu()
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+
+
+def dist_info():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def max_over_ranks(value, device=None):
+    """Max of a python float over all ranks (identity when not distributed)."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return value
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.barrier()
+
+
+# ----------------------------------------------------------------------------- the CUDA arm
+
+def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True):
+    import paper_2609_24197_b200 as hs
+    cfg = synth.get_config(name)
+    B, k = cfg["B"], cfg["k"]
+    dev = torch.device("cuda", torch.cuda.current_device())
+    weights = synth.make_weights(cfg, device=dev)
+    batch = synth.make_request_batch(cfg, device=dev, seed_offset=1000 * rank)
+    ctx = batch["ctx_lens_host"]
+    max_ctx = max(ctx)
+    drafter = hs.Drafter(cfg, weights, B, k, max_ctx)
+    del weights                                   # the library holds its own (fp16) copies
+    torch.cuda.empty_cache()
+    acct = workload_accounting(cfg, ctx, B, k)
+    stream = torch.cuda.current_stream()
+
+    ids = torch.empty((B, k), dtype=torch.int32, device=dev)
+
+    def step():
+        hs.hspec_draft_block(drafter.handle, batch["page_table"], batch["ctx_lens"], batch["last_hidden"],
+                             batch["last_token"], k, batch["k_pools"], batch["v_pools"], drafter.workspace, ids,
+                             max_ctx=max_ctx)
+
+    hs.hspec_set_profiling(drafter.handle, True)
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    barrier()
+    sampler = ClockSampler(clock_gpu) if clock_gpu is not None else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.25)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    prof = {}
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ev[0].record(stream)
+    for i in range(steps):
+        step()
+        ev[i + 1].record(stream)
+        # per-launch events of this step (reading them waits for the step: nothing else is queued meanwhile)
+        for e in hs.hspec_get_profile(drafter.handle):
+            a = prof.setdefault(e["name"], dict(ms=0.0, n=0, flops=0.0, bytes=0.0))
+            a["ms"] += e["ms"]; a["n"] += 1; a["flops"] += e["flops"]; a["bytes"] += e["bytes"]
+    torch.cuda.synchronize()
+    t1 = time.time()
+    barrier()
+    clocks = sampler.stop(t0, t1) if sampler else None
+    step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    total_ms = max_over_ranks(sum(step_ms), dev)
+    stats = drafter.stats()
+    assert stats["device_status"] == 0, f"device status {stats['device_status']:#x}"
+    launches = stats["launches_last_step"]
+    out = dict(name=name, B=B, k=k, ms_per_step=total_ms / steps, step_ms=step_ms, acct=acct, prof=prof,
+               launches_per_step=launches, clocks=clocks, ctx_sum=sum(ctx), ctx_max=max_ctx, cfg=cfg)
+
+    # without per-launch events, to show what they cost
+    hs.hspec_set_profiling(drafter.handle, False)
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    out["ms_per_step_unprofiled"] = e0.elapsed_time(e1) / steps
+
+    if want_e2e:
+        # through the public call with HOST inputs: pinned page table, context lengths, last hidden state and last
+        # token are copied to the device every step and the draft ids are read back.  The target's KV cache is
+        # device-resident by definition of the method (it is the serving engine's cache, read in place).
+        host = {n: batch[n].cpu().pin_memory() for n in ("page_table", "ctx_lens", "last_hidden", "last_token")}
+        devb = {n: torch.empty_like(batch[n]) for n in host}
+        ids_host = torch.empty((B, k), dtype=torch.int32).pin_memory()
+        h2d = sum(t.numel() * t.element_size() for t in host.values())
+        d2h = ids_host.numel() * 4
+
+        def e2e_step():
+            for n in host:
+                devb[n].copy_(host[n], non_blocking=True)
+            hs.hspec_draft_block(drafter.handle, devb["page_table"], devb["ctx_lens"], devb["last_hidden"],
+                                 devb["last_token"], k, batch["k_pools"], batch["v_pools"], drafter.workspace, ids,
+                                 max_ctx=max_ctx)
+            ids_host.copy_(ids, non_blocking=True)
+            stream.synchronize()
+            return int(ids_host[0, 0])
+        for _ in range(3):
+            e2e_step()
+        barrier()
+        e0.record(stream)
+        for _ in range(steps):
+            e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev) / steps
+        out["e2e"] = dict(ms_per_step=e2e_ms, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h)
+    out["_keep"] = (drafter, batch)
+    return out
+
+
+def cpu_baseline(cfg_name, k_rows=None, rank=0):
+    """Times the oracle as it stands on one request (median context) of the workload, on the host cores."""
+    from oracle import hspec_oracle as O
+    cfg = synth.get_config(cfg_name)
+    k = k_rows or cfg["k"]
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    weights = {n: to_np(t) for n, t in synth.make_weights(cfg, device=dev).items()}
+    if dev == "cuda":
+        torch.cuda.empty_cache()
+    ctx_all = synth.make_ctx_lens(cfg)
+    b = int(np.argsort(ctx_all)[len(ctx_all) // 2])
+    batch = synth.make_request_batch(cfg, ctx_lens=[ctx_all[b]], device="cpu", seed_offset=1000 * rank)
+    t0 = time.time()
+    out = O.draft_block(cfg, weights, [to_np(t) for t in batch["k_pools"]], [to_np(t) for t in batch["v_pools"]],
+                        to_np(batch["page_table"]), batch["ctx_lens_host"], to_np(batch["last_hidden"]),
+                        to_np(batch["last_token"]), k, dtype=np.float32)
+    dt = time.time() - t0
+    cores = len(os.sched_getaffinity(0))
+    return dict(value=k / dt, unit="draft tokens/s", cores=cores, kind="oracle",
+                sample=f"1 request of {cfg_name} (context {ctx_all[b]}, k={k}), numpy float32, {dt:.1f} s",
+                seconds=dt, ids=out["draft_ids"][0].tolist()), (cfg, weights, batch)
+
+
+def kernel_table(res):
+    steps = len(res["step_ms"])
+    total = sum(v["ms"] for v in res["prof"].values())
+    rows = {}
+    for name, v in sorted(res["prof"].items(), key=lambda kv: -kv[1]["ms"]):
+        rows[name] = dict(ms_per_step=round(v["ms"] / steps, 4), launches_per_step=v["n"] // steps,
+                          share=round(v["ms"] / total, 4))
+    return rows
+
+
+def summarize(res, peaks):
+    """Roofline numbers of one workload from the per-launch event times."""
+    steps = len(res["step_ms"])
+    a = res["acct"]
+    ms = res["ms_per_step"]
+    hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
+    hbm_time_ms = (a["weight_bytes"] + a["kv_bytes"]) / (hbm * 1e9) * 1e3
+    tensor_time_ms = (a["gemm_flops"] + a["attn_flops"]) / (tf * 1e12) * 1e3
+    gemm = [v for n, v in res["prof"].items() if n.startswith("gemm:")]
+    gemm_ms = sum(v["ms"] for v in gemm) / steps
+    gemm_flops = sum(v["flops"] for v in gemm) / steps
+    gemm_bytes = sum(v["bytes"] for v in gemm) / steps
+    att = res["prof"].get("attn_partial")
+    n_attn = max(1, sum(res["cfg"]["has_attn"]))
+    att_ms = att["ms"] / steps if att else 0.0
+    att_gbs = a["kv_bytes"] / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
+    gemm_tfs = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    gemm_launches = sum(v["n"] for v in gemm) // steps
+    # the GEMM kernel is bound by whichever of its two rooflines takes longer on this workload
+    gemm_tensor_bound = gemm_flops / (tf * 1e12) >= gemm_bytes / (hbm * 1e9)
+    if gemm_ms >= att_ms:
+        if gemm_tensor_bound:
+            roof = dict(kernel="gemm_tcgen05_kernel", bound="tensor", achieved=round(gemm_tfs, 1), peak=tf,
+                        unit="TFLOP/s", frac=round(gemm_tfs / tf, 4), traffic=None,
+                        note=f"sum over the {gemm_launches} GEMM launches of a step: 2*M*N*K flops / CUDA-event time; "
+                             f"peak = cuBLAS bf16 sustained, of {peaks['source']} (fp16 has the same nominal rate)")
+        else:
+            roof = dict(kernel="gemm_tcgen05_kernel", bound="hbm", achieved=round(gemm_gbs, 1), peak=hbm, unit="GB/s",
+                        frac=round(gemm_gbs / hbm, 4), traffic=None,
+                        note=f"sum over the {gemm_launches} GEMM launches of a step: weight bytes / CUDA-event time; "
+                             f"peak = copy bandwidth, of {peaks['source']}")
+    else:
+        roof = dict(kernel="attn_partial_kernel", bound="hbm", achieved=round(att_gbs, 1), peak=hbm, unit="GB/s",
+                    frac=round(att_gbs / hbm, 4), traffic=None,
+                    note=f"visible target-KV bytes of all attention layers / CUDA-event time, of {peaks['source']}")
+    return dict(
+        ms_per_step=round(ms, 4), draft_tokens_per_s=round(res["B"] * res["k"] / (ms * 1e-3), 1),
+        hbm_roofline_ms=round(hbm_time_ms, 4), hbm_roofline_frac=round(hbm_time_ms / ms, 4),
+        tensor_roofline_ms=round(tensor_time_ms, 4),
+        max_roofline_frac=round(max(hbm_time_ms, tensor_time_ms) / ms, 4),
+        weight_GB=round(a["weight_bytes"] / 1e9, 3), kv_GB=round(a["kv_bytes"] / 1e9, 3),
+        attention=dict(ms_per_step=round(att_ms, 4), achieved_GBs=round(att_gbs, 1), frac_of_hbm=round(att_gbs / hbm, 4),
+                       launches_per_step=n_attn),
+        gemm=dict(ms_per_step=round(gemm_ms, 4), achieved_TFs=round(gemm_tfs, 1), frac_of_tensor=round(gemm_tfs / tf, 4),
+                  achieved_weight_GBs=round(gemm_gbs, 1), frac_of_hbm=round(gemm_gbs / hbm, 4)),
+        roofline=roof, drafter_kv_GB_avoided=round(a["drafter_kv_bytes_avoided"] / 1e9, 3),
+        launches_per_step=res["launches_per_step"],
+        ms_per_step_unprofiled=round(res["ms_per_step_unprofiled"], 4),
+    )
+
+
+# ----------------------------------------------------------------------------- entry points
+
+def main_ours(args):
+    rank, local_rank, world = dist_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the draft step has no CPU path")
+    torch.cuda.set_device(local_rank % torch.cuda.device_count())
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", torch.cuda.current_device()))
+    from paper_2609_24197_b200 import build
+    if rank == 0:
+        build.build()
+    barrier()
+    peaks = load_peaks()
+    head = run_workload(args.workload, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device())
+    s = summarize(head, peaks)
+    e2e_ms = head["e2e"]["ms_per_step"]
+    units = head["B"] * head["k"] * world
+    line = {
+        "metric": METRIC, "value": round(units / (head["ms_per_step"] * 1e-3), 1), "unit": "draft tokens/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": s["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f16 tensor-core operands (bf16 weights widened at load), f32 accumulate; bf16 target KV",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "B": head["B"], "k": head["k"], "ctx_sum": head["ctx_sum"],
+                   "ctx_max": head["ctx_max"], "window": head["cfg"]["window"],
+                   "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "l2": f"inputs larger than L2: {s['weight_GB'] + s['kv_GB']:.1f} GB touched per step, no flush"},
+        "e2e": {"value": round(units / (e2e_ms * 1e-3), 1), "unit": "draft tokens/s",
+                "h2d_bytes_per_step": head["e2e"]["h2d_bytes_per_step"],
+                "d2h_bytes_per_step": head["e2e"]["d2h_bytes_per_step"], "ms_per_step": round(e2e_ms, 4)},
+        "gpu_launches": head["launches_per_step"] * args.steps,
+        "clocks": head["clocks"],
+        "roofline": s["roofline"],
+        "step": {k: s[k] for k in ("hbm_roofline_ms", "hbm_roofline_frac", "tensor_roofline_ms", "max_roofline_frac",
+                                   "weight_GB", "kv_GB", "drafter_kv_GB_avoided", "ms_per_step_unprofiled")},
+        "attention": s["attention"], "gemm": s["gemm"], "kernels": kernel_table(head),
+        "peaks": peaks,
+    }
+    del head["_keep"]
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cb, _ = cpu_baseline(args.workload)
+        cb.pop("ids")
+        line["cpu_baseline"] = {k: (round(v, 3) if isinstance(v, float) else v) for k, v in cb.items()}
+        torch.cuda.empty_cache()
+    if world == 1 and not args.headline_only:
+        byc = {}
+        for conc, name in BY_CONCURRENCY.items():
+            if name == args.workload:
+                byc[conc] = dict(workload=name, draft_tokens_per_s=s["draft_tokens_per_s"], ms_per_step=s["ms_per_step"],
+                                 hbm_roofline_frac=s["hbm_roofline_frac"], max_roofline_frac=s["max_roofline_frac"],
+                                 attention_frac_of_hbm=s["attention"]["frac_of_hbm"])
+                continue
+            r = run_workload(name, args.steps, args.warmup, rank, want_e2e=False)
+            t = summarize(r, peaks)
+            byc[conc] = dict(workload=name, draft_tokens_per_s=t["draft_tokens_per_s"], ms_per_step=t["ms_per_step"],
+                             hbm_roofline_frac=t["hbm_roofline_frac"], max_roofline_frac=t["max_roofline_frac"],
+                             attention_frac_of_hbm=t["attention"]["frac_of_hbm"], gemm=t["gemm"],
+                             kernels=kernel_table(r))
+            del r
+            torch.cuda.empty_cache()
+        line["by_concurrency"] = byc
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def main_reference(args):
+    """The reference arm is the CPU oracle, timed as it stands on a bounded sample of the same workload."""
+    rank, _, world = dist_info()
+    if rank != 0:
+        return
+    cfg = synth.get_config(args.workload)
+    k = cfg["k"]
+    first, state = cpu_baseline(args.workload, k)
+    # keep the whole run within a few minutes: shrink the sample to the first k' block rows (causal prefix property)
+    n_runs = args.steps + args.warmup
+    budget_s = 240.0
+    if first["seconds"] * n_runs > budget_s and k > 1:
+        k = max(1, int(k * budget_s / (first["seconds"] * n_runs)))
+    from oracle import hspec_oracle as O
+    cfg, weights, batch = state
+    pools = [to_np(t) for t in batch["k_pools"]], [to_np(t) for t in batch["v_pools"]]
+    times = []
+    for i in range(n_runs):
+        t0 = time.time()
+        O.draft_block(cfg, weights, pools[0], pools[1], to_np(batch["page_table"]), batch["ctx_lens_host"],
+                      to_np(batch["last_hidden"]), to_np(batch["last_token"]), k, dtype=np.float32)
+        if i >= args.warmup:
+            times.append(time.time() - t0)
+    sec = sum(times) / len(times)
+    value = k / sec
+    cores = len(os.sched_getaffinity(0))
+    sample = f"1 request of {args.workload} (context {batch['ctx_lens_host'][0]}), first {k} of {cfg['k']} block rows per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": "draft tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32 (numpy oracle on host cores)", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": sample},
+        "cpu_baseline": {"value": round(value, 3), "unit": "draft tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": round(value, 3), "unit": "draft tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=sorted(synth.CONFIGS))
+    ap.add_argument("--headline-only", action="store_true", help="skip the concurrency-1 and -32 workloads")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        main_reference(args)
+    else:
+        main_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -143,6 +143,15 @@ typedef struct {
   uint32_t launches_last_step;
 } hspec_stats;
 
+/* One kernel launch of the last step, as recorded when profiling is on. */
+typedef struct {
+  char name[40];     /* kernel label, e.g. "gemm:proj_ds", "attn_partial", "mamba_scan" */
+  float ms;          /* device time between CUDA events recorded around the launch on the step's stream */
+  double flops;      /* algorithmic flops of the launch (GEMMs: 2*M*N*K), 0 if not a contraction */
+  double bytes;      /* algorithmic bytes where the library knows them without the context lengths (GEMMs: the
+                        weight matrix; scan: S_init), else 0 */
+} hspec_prof_entry;
+
 /* Validates the config, creates the handle (host memory only; no weights yet).  Sec. 3.3 / App. B.1. */
 int hspec_init(const hspec_config* cfg, hspec_handle** out);
 /* Device scratch bytes a step of up to (max_batch, max_k, max_pages_per_req) needs. */
@@ -157,6 +166,11 @@ int hspec_destroy(hspec_handle* h);
 /* Message of the last failure on this handle (or of the last failed hspec_init if h is NULL). */
 const char* hspec_last_error(const hspec_handle* h);
 int hspec_get_stats(hspec_handle* h, hspec_stats* out);
+/* Measurement aid: when on, every kernel launch of a step is bracketed by CUDA events on the step's stream. */
+int hspec_set_profiling(hspec_handle* h, int32_t on);
+/* Per-launch times of the LAST step (synchronises its stream).  Returns the number of entries written (<= max_entries)
+ * or a negative hspec_status. */
+int hspec_get_profile(hspec_handle* h, hspec_prof_entry* out, int32_t max_entries);
 
 /* ------------------------------------------------------------------------------------------------
  * Single-operation entry points: the same kernels the step uses, exposed one at a time so that each

@@ -18,7 +18,7 @@ _DT = {torch.bfloat16: 0, torch.float32: 1, torch.int32: 2, torch.float16: 3}
 
 EXPORTS = [
     "hspec_init", "hspec_workspace_bytes", "hspec_load_weights", "hspec_draft_block", "hspec_destroy",
-    "hspec_last_error", "hspec_get_stats", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
+    "hspec_last_error", "hspec_get_stats", "hspec_set_profiling", "hspec_get_profile", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
     "hspec_op_lm_head_argmax", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
 ]
@@ -62,6 +62,10 @@ class hspec_stats(C.Structure):
     _fields_ = [("kernel_launches", C.c_uint64), ("device_status", C.c_uint32), ("launches_last_step", C.c_uint32)]
 
 
+class hspec_prof_entry(C.Structure):
+    _fields_ = [("name", C.c_char * 40), ("ms", C.c_float), ("flops", C.c_double), ("bytes", C.c_double)]
+
+
 _lib = None
 
 
@@ -84,6 +88,8 @@ def load_library(path=None):
     lib.hspec_last_error.argtypes = [C.c_void_p]
     lib.hspec_last_error.restype = C.c_char_p
     lib.hspec_get_stats.argtypes = [C.c_void_p, C.POINTER(hspec_stats)]
+    lib.hspec_set_profiling.argtypes = [C.c_void_p, C.c_int32]
+    lib.hspec_get_profile.argtypes = [C.c_void_p, C.POINTER(hspec_prof_entry), C.c_int32]
     vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
     lib.hspec_op_gemm.argtypes = [vp, vp, i32, vp, i32, i32, i32, i64, i32, i32, i32, vp, sz, vp]
     lib.hspec_gemm_workspace_bytes.argtypes = [i32, i32, i32]
@@ -204,6 +210,20 @@ def hspec_get_stats(handle):
     rc = load_library().hspec_get_stats(handle, C.byref(s))
     return dict(kernel_launches=int(s.kernel_launches), device_status=int(s.device_status),
                 launches_last_step=int(s.launches_last_step), rc=rc)
+
+
+def hspec_set_profiling(handle, on):
+    _check(load_library().hspec_set_profiling(handle, int(on)), handle, "hspec_set_profiling")
+
+
+def hspec_get_profile(handle, max_entries=512):
+    """Per-launch (name, ms, flops, bytes) of the last step; needs hspec_set_profiling(handle, True) before it."""
+    arr = (hspec_prof_entry * max_entries)()
+    n = load_library().hspec_get_profile(handle, arr, max_entries)
+    if n < 0:
+        _check(n, handle, "hspec_get_profile")
+    return [dict(name=arr[i].name.decode(), ms=float(arr[i].ms), flops=float(arr[i].flops), bytes=float(arr[i].bytes))
+            for i in range(n)]
 
 
 # ----------------------------------------------------------------------------- single operations

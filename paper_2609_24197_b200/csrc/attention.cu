@@ -299,7 +299,7 @@ size_t attn_workspace_bytes(int B, int k, int Hq, int Hkv, int dh, int max_ctx, 
   return slabs * R * (dh + 2) * sizeof(float) + 256;
 }
 
-cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, uint64_t* launches, std::string* err) {
+cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (c.dh != 64 && c.dh != 128) { if (err) *err = "attention head dim must be 64 or 128"; return cudaErrorInvalidValue; }
   if (c.Hq % c.Hkv) { if (err) *err = "Hq must be a multiple of Hkv"; return cudaErrorInvalidValue; }
   AttnArgs a{};
@@ -322,6 +322,7 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, uint64_t* l
   dim3 grid(a.max_chunks * a.n_row_tiles, c.Hkv, c.B);
   const int threads = a.RT * 2;
   cudaError_t e;
+  trk_begin(trk, "attn_partial");
   if (c.dh == 128) {
     static bool set128 = false;
     if (!set128) { e = cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); if (e != cudaSuccess) return e; set128 = true; }
@@ -331,13 +332,14 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, uint64_t* l
     if (!set64) { e = cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); if (e != cudaSuccess) return e; set64 = true; }
     attn_partial_kernel<64><<<grid, threads, smem, stream>>>(a);
   }
-  if (launches) ++*launches;
+  trk_end(trk);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   dim3 mgrid(c.B * c.k, c.Hq);
+  trk_begin(trk, "attn_merge");
   if (c.dh == 128) attn_merge_kernel<128><<<mgrid, 128, 0, stream>>>(a);
   else attn_merge_kernel<64><<<mgrid, 64, 0, stream>>>(a);
-  if (launches) ++*launches;
+  trk_end(trk);
   return cudaGetLastError();
 }
 

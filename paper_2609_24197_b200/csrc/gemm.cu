@@ -324,7 +324,7 @@ size_t gemm_splitk_bytes(int M, int n_out, int splits) {
 }
 
 // Launches y = x W^T.  tmW must describe W with box rows 128; x is described here (box rows BN).
-cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launches, std::string* err) {
+cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (g_smem_optin < 0) {
     int dev = 0;
     cudaGetDevice(&dev);
@@ -369,26 +369,29 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launch
   if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BN, c.f16, err)) return cudaErrorInvalidValue;
   dim3 grid((c.M + g.BN - 1) / g.BN, (c.n_out + TILE_W - 1) / TILE_W, splits);
   const size_t smem = size_t(stages) * stage_bytes + fixed;
+  trk_begin(trk, c.label ? c.label : "gemm", 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
   gemm_tcgen05_kernel<<<grid, 192, smem, stream>>>(*c.tmW, tmB, g);
-  if (launches) ++*launches;
+  trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (splits > 1) {
     const long long total = (long long)c.M * c.n_out;
     int blocks = int((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
+    trk_begin(trk, "splitk_reduce", 0, double(splits + 1) * c.M * c.n_out * 4);
     splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M,
                                                      c.n_out, c.out, c.ldo, c.mode);
-    if (launches) ++*launches;
+    trk_end(trk);
     e = cudaGetLastError();
   }
   return e;
 }
 
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
-                                 uint64_t* launches) {
+                                 Tracker* trk) {
+  trk_begin(trk, "argmax_reduce", 0, double(n_tiles) * M * 8);
   argmax_reduce_kernel<<<M, 256, 0, stream>>>(pv, pi, n_tiles, M, ids);
-  if (launches) ++*launches;
+  trk_end(trk);
   return cudaGetLastError();
 }
 

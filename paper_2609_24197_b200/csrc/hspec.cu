@@ -136,12 +136,44 @@ int fail(hspec_handle* h, int code, const std::string& msg);
 
 }  // namespace
 
+namespace hspec {
+
+void Tracker::begin(const char* name, double flops, double bytes) {
+  ++launches;
+  if (!profiling) return;
+  if (used == entries.size()) {
+    Entry e;
+    cudaEventCreate(&e.a);
+    cudaEventCreate(&e.b);
+    entries.push_back(e);
+  }
+  Entry& e = entries[used];
+  memset(e.name, 0, sizeof(e.name));
+  strncpy(e.name, name, sizeof(e.name) - 1);
+  e.flops = flops; e.bytes = bytes;
+  cudaEventRecord(e.a, stream);
+}
+
+void Tracker::end() {
+  if (!profiling) return;
+  cudaEventRecord(entries[used].b, stream);
+  ++used;
+}
+
+void Tracker::destroy() {
+  for (Entry& e : entries) { cudaEventDestroy(e.a); cudaEventDestroy(e.b); }
+  entries.clear();
+  used = 0;
+}
+
+}  // namespace hspec
+
 struct hspec_handle {
   hspec_config cfg;
   Dims d;
   std::unordered_map<std::string, Weight> w;
   std::string err;
-  uint64_t launches = 0;
+  Tracker trk;
   uint32_t launches_last_step = 0;
   uint32_t* d_status = nullptr;
   cudaStream_t last_stream = nullptr;
@@ -301,13 +333,14 @@ int hspec_destroy(hspec_handle* h) {
   if (!h) return HSPEC_ERR_INVALID_ARG;
   if (h->d_status) cudaFree(h->d_status);
   for (auto& kv : h->w) cudaFree(kv.second.data);
+  h->trk.destroy();
   delete h;
   return HSPEC_OK;
 }
 
 int hspec_get_stats(hspec_handle* h, hspec_stats* out) {
   if (!h || !out) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_get_stats: NULL argument");
-  out->kernel_launches = h->launches;
+  out->kernel_launches = h->trk.launches;
   out->launches_last_step = h->launches_last_step;
   out->device_status = 0;
   if (h->d_status) {
@@ -376,45 +409,53 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   float* DT = reinterpret_cast<float*>(ws + p.DT);
   float* YG = reinterpret_cast<float*>(ws + p.YG);
   void *Q = ws + p.Q, *KB = ws + p.KB, *VB = ws + p.VB;
-  const uint64_t launches0 = h->launches;
+  Tracker* trk = &h->trk;
+  trk->begin_step(st);
+  const uint64_t launches0 = trk->launches;
+  const double Md = double(M);
 
   auto W = [&](const std::string& nm) -> const Weight& { return h->w.at(nm); };
   auto fptr = [&](const std::string& nm) { return reinterpret_cast<const float*>(h->w.at(nm).data); };
-  auto gemm = [&](const std::string& wname, const void* x, int rows, int mode, void* o, long long ldo) -> cudaError_t {
+  auto gemm = [&](const std::string& wname, const char* label, const void* x, int rows, int mode, void* o,
+                  long long ldo) -> cudaError_t {
     const Weight& w = W(wname);
     GemmCall g{};
     g.tmW = &w.tm; g.x = x; g.f16 = true; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
     g.mode = mode; g.out = o; g.ldo = ldo;
     g.splits = gemm_pick_splits(rows, g.n_out, g.K, kNumSMs);
     g.splitk_ws = ws + p.SPLITK; g.splitk_ws_bytes = p.splitk_bytes;
-    g.status = h->d_status;
-    return gemm_launch(g, st, &h->launches, &errtxt);
+    g.status = h->d_status; g.label = label;
+    return gemm_launch(g, st, trk, &errtxt);
   };
+  // element-wise launches: bracket with the tracker (name, algorithmic bytes)
+#define EW(name, bytes, call) do { trk->begin(name, 0, bytes); cudaError_t e_ = (call); trk->end(); CUDA_TRY(h, e_); } while (0)
 
-  CUDA_TRY(h, embed_rows_launch(W("embed").data, in->last_token, c.mask_id, X, B, k, c.D, st)); ++h->launches;
+  EW("embed_rows", Md * c.D * 6, embed_rows_launch(W("embed").data, in->last_token, c.mask_id, X, B, k, c.D, st));
   // S_init = Proj_dS(Proj_r(concat h)): once per step, shared by all layers
   {
     const size_t n_lh = size_t(B) * c.n_fuse * c.D;
+    trk->begin("cvt_last_hidden", 0, double(n_lh) * 4);
     bf16_to_f16_kernel<<<int(std::min<size_t>((n_lh + 255) / 256, 148 * 8)), 256, 0, st>>>(
         reinterpret_cast<const __nv_bfloat16*>(in->last_hidden), reinterpret_cast<__half*>(LH), n_lh);
-    ++h->launches;
+    trk->end();
     CUDA_TRY(h, cudaGetLastError());
   }
-  CUDA_TRY(h, gemm("proj_r", LH, B, EPI_STORE_F16, Fv, c.r));
-  CUDA_TRY(h, gemm("proj_ds", Fv, B, EPI_STORE_F16, SINIT, d.d_S));
+  CUDA_TRY(h, gemm("proj_r", "gemm:proj_r", LH, B, EPI_STORE_F16, Fv, c.r));
+  CUDA_TRY(h, gemm("proj_ds", "gemm:proj_ds", Fv, B, EPI_STORE_F16, SINIT, d.d_S));
 
   for (int l = 0; l < c.L; ++l) {
     const std::string pre = "layers." + std::to_string(l) + ".";
     // ---- Mamba-2 mixer from the injected state
-    CUDA_TRY(h, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st)); ++h->launches;
-    CUDA_TRY(h, gemm(pre + "mamba.in_proj", U, M, EPI_STORE_F32, BIG, d.d_in_proj));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st));
+    CUDA_TRY(h, gemm(pre + "mamba.in_proj", "gemm:in_proj", U, M, EPI_STORE_F32, BIG, d.d_in_proj));
     const float* dt_raw = nullptr;
     if (c.dt_rank > 0) {
+      trk->begin("cvt_dt_cols", 0, Md * c.dt_rank * 6);
       cvt_cols_f16_kernel<<<(M * c.dt_rank + 255) / 256, 256, 0, st>>>(BIG, d.d_in_proj, c.Di + d.d_xBC, c.dt_rank, M,
                                                                      reinterpret_cast<__half*>(DTL));
-      ++h->launches;
+      trk->end();
       CUDA_TRY(h, cudaGetLastError());
-      CUDA_TRY(h, gemm(pre + "mamba.dt_up", DTL, M, EPI_STORE_F32, DT, d.H));
+      CUDA_TRY(h, gemm(pre + "mamba.dt_up", "gemm:dt_up", DTL, M, EPI_STORE_F32, DT, d.H));
       dt_raw = DT;
     }
     ScanCall sc{};
@@ -422,15 +463,16 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     sc.conv_w = fptr(pre + "mamba.conv_w"); sc.conv_b = fptr(pre + "mamba.conv_b");
     sc.dt_bias = fptr(pre + "mamba.dt_bias"); sc.A_log = fptr(pre + "mamba.A_log"); sc.Dskip = fptr(pre + "mamba.Dskip");
     sc.y_gated = YG; sc.B = B; sc.k = k; sc.Di = c.Di; sc.P = c.P; sc.N = c.N; sc.G = c.G; sc.d_conv = c.d_conv;
-    CUDA_TRY(h, scan_launch(sc, st, &h->launches, &errtxt));
-    CUDA_TRY(h, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st)); ++h->launches;
-    CUDA_TRY(h, gemm(pre + "mamba.out_proj", U, M, EPI_ACCUM_F32, X, c.D));
+    CUDA_TRY(h, scan_launch(sc, st, trk, &errtxt));
+    EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st));
+    CUDA_TRY(h, gemm(pre + "mamba.out_proj", "gemm:out_proj", U, M, EPI_ACCUM_F32, X, c.D));
     // ---- attention over the target's KV (in place) + the block
     if (c.has_attn[l]) {
-      CUDA_TRY(h, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st)); ++h->launches;
-      CUDA_TRY(h, gemm(pre + "attn.wqkv", U, M, EPI_STORE_F32, BIG, d.d_qkv));
-      CUDA_TRY(h, qk_norm_rope_launch(BIG, fptr(pre + "attn.q_norm"), fptr(pre + "attn.k_norm"), in->ctx_lens, Q, KB, VB, B,
-                                      k, c.Hq, c.Hkv, c.dh, c.rope_theta, c.rms_eps, c.qk_norm, st)); ++h->launches;
+      EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st));
+      CUDA_TRY(h, gemm(pre + "attn.wqkv", "gemm:wqkv", U, M, EPI_STORE_F32, BIG, d.d_qkv));
+      EW("qk_norm_rope", Md * d.d_qkv * 6,
+         qk_norm_rope_launch(BIG, fptr(pre + "attn.q_norm"), fptr(pre + "attn.k_norm"), in->ctx_lens, Q, KB, VB, B, k, c.Hq,
+                             c.Hkv, c.dh, c.rope_theta, c.rms_eps, c.qk_norm, st));
       AttnCall a{};
       a.q = Q; a.kb = KB; a.vb = VB;
       a.k_pool = in->k_pools[c.kv_slot[l]]; a.v_pool = in->v_pools[c.kv_slot[l]];
@@ -438,30 +480,54 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
       a.max_ctx = max_ctx; a.o = U; a.B = B; a.k = k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.dh = c.dh;
       a.page_size = c.page_size; a.window = c.window; a.chunk_tokens = p.attn_chunk;
       a.ws = ws + p.ATT; a.ws_bytes = p.att_bytes;
-      CUDA_TRY(h, attention_launch(a, st, &h->launches, &errtxt));
-      CUDA_TRY(h, gemm(pre + "attn.wo", U, M, EPI_ACCUM_F32, X, c.D));
+      CUDA_TRY(h, attention_launch(a, st, trk, &errtxt));
+      CUDA_TRY(h, gemm(pre + "attn.wo", "gemm:wo", U, M, EPI_ACCUM_F32, X, c.D));
     }
     // ---- SwiGLU MLP
-    CUDA_TRY(h, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st)); ++h->launches;
-    CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
-    CUDA_TRY(h, swiglu_launch(BIG, U, M, c.F, st)); ++h->launches;
-    CUDA_TRY(h, gemm(pre + "mlp.w_down", U, M, EPI_ACCUM_F32, X, c.D));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st));
+    CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
+    EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U, M, c.F, st));
+    CUDA_TRY(h, gemm(pre + "mlp.w_down", "gemm:down", U, M, EPI_ACCUM_F32, X, c.D));
   }
-  if (out->hidden) { CUDA_TRY(h, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st)); ++h->launches; }
+  if (out->hidden) EW("copy_hidden", Md * c.D * 8, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st));
   // ---- final norm, LM head fused with the per-row arg-max
-  CUDA_TRY(h, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st)); ++h->launches;
+  EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st));
   {
     const Weight& w = W("lm_head");
     GemmCall g{};
     g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = c.V; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
     g.logits = out->logits; g.ldo = c.V;
     g.part_val = reinterpret_cast<float*>(ws + p.AMAXV); g.part_idx = reinterpret_cast<int*>(ws + p.AMAXI);
-    g.status = h->d_status;
-    CUDA_TRY(h, gemm_launch(g, st, &h->launches, &errtxt));
-    CUDA_TRY(h, argmax_reduce_launch(g.part_val, g.part_idx, (c.V + 127) / 128, M, out->draft_ids, st, &h->launches));
+    g.status = h->d_status; g.label = "gemm:lm_head_argmax";
+    CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
+    CUDA_TRY(h, argmax_reduce_launch(g.part_val, g.part_idx, (c.V + 127) / 128, M, out->draft_ids, st, trk));
   }
-  h->launches_last_step = uint32_t(h->launches - launches0);
+#undef EW
+  h->launches_last_step = uint32_t(trk->launches - launches0);
   return HSPEC_OK;
+}
+
+int hspec_set_profiling(hspec_handle* h, int32_t on) {
+  if (!h) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_set_profiling: NULL handle");
+  h->trk.profiling = on != 0;
+  return HSPEC_OK;
+}
+
+int hspec_get_profile(hspec_handle* h, hspec_prof_entry* out, int32_t max_entries) {
+  if (!h || (!out && max_entries > 0)) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_get_profile: NULL argument");
+  std::string errtxt;
+  if (!h->trk.profiling) return 0;
+  CUDA_TRY(h, cudaStreamSynchronize(h->trk.stream));
+  int n = 0;
+  for (size_t i = 0; i < h->trk.used && n < max_entries; ++i, ++n) {
+    const Tracker::Entry& e = h->trk.entries[i];
+    float ms = 0.f;
+    CUDA_TRY(h, cudaEventElapsedTime(&ms, e.a, e.b));
+    memset(out[n].name, 0, sizeof(out[n].name));
+    strncpy(out[n].name, e.name, sizeof(out[n].name) - 1);
+    out[n].ms = ms; out[n].flops = e.flops; out[n].bytes = e.bytes;
+  }
+  return n;
 }
 
 // ------------------------------------------------------------------ single-op entry points

@@ -5,10 +5,32 @@
 #include <stdint.h>
 
 #include <string>
+#include <vector>
 
 namespace hspec {
 
 constexpr int GEMM_MAX_STAGES = 8;
+
+// Counts kernel launches and, when profiling is on, brackets each launch with a pair of CUDA events
+// recorded on the launching stream (read back with elapsed() after the stream is synchronised).
+struct Tracker {
+  struct Entry {
+    char name[40];
+    cudaEvent_t a = nullptr, b = nullptr;
+    double flops = 0, bytes = 0;
+  };
+  uint64_t launches = 0;
+  bool profiling = false;
+  cudaStream_t stream = nullptr;
+  std::vector<Entry> entries;
+  size_t used = 0;
+  void begin_step(cudaStream_t st) { used = 0; stream = st; }
+  void begin(const char* name, double flops = 0, double bytes = 0);   // call right before a launch
+  void end();                                                         // call right after it
+  void destroy();
+};
+inline void trk_begin(Tracker* t, const char* name, double flops = 0, double bytes = 0) { if (t) t->begin(name, flops, bytes); }
+inline void trk_end(Tracker* t) { if (t) t->end(); }
 
 enum GemmEpilogue : int {
   EPI_STORE_F32 = 0,    // y fp32 = acc
@@ -51,6 +73,7 @@ struct GemmCall {       // host-side description of one y = x W^T
   float* part_val;
   int* part_idx;
   uint32_t* status;
+  const char* label;        // profile name (may be null)
 };
 
 bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
@@ -58,9 +81,9 @@ bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t
 int gemm_pick_bn(int M);
 int gemm_pick_splits(int M, int n_out, int K, int num_sms);
 size_t gemm_splitk_bytes(int M, int n_out, int splits);
-cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
-                                 uint64_t* launches);
+                                 Tracker* trk);
 
 // ---- attention (attention.cu)
 struct AttnCall {
@@ -78,7 +101,7 @@ struct AttnCall {
 };
 int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms);
 size_t attn_workspace_bytes(int B, int k, int Hq, int Hkv, int dh, int max_ctx, int window, int chunk_tokens);
-cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t gather_kv_launch(const void* pool, const int32_t* row, int ctx_len, int page_size, int Hkv, int dh,
                              void* dst, cudaStream_t stream);
 
@@ -91,7 +114,7 @@ struct ScanCall {
   float* y_gated;                   // [B*k, Di]
   int B, k, Di, P, N, G, d_conv;
 };
-cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launches, std::string* err);
+cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 
 // ---- element-wise kernels (elementwise.cu)
 cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,

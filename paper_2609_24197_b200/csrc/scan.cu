@@ -144,9 +144,190 @@ mamba_scan_kernel(ScanArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Fast path for the serving shapes (P = 64, N = 128 here; any N % 32 == 0, P % 8 == 0 instantiation):
+// one warp per head, HPC heads of one B/C group per CTA.  The state term  Y[t, p] = sum_n C[t, n] S[p, n]
+// is a [k x N] x [N x P] contraction per head and runs on mma.sync m16n8k16 (fp16 in, fp32 out):
+//   * S_init goes from HBM straight into the B fragments: each lane loads 16 contiguous bytes
+//     S[p = 8j + lane/4][32 kp + 8 (lane%4) .. +7], which feed TWO k-steps; the contraction index is
+//     permuted accordingly (a sum does not care), and the A fragments of C use the same permutation;
+//   * no shared-memory staging of the state, every byte of S_init is read exactly once.
+// The conv + SiLU of the group's B and C is computed once per CTA and shared by its heads; the k x k
+// intra-block term, the decay prefix sums (warp shuffle scan), the D skip and the SiLU(z) gate stay fp32.
+template <int P, int N, int MT>
+__global__ void __launch_bounds__(128)
+mamba_scan_mma_kernel(ScanArgs a) {
+  constexpr int HPC = 4;                 // heads (= warps) per CTA
+  constexpr int NT = P / 8;              // n-tiles of the MMA (head channels)
+  constexpr int KP = N / 32;             // k-step pairs
+  constexpr int ROWS = MT * 16;          // padded block positions
+  extern __shared__ __align__(16) float sm[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int h0 = blockIdx.x * HPC, b = blockIdx.y;
+  const int hpg = a.H / a.G;
+  const int g = h0 / hpg;
+  const int k = a.k;
+  float* Bs = sm;                                    // [ROWS][N+1]
+  float* Cs = Bs + ROWS * (N + 1);                   // [ROWS][N+1]
+  float* CB = Cs + ROWS * (N + 1);                   // [ROWS][ROWS+1]   C_t . B_s
+  float* xs = CB + ROWS * (ROWS + 1);                // [ROWS][HPC*P]
+  float* Wm = xs + ROWS * HPC * P;                   // [HPC][ROWS][ROWS+1]
+  float* dts = Wm + HPC * ROWS * (ROWS + 1);         // [HPC][ROWS]
+  float* cum = dts + HPC * ROWS;                     // [HPC][ROWS]
+  __half* C16 = reinterpret_cast<__half*>(cum + HPC * ROWS);   // [ROWS][N] fp16 head of C (rows >= k are zero)
+  __half* C16lo = C16 + ROWS * N;                              // [ROWS][N] fp16 of the remainder C - head
+  const size_t row0 = size_t(b) * k;
+
+  // ---- phase 1: causal conv + SiLU for x of the CTA's heads and B, C of their group
+  constexpr int NCH = HPC * P + 2 * N;
+  for (int idx = tid; idx < ROWS * NCH; idx += 128) {
+    const int i = idx / NCH, cc = idx % NCH;
+    float v = 0.f;
+    if (i < k) {
+      int ch;
+      if (cc < HPC * P) ch = h0 * P + cc;
+      else if (cc < HPC * P + N) ch = a.Di + g * N + (cc - HPC * P);
+      else ch = a.Di + a.G * N + g * N + (cc - HPC * P - N);
+      float acc = a.conv_b[ch];
+      for (int j = 0; j < a.d_conv; ++j) {
+        const int src = i - (a.d_conv - 1) + j;
+        if (src >= 0) acc += a.conv_w[ch * a.d_conv + j] * a.zxbcdt[(row0 + src) * a.ld_in + a.Di + ch];
+      }
+      v = silu_f(acc);
+    }
+    if (cc < HPC * P) xs[i * HPC * P + cc] = v;
+    else if (cc < HPC * P + N) Bs[i * (N + 1) + (cc - HPC * P)] = v;
+    else {
+      // C = hi + lo with both parts fp16: the tensor-core contraction then carries ~22 bits of C
+      const __half hi = __float2half_rn(v);
+      Cs[i * (N + 1) + (cc - HPC * P - N)] = v;
+      C16[i * N + (cc - HPC * P - N)] = hi;
+      C16lo[i * N + (cc - HPC * P - N)] = __float2half_rn(v - __half2float(hi));
+    }
+  }
+  // ---- per head (warp): dt, inclusive prefix sum of dt * A over the block positions
+  const int h = h0 + warp;
+  {
+    float dt = 0.f, dA = 0.f;
+    if (lane < k) {
+      const float raw = a.dt_raw ? a.dt_raw[(row0 + lane) * a.H + h]
+                                 : a.zxbcdt[(row0 + lane) * a.ld_in + a.Di + a.d_xBC + h];
+      dt = softplus_f(raw + a.dt_bias[h]);
+      dA = dt * (-expf(a.A_log[h]));
+    }
+    float c = dA;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const float up = __shfl_up_sync(0xffffffffu, c, off);
+      if (lane >= off) c += up;
+    }
+    if (lane < ROWS) { dts[warp * ROWS + lane] = dt; cum[warp * ROWS + lane] = c; }
+  }
+  __syncthreads();
+  // ---- phase 2: CB[t][s] = C_t . B_s (shared by the CTA's heads), s <= t
+  for (int idx = tid; idx < ROWS * ROWS; idx += 128) {
+    const int t = idx / ROWS, s2 = idx % ROWS;
+    float dot = 0.f;
+    if (s2 <= t && t < k) {
+      const float* cr = Cs + t * (N + 1);
+      const float* br = Bs + s2 * (N + 1);
+#pragma unroll 8
+      for (int n = 0; n < N; ++n) dot += cr[n] * br[n];
+    }
+    CB[t * (ROWS + 1) + s2] = dot;
+  }
+  __syncthreads();
+  // ---- per head: W[t][s] = exp(c_t - c_s) dt_s CB[t][s]
+  float* Wh = Wm + warp * ROWS * (ROWS + 1);
+  for (int idx = lane; idx < ROWS * ROWS; idx += 32) {
+    const int t = idx / ROWS, s2 = idx % ROWS;
+    float w = 0.f;
+    if (s2 <= t && t < k) w = expf(cum[warp * ROWS + t] - cum[warp * ROWS + s2]) * dts[warp * ROWS + s2] * CB[t * (ROWS + 1) + s2];
+    Wh[t * (ROWS + 1) + s2] = w;
+  }
+  __syncwarp();
+
+  // ---- phase 3: state term on the tensor cores, S_init read once from global into the B fragments
+  const int gq = lane >> 2, tq = lane & 3;
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int j = 0; j < NT; ++j) { acc[mt][j][0] = acc[mt][j][1] = acc[mt][j][2] = acc[mt][j][3] = 0.f; }
+  if (a.s_init != nullptr) {
+    const __half* S = a.s_init + (size_t(b) * a.H + h) * P * N;
+#pragma unroll
+    for (int kp = 0; kp < KP; ++kp) {
+      uint4 sv[NT];
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        sv[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + kp * 32 + tq * 8));
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const uint4 c_lo = *reinterpret_cast<const uint4*>(C16 + (mt * 16 + gq) * N + kp * 32 + tq * 8);
+        const uint4 c_hi = *reinterpret_cast<const uint4*>(C16 + (mt * 16 + gq + 8) * N + kp * 32 + tq * 8);
+        const uint4 r_lo = *reinterpret_cast<const uint4*>(C16lo + (mt * 16 + gq) * N + kp * 32 + tq * 8);
+        const uint4 r_hi = *reinterpret_cast<const uint4*>(C16lo + (mt * 16 + gq + 8) * N + kp * 32 + tq * 8);
+        const uint32_t a0[4] = {c_lo.x, c_hi.x, c_lo.y, c_hi.y};     // first virtual k-step
+        const uint32_t a1[4] = {c_lo.z, c_hi.z, c_lo.w, c_hi.w};     // second virtual k-step
+        const uint32_t e0[4] = {r_lo.x, r_hi.x, r_lo.y, r_hi.y};     // the same two k-steps of the remainder
+        const uint32_t e1[4] = {r_lo.z, r_hi.z, r_lo.w, r_hi.w};
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          mma_f16_16816(acc[mt][j], a0, sv[j].x, sv[j].y);
+          mma_f16_16816(acc[mt][j], a1, sv[j].z, sv[j].w);
+          mma_f16_16816(acc[mt][j], e0, sv[j].x, sv[j].y);
+          mma_f16_16816(acc[mt][j], e1, sv[j].z, sv[j].w);
+        }
+      }
+    }
+  }
+  // ---- epilogue: decay, intra-block term, D skip, gate
+  const float Dh = a.Dskip[h];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int t = mt * 16 + gq + half * 8;
+      if (t >= k) continue;
+      const float dec = expf(cum[warp * ROWS + t]);
+      float y[NT][2];
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        const float2 xv = *reinterpret_cast<const float2*>(xs + t * HPC * P + warp * P + j * 8 + tq * 2);
+        y[j][0] = dec * acc[mt][j][half * 2] + Dh * xv.x;
+        y[j][1] = dec * acc[mt][j][half * 2 + 1] + Dh * xv.y;
+      }
+      for (int s2 = 0; s2 <= t; ++s2) {
+        const float w = Wh[t * (ROWS + 1) + s2];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          const float2 xv = *reinterpret_cast<const float2*>(xs + s2 * HPC * P + warp * P + j * 8 + tq * 2);
+          y[j][0] += w * xv.x;
+          y[j][1] += w * xv.y;
+        }
+      }
+      const size_t row = row0 + t;
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        const int col = h * P + j * 8 + tq * 2;
+        const float2 z = *reinterpret_cast<const float2*>(a.zxbcdt + row * a.ld_in + col);
+        *reinterpret_cast<float2*>(a.y + row * a.Di + col) = make_float2(y[j][0] * silu_f(z.x), y[j][1] * silu_f(z.y));
+      }
+    }
+  }
+}
+
+template <int MT>
+size_t scan_mma_smem() {
+  constexpr int P = 64, N = 128, HPC = 4, ROWS = MT * 16;
+  return sizeof(float) * (2 * ROWS * (N + 1) + ROWS * (ROWS + 1) + ROWS * HPC * P + HPC * ROWS * (ROWS + 1) + 2 * HPC * ROWS) +
+         sizeof(__half) * 2 * ROWS * N;
+}
+
 }  // namespace
 
-cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launches, std::string* err) {
+cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (c.k < 1 || c.k > KMAX) { if (err) *err = "scan: k out of range"; return cudaErrorInvalidValue; }
   if (c.Di % c.P) { if (err) *err = "scan: Di must be a multiple of P"; return cudaErrorInvalidValue; }
   ScanArgs a{};
@@ -156,6 +337,25 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launch
   a.d_conv = c.d_conv; a.d_xBC = c.Di + 2 * c.G * c.N;
   a.NP = c.N + 1;                                    // odd pitch: threads of a warp own consecutive p
   if (a.H % c.G) { if (err) *err = "scan: heads must divide into groups"; return cudaErrorInvalidValue; }
+  // serving shapes: tensor-core path (needs 8-byte aligned rows for the float2 accesses)
+  if (c.P == 64 && c.N == 128 && (a.H / c.G) % 4 == 0 && c.ld_in % 2 == 0 && c.Di % 2 == 0) {
+    const bool two = c.k > 16;
+    const size_t smem_f = two ? scan_mma_smem<2>() : scan_mma_smem<1>();
+    static bool set1 = false, set2 = false;
+    bool& was_set = two ? set2 : set1;
+    if (!was_set) {
+      cudaError_t e = two ? cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f))
+                          : cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f));
+      if (e != cudaSuccess) return e;
+      was_set = true;
+    }
+    dim3 grid_f(a.H / 4, c.B);
+    trk_begin(trk, "mamba_scan", 2.0 * c.B * c.k * a.H * c.P * c.N, double(c.B) * a.H * c.P * c.N * 2);
+    if (two) mamba_scan_mma_kernel<64, 128, 2><<<grid_f, 128, smem_f, stream>>>(a);
+    else mamba_scan_mma_kernel<64, 128, 1><<<grid_f, 128, smem_f, stream>>>(a);
+    trk_end(trk);
+    return cudaGetLastError();
+  }
   const size_t smem = sizeof(float) * (size_t(KMAX) * c.P + 2 * size_t(KMAX) * c.N + KMAX * KMAX + 3 * KMAX +
                                        size_t(c.P) * a.NP);
   static size_t smem_set = 0;
@@ -165,8 +365,9 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, uint64_t* launch
     smem_set = smem;
   }
   dim3 grid(a.H, c.B);
+  trk_begin(trk, "mamba_scan", 0, double(c.B) * a.H * c.P * c.N * 2);
   mamba_scan_kernel<<<grid, SCAN_THREADS, smem, stream>>>(a);
-  if (launches) ++*launches;
+  trk_end(trk);
   return cudaGetLastError();
 }
 

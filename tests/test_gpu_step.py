@@ -104,6 +104,7 @@ def _full_size(name, n_check, **over):
     order = np.argsort(batch["ctx_lens_host"])
     pick = sorted(set([int(order[-1]), int(order[0])][:n_check]))
     r = check_step(cfg, drafter, w, batch, cfg["k"], requests=pick, dtype=np.float32, what=name)
+    print(name, "requests", pick, r)
     drafter.close()
     del w, batch
     torch.cuda.empty_cache()
