@@ -144,7 +144,7 @@ def barrier():
 
 # ----------------------------------------------------------------------------- the CUDA arm
 
-def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True):
+def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=False):
     import paper_2609_24197_b200 as hs
     cfg = synth.get_config(name)
     B, k = cfg["B"], cfg["k"]
@@ -199,6 +199,11 @@ def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True):
     out = dict(name=name, B=B, k=k, ms_per_step=total_ms / steps, step_ms=step_ms, acct=acct, prof=prof,
                launches_per_step=launches, clocks=clocks, ctx_sum=sum(ctx), ctx_max=max_ctx, cfg=cfg)
 
+    if lean:                                       # launch-list captures: nothing but warm-up + timed steps
+        out["ms_per_step_unprofiled"] = float("nan")
+        out["e2e"] = dict(ms_per_step=float("nan"), h2d_bytes_per_step=0, d2h_bytes_per_step=0)
+        out["_keep"] = (drafter, batch)
+        return out
     # without per-launch events, to show what they cost
     hs.hspec_set_profiling(drafter.handle, False)
     step()
@@ -344,7 +349,8 @@ def main_ours(args):
         build.build()
     barrier()
     peaks = load_peaks()
-    head = run_workload(args.workload, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device())
+    head = run_workload(args.workload, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device(),
+                        lean=args.lean)
     s = summarize(head, peaks)
     e2e_ms = head["e2e"]["ms_per_step"]
     units = head["B"] * head["k"] * world
@@ -447,6 +453,7 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=sorted(synth.CONFIGS))
     ap.add_argument("--headline-only", action="store_true", help="skip the concurrency-1 and -32 workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lean", action="store_true", help="only warm-up + timed steps (for profiler launch lists)")
     args = ap.parse_args()
     if args.impl == "reference":
         main_reference(args)
