@@ -211,9 +211,10 @@ int hspec_op_qk_norm_rope(const float* qkv, const float* q_norm_w, const float* 
 /* Block-query GQA attention over the target's paged KV (read in place) plus the block's causal keys (Sec. 3.3.2).
  * q/kb/vb as produced by hspec_op_qk_norm_rope; k_pool/v_pool bf16 [num_pages, page_size, Hkv, dh];
  * o fp16 [B*k, Hq*dh].  window 0 = full.  max_ctx: host upper bound on ctx_lens (0 = stride*page_size).
- * chunk_tokens <= 0 lets the library pick the context split. */
+ * chunk_tokens <= 0 lets the library pick the context split (otherwise rounded up to a multiple of 128).
+ * num_pages = pages in each pool. */
 int hspec_op_attention(const void* q, const void* kb, const void* vb, const void* k_pool, const void* v_pool,
-                       const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens,
+                       int64_t num_pages, const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens,
                        int32_t max_ctx, void* o, int32_t B, int32_t k, int32_t Hq, int32_t Hkv, int32_t dh,
                        int32_t page_size, int32_t window, int32_t chunk_tokens, void* workspace,
                        size_t workspace_bytes, void* stream);

@@ -98,7 +98,7 @@ def load_library(path=None):
     lib.hspec_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, f32, vp]
     lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
     lib.hspec_op_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, vp]
-    lib.hspec_op_attention.argtypes = [vp, vp, vp, vp, vp, vp, i32, vp, i32, vp, i32, i32, i32, i32, i32, i32, i32,
+    lib.hspec_op_attention.argtypes = [vp, vp, vp, vp, vp, i64, vp, i32, vp, i32, vp, i32, i32, i32, i32, i32, i32, i32,
                                        i32, vp, sz, vp]
     lib.hspec_attention_workspace_bytes.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32]
     lib.hspec_attention_workspace_bytes.restype = sz
@@ -279,7 +279,7 @@ def hspec_op_attention(q, kb, vb, k_pool, v_pool, page_table, ctx_lens, max_ctx,
                        window, chunk_tokens, workspace):
     _check(load_library().hspec_op_attention(
         _ptr(q, torch.bfloat16), _ptr(kb, torch.bfloat16), _ptr(vb, torch.bfloat16), _ptr(k_pool, torch.bfloat16),
-        _ptr(v_pool, torch.bfloat16), _ptr(page_table, torch.int32), int(page_table.shape[1]),
+        _ptr(v_pool, torch.bfloat16), int(k_pool.shape[0]), _ptr(page_table, torch.int32), int(page_table.shape[1]),
         _ptr(ctx_lens, torch.int32), int(max_ctx), _ptr(o, torch.float16), B, k, Hq, Hkv, dh, page_size, window,
         chunk_tokens, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
         None, "hspec_op_attention")

@@ -10,6 +10,8 @@
 #include "common.cuh"
 #include "kernels.h"
 
+#include <cstdlib>
+
 namespace hspec {
 
 namespace {
@@ -281,14 +283,15 @@ int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms) {
   if (nsplit < 1) nsplit = 1;
   if (nsplit > 32) nsplit = 32;
   int chunk = (lmax + nsplit - 1) / nsplit;
-  chunk = ((chunk + KT - 1) / KT) * KT;
+  chunk = ((chunk + 127) / 128) * 128;
   if (chunk < 256) chunk = 256;
   if (chunk > 4096) chunk = 4096;
   return chunk;
 }
 
 static int max_chunks_of(int max_ctx, int window, int chunk) {
-  int lmax = (window > 0 && window < max_ctx) ? window : max_ctx;
+  // with a window the visible range may start up to 15 tokens earlier (page-aligned chunk grid of the tcgen05 path)
+  int lmax = (window > 0 && window + 15 < max_ctx) ? window + 15 : max_ctx;
   int n = (lmax + chunk - 1) / chunk;
   return n < 1 ? 1 : n;
 }
@@ -315,6 +318,10 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* tr
   if (c.k > KT) { if (err) *err = "block longer than one key tile"; return cudaErrorInvalidValue; }
   const size_t need = attn_workspace_bytes(c.B, c.k, c.Hq, c.Hkv, c.dh, c.max_ctx, c.window, c.chunk_tokens);
   if (c.ws == nullptr || c.ws_bytes < need) { if (err) *err = "attention workspace too small"; return cudaErrorInvalidValue; }
+  {
+    static const bool legacy = [] { const char* e = getenv("HSPEC_ATTN_MMA_SYNC"); return e && e[0] == '1'; }();
+    if (!legacy && attention_tc_supported(c)) return attention_tc_launch(c, a.max_chunks, stream, trk, err);
+  }
   const size_t slabs = size_t(c.B) * c.Hkv * a.max_chunks;
   a.ws_o = reinterpret_cast<float*>(c.ws);
   a.ws_ml = a.ws_o + slabs * a.R * c.dh;

@@ -476,6 +476,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
       AttnCall a{};
       a.q = Q; a.kb = KB; a.vb = VB;
       a.k_pool = in->k_pools[c.kv_slot[l]]; a.v_pool = in->v_pools[c.kv_slot[l]];
+      a.num_pages = in->num_pages; a.status = h->d_status;
       a.page_table = in->page_table; a.page_table_stride = in->page_table_stride; a.ctx_lens = in->ctx_lens;
       a.max_ctx = max_ctx; a.o = U; a.B = B; a.k = k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.dh = c.dh;
       a.page_size = c.page_size; a.window = c.window; a.chunk_tokens = p.attn_chunk;
@@ -620,7 +621,7 @@ int hspec_op_qk_norm_rope(const float* qkv, const float* qw, const float* kw, co
 }
 
 static int resolve_chunk(int B, int Hkv, int max_ctx, int window, int chunk_tokens) {
-  if (chunk_tokens > 0) return ((chunk_tokens + 63) / 64) * 64;
+  if (chunk_tokens > 0) return ((chunk_tokens + 127) / 128) * 128;
   return attn_pick_chunk(B, Hkv, max_ctx, window, kNumSMs);
 }
 
@@ -630,7 +631,7 @@ size_t hspec_attention_workspace_bytes(int32_t B, int32_t k, int32_t Hq, int32_t
 }
 
 int hspec_op_attention(const void* q, const void* kb, const void* vb, const void* k_pool, const void* v_pool,
-                       const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens, int32_t max_ctx,
+                       int64_t num_pages, const int32_t* page_table, int32_t page_table_stride, const int32_t* ctx_lens, int32_t max_ctx,
                        void* o, int32_t B, int32_t k, int32_t Hq, int32_t Hkv, int32_t dh, int32_t page_size, int32_t window,
                        int32_t chunk_tokens, void* workspace, size_t workspace_bytes, void* stream) {
   if (!q || !kb || !vb || !k_pool || !v_pool || !page_table || !ctx_lens || !o || !workspace || B < 1 || k < 1 ||
@@ -639,6 +640,8 @@ int hspec_op_attention(const void* q, const void* kb, const void* vb, const void
   std::string errtxt;
   AttnCall a{};
   a.q = q; a.kb = kb; a.vb = vb; a.k_pool = k_pool; a.v_pool = v_pool; a.page_table = page_table;
+  a.num_pages = num_pages; a.status = global_status();
+  if (!a.status) return fail(nullptr, HSPEC_ERR_CUDA, "hspec_op_attention: cannot allocate the status word");
   a.page_table_stride = page_table_stride; a.ctx_lens = ctx_lens;
   a.max_ctx = max_ctx > 0 ? max_ctx : page_table_stride * page_size;
   a.o = o; a.B = B; a.k = k; a.Hq = Hq; a.Hkv = Hkv; a.dh = dh; a.page_size = page_size; a.window = window;

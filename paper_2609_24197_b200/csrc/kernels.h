@@ -89,6 +89,8 @@ cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, in
 struct AttnCall {
   const void *q, *kb, *vb;          // bf16 [B*k, Hq, dh], [B*k, Hkv, dh] x2
   const void *k_pool, *v_pool;      // bf16 [num_pages, page, Hkv, dh]
+  long long num_pages;
+  uint32_t* status;                 // device status word for bounded waits
   const int32_t* page_table;
   int page_table_stride;
   const int32_t* ctx_lens;
@@ -102,6 +104,8 @@ struct AttnCall {
 int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms);
 size_t attn_workspace_bytes(int B, int k, int Hq, int Hkv, int dh, int max_ctx, int window, int chunk_tokens);
 cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
+bool attention_tc_supported(const AttnCall& c);
+cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t gather_kv_launch(const void* pool, const int32_t* row, int ctx_len, int page_size, int Hkv, int dh,
                              void* dst, cudaStream_t stream);
 

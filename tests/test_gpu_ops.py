@@ -217,7 +217,7 @@ def _attn_case(hs, B, k, Hq, Hkv, dh, ctxs, window, chunk, seed=0, poison=True):
         sl = slice(b * k, (b + 1) * k)
         ref = O.attention_paged(to_np(q[sl]), kp, vp, pt[b], ctxs[b], to_np(kb[sl]), to_np(vb[sl]), window=window)
         # P enters its MMA in bf16 (V is the target's bf16 cache, and both MMA operands share a type): 2^-9 per weight
-        worst = max(worst, assert_close(got[b], ref, f"attention request {b} ctx {ctxs[b]}", tol=1.2e-2))
+        worst = max(worst, assert_close(got[b], ref, f"attention request {b} ctx {ctxs[b]}", tol=2e-2))
         assert rms_err(got[b], ref) < 2e-3, f"attention request {b}: RMS error {rms_err(got[b], ref):.2e}"
     return worst
 
