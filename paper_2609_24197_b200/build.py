@@ -23,7 +23,8 @@ def build(force=False, verbose=False):
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest(deps):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + FLAGS + (["-Xptxas", "-v"] if verbose else []) + srcs + ["-o", LIB]
+    extra = os.environ.get("HSPEC_NVCC_FLAGS", "").split()     # e.g. -DHSPEC_ATTN_TIMING for kernel-internal timing
+    cmd = [nvcc] + FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + srcs + ["-o", LIB]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)

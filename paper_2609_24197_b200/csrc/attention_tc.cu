@@ -8,15 +8,17 @@
 //               of this KV head exactly as the target stored them).  The ragged end of the context and the block's
 //               own keys/values go through plain 16-byte loads with zero fill, so no garbage row is ever multiplied.
 //   warp 5      issues S = Q K^T (A = Q, B = K tile, both K-major) into one of two TMEM S buffers, then
-//               O += P V (A = P from shared memory, B = V tile as an MN-major operand) into the TMEM O buffer.
+//               O += P V (A = P read from TMEM, B = V tile as an MN-major operand) into the TMEM O buffer.
 //   warps 0..3  softmax: thread = query row = TMEM lane.  Reads its S row (128 fp32), masks by selection, keeps a
 //               reference maximum that only moves when the row maximum outgrows it by 2^8 (then, rarely, rescales
-//               its O row in TMEM), writes P (bf16) into shared memory in the MMA's K-major swizzled layout.
+//               its O row in TMEM), writes P (bf16, two keys per 32-bit column) into one of two TMEM P buffers.
 //
 // The MMA warp issues S_{t+1} before it waits for P_t, so the tensor core works on the next tile's scores while
 // the softmax warps are busy, and the producer runs NS tiles ahead.  Every wait is bounded.
 #include "common.cuh"
 #include "kernels.h"
+
+#include <cstdio>
 
 namespace hspec {
 
@@ -24,7 +26,7 @@ namespace {
 
 constexpr int KT = 128;            // keys per tile
 constexpr int DH = 128;
-constexpr int NS = 2;              // K/V stages in shared memory
+constexpr int NS = 3;              // K/V stages in shared memory
 constexpr int HALF_BYTES = 128 * 128;            // [128 rows x 64 bf16] = 16 KiB
 constexpr int TILE_BYTES = 2 * HALF_BYTES;       // one operand tile [128 x 128] bf16
 constexpr float NEG = -1.0e30f;
@@ -97,7 +99,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+// 2^x by the special-function unit alone (flush-to-zero form: no range fix-up code around it)
+__device__ __forceinline__ float ex2_ftz(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// D[tmem] (+)= A[tmem] * B[smem desc]: the A operand (128 rows x 16 bf16 = 8 columns) is read from tensor memory
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 
 // instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128, A K-major, B K-major or MN-major
 __device__ __forceinline__ uint32_t idesc_bf16_128x128(bool b_mn_major) {
@@ -146,8 +164,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sQ = smem;                               // 32 KiB
-  uint8_t* sP = sQ + TILE_BYTES;                    // 2 x 32 KiB
-  uint8_t* sKV = sP + 2 * TILE_BYTES;               // NS x (K 32 KiB + V 32 KiB)
+  uint8_t* sKV = sQ + TILE_BYTES;                   // NS x (K 32 KiB + V 32 KiB)
   AttnTcBars* bars = reinterpret_cast<AttnTcBars*>(sKV + NS * 2 * TILE_BYTES);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -185,6 +202,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   const uint32_t tmem = bars->tmem_base;
   const uint32_t tmem_o = tmem;                     // columns [0, 128)
   const uint32_t tmem_s0 = tmem + 128;              // S buffers: columns [128, 256) and [256, 384)
+  const uint32_t tmem_p0 = tmem + 384;              // P buffers (bf16 pairs): columns [384, 448) and [448, 512)
   volatile uint32_t* abort_flag = &bars->abort_flag;
   const int row0 = rt * 128;
 
@@ -286,12 +304,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             !mbar_wait(smem_u32(&bars->v_full[s]), (t / NS) & 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t vbase = smem_u32(sKV + s * 2 * TILE_BYTES + TILE_BYTES);
-        const uint32_t pbase = smem_u32(sP + (t & 1) * TILE_BYTES);
 #pragma unroll
         for (int ks = 0; ks < KT / 16; ++ks) {
-          const uint64_t da = umma_desc_kmajor_sw128(pbase + (ks >> 2) * HALF_BYTES) + uint64_t((ks & 3) * 2);
+          // A = 16 keys of P = 8 TMEM columns of the P buffer; B = the same 16 keys (rows) of V
           const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
-          umma_bf16(tmem_o, da, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+          umma_bf16_ts(tmem_o, tmem_p0 + (t & 1) * 64 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars->kv_empty[s]));
         umma_commit(smem_u32(&bars->pv_done[t & 1]));
@@ -322,24 +339,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     const uint32_t lane_base = uint32_t(warp * 32) << 16;
     float m_ref = NEG, l_sum = 0.f;
     bool ok = true;
+#ifdef HSPEC_ATTN_TIMING
+    long long t_wait_s = 0, t_wait_pv = 0, t_start = clock64(), t_mark;
+#endif
     for (int t = 0; t < g.T && ok; ++t) {
+#ifdef HSPEC_ATTN_TIMING
+      t_mark = clock64();
+#endif
       if (!mbar_wait(smem_u32(&bars->s_ready[t & 1]), (t >> 1) & 1)) { ok = false; break; }
+#ifdef HSPEC_ATTN_TIMING
+      t_wait_s += clock64() - t_mark;
+#endif
       tc_fence_after();
       float s[KT];
 #pragma unroll
       for (int j = 0; j < KT / 32; ++j) tmem_ld32(tmem_s0 + (t & 1) * 128 + lane_base + j * 32, reinterpret_cast<uint32_t*>(s + j * 32));
       tmem_ld_wait();
-      // ---- scale and mask by selection
-      float mx = -INFINITY;
+      // ---- mask by selection (raw scores; the positive scale is folded into the exponent below)
       if (t < g.n_full) {
         const int key0 = g.p_begin + t * KT;
-        const bool edge = a.window > 0 && key0 < g.base + 16 + a.k;       // leading edge of the window
+        if (a.window > 0 && key0 < g.base + 16 + a.k) {                   // leading edge of the window
 #pragma unroll
-        for (int j = 0; j < KT; ++j) {
-          float v = s[j] * a.scale_log2;
-          if (edge && (ctx + i_blk) - (key0 + j) >= a.window) v = -INFINITY;
-          s[j] = v;
-          mx = fmaxf(mx, v);
+          for (int j = 0; j < KT; ++j)
+            if ((ctx + i_blk) - (key0 + j) >= a.window) s[j] = -INFINITY;
         }
       } else {
         int n_prefix, prefix_start, n_block;
@@ -352,15 +374,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             const int jb = j - n_prefix;
             vis = jb < n_block && jb <= i_blk && (a.window <= 0 || i_blk - jb < a.window);
           }
-          const float v = vis ? s[j] * a.scale_log2 : -INFINITY;
-          s[j] = v;
-          mx = fmaxf(mx, v);
+          if (!vis) s[j] = -INFINITY;
         }
       }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};         // four chains instead of one
+#pragma unroll
+      for (int j = 0; j < KT; j += 4) {
+        mx4[0] = fmaxf(mx4[0], s[j]); mx4[1] = fmaxf(mx4[1], s[j + 1]);
+        mx4[2] = fmaxf(mx4[2], s[j + 2]); mx4[3] = fmaxf(mx4[3], s[j + 3]);
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
       // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY
       float factor = 1.f;
       const bool grow = mx > m_ref + LAZY;
-      if (grow) { factor = exp2f(m_ref - mx); m_ref = mx; }
+      if (grow) { factor = ex2_ftz(m_ref - mx); m_ref = mx; }
       if (t > 0 && __any_sync(0xffffffffu, grow)) {
         // O of the tiles so far must be complete before it is rescaled
         if (!mbar_wait(smem_u32(&bars->pv_done[(t - 1) & 1]), ((t - 1) >> 1) & 1)) { ok = false; break; }
@@ -378,21 +405,37 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
       l_sum *= factor;
       // ---- P = exp2(s - m_ref) -> bf16 -> shared memory (K-major swizzled A operand of the PV MMA)
+#ifdef HSPEC_ATTN_TIMING
+      t_mark = clock64();
+#endif
       if (t >= 2 && !mbar_wait(smem_u32(&bars->pv_done[t & 1]), ((t >> 1) - 1) & 1)) { ok = false; break; }
-      uint8_t* pdst = sP + (t & 1) * TILE_BYTES;
+#ifdef HSPEC_ATTN_TIMING
+      t_wait_pv += clock64() - t_mark;
+#endif
+      const float neg_m = -m_ref;
+      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
-        float p[8];
+      for (int hh = 0; hh < 2; ++hh) {                 // 64 keys = 32 packed columns per TMEM store
+        uint32_t w[32];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) { p[e] = exp2f(s[ch * 8 + e] - m_ref); l_sum += p[e]; }
-        uint4 w;
-        w.x = pack_bf16(p[0], p[1]); w.y = pack_bf16(p[2], p[3]); w.z = pack_bf16(p[4], p[5]); w.w = pack_bf16(p[6], p[7]);
-        *reinterpret_cast<uint4*>(pdst + tile_off(r_local, ch)) = w;
+        for (int e = 0; e < 32; ++e) {
+          const float p0 = ex2_ftz(fmaf(s[hh * 64 + 2 * e], a.scale_log2, neg_m));
+          const float p1 = ex2_ftz(fmaf(s[hh * 64 + 2 * e + 1], a.scale_log2, neg_m));
+          ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
+          w[e] = pack_bf16(p0, p1);
+        }
+        tmem_st32(tmem_p0 + (t & 1) * 64 + lane_base + hh * 32, w);
       }
-      fence_proxy_async();
+      l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+      tmem_st_wait();
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->p_ready[t & 1]));
     }
+#ifdef HSPEC_ATTN_TIMING
+    if (tid == 0 && (blockIdx.x + blockIdx.y * 7 + blockIdx.z * 13) % 97 == 0)
+      printf("attn cta (%d,%d,%d): T=%d total=%lld wait_s=%lld wait_pv=%lld clocks\n", blockIdx.x, blockIdx.y, blockIdx.z, g.T,
+             clock64() - t_start, t_wait_s, t_wait_pv);
+#endif
     if (!ok) { atomicExch(a.status, STATUS_TIMEOUT_EPILOGUE); *abort_flag = 1; }
     // ---- partial (m, l, O) of this chunk
     if (ok && mbar_wait(smem_u32(&bars->o_done), 0) && !*abort_flag) {
@@ -497,7 +540,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   CUtensorMap tmK, tmV;
   if (!make_pool_tmap(&tmK, c.k_pool, c.num_pages, c.Hkv, err) || !make_pool_tmap(&tmV, c.v_pool, c.num_pages, c.Hkv, err))
     return cudaErrorInvalidValue;
-  const size_t smem = size_t(TILE_BYTES) * (1 + 2 + 2 * NS) + sizeof(AttnTcBars) + 1024;
+  const size_t smem = size_t(TILE_BYTES) * (1 + 2 * NS) + sizeof(AttnTcBars) + 1024;
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
