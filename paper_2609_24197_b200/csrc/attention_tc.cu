@@ -51,12 +51,18 @@ struct __align__(8) AttnTcBars {
   uint64_t s_ready[2], p_ready[2], pv_done[2];
   uint32_t tmem_base;
   uint32_t abort_flag;
+  int32_t pages[256];      // physical page ids of this chunk's full tiles (chunk <= 4096 tokens)
 };
 
 // byte offset of (row, 16-byte chunk 0..15) inside a [128 x 128] bf16 operand tile stored as two K-major halves
 // with the 128-byte swizzle (the layout TMA writes and the UMMA descriptors read)
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
   return uint32_t((chunk >> 3) * HALF_BYTES + (row >> 3) * 1024 + (row & 7) * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+}
+
+// adds to the barrier's expected byte count without arriving on it
+__device__ __forceinline__ void mbar_expect_tx_only(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int c0, int c1, int c2, int c3, uint32_t bar) {
@@ -209,6 +215,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (warp == 4) {
     // ================================================================= producer
     const int32_t* ptab = a.page_table + size_t(b) * a.page_table_stride;
+    // page ids of all full tiles up front: no dependent global load on the per-tile issue path
+    for (int i = lane; i < g.n_full * 8; i += 32) bars->pages[i] = ptab[(g.p_begin >> 4) + i];
+    __syncwarp();
     for (int t = 0; t < g.T; ++t) {
       const int s = t % NS;
       if (t >= NS && !mbar_wait(smem_u32(&bars->kv_empty[s]), ((t / NS) - 1) & 1)) {
@@ -219,57 +228,56 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       uint8_t* dK = sKV + s * 2 * TILE_BYTES;
       uint8_t* dV = dK + TILE_BYTES;
       if (t < g.n_full) {
-        const int page0 = (g.p_begin + t * KT) >> 4;
-        const int my_page = (lane < 8) ? ptab[page0 + lane] : 0;
         const uint32_t kf = smem_u32(&bars->k_full[s]), vf = smem_u32(&bars->v_full[s]);
         if (lane == 0) { mbar_expect_tx(kf, TILE_BYTES); mbar_expect_tx(vf, TILE_BYTES); }
         __syncwarp();
-#pragma unroll
-        for (int pi = 0; pi < 8; ++pi) {
-          const int page = __shfl_sync(0xffffffffu, my_page, pi);
-          if (lane == 0) {
-            tma_load_4d(smem_u32(dK) + pi * 2048, &tmK, 0, kvh, 0, page, kf);
-            tma_load_4d(smem_u32(dK) + HALF_BYTES + pi * 2048, &tmK, 64, kvh, 0, page, kf);
-          }
+        if (lane < 8) {                                   // one lane per page: K first (the score MMA needs it first)
+          const int page = bars->pages[t * 8 + lane];
+          tma_load_4d(smem_u32(dK) + lane * 2048, &tmK, 0, kvh, 0, page, kf);
+          tma_load_4d(smem_u32(dK) + HALF_BYTES + lane * 2048, &tmK, 64, kvh, 0, page, kf);
         }
-#pragma unroll
-        for (int pi = 0; pi < 8; ++pi) {
-          const int page = __shfl_sync(0xffffffffu, my_page, pi);
-          if (lane == 0) {
-            tma_load_4d(smem_u32(dV) + pi * 2048, &tmV, 0, kvh, 0, page, vf);
-            tma_load_4d(smem_u32(dV) + HALF_BYTES + pi * 2048, &tmV, 64, kvh, 0, page, vf);
-          }
+        __syncwarp();
+        if (lane < 8) {
+          const int page = bars->pages[t * 8 + lane];
+          tma_load_4d(smem_u32(dV) + lane * 2048, &tmV, 0, kvh, 0, page, vf);
+          tma_load_4d(smem_u32(dV) + HALF_BYTES + lane * 2048, &tmV, 64, kvh, 0, page, vf);
         }
       } else {
-        // ragged end of the prefix and / or the block's own keys: 16-byte loads, zero fill for unused rows
+        // ragged end of the prefix and / or the block's own keys.  Whole pages of the ragged end still come by
+        // TMA; the last partial page and the block rows come through cp.async (zero fill for every unused row,
+        // so nothing that is not a real key or value is ever multiplied).
         int n_prefix, prefix_start, n_block;
         manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
-        const int chunk16 = lane & 15;
-        for (int rb = 0; rb < KT; rb += 16) {                 // 8 rows per lane in flight
-          uint4 kv4[8], vv4[8];
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int r = rb + 2 * u + (lane >> 4);
-            kv4[u] = make_uint4(0, 0, 0, 0); vv4[u] = make_uint4(0, 0, 0, 0);
-            if (r < n_prefix) {
-              const int p = prefix_start + r;
-              const int page = ptab[p >> 4];
-              const size_t off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
-              kv4[u] = *reinterpret_cast<const uint4*>(a.k_pool + off);
-              vv4[u] = *reinterpret_cast<const uint4*>(a.v_pool + off);
-            } else if (r < n_prefix + n_block) {
-              const size_t off = ((size_t(b) * a.k + (r - n_prefix)) * a.Hkv + kvh) * DH + chunk16 * 8;
-              kv4[u] = *reinterpret_cast<const uint4*>(a.kb + off);
-              vv4[u] = *reinterpret_cast<const uint4*>(a.vb + off);
-            }
-          }
-#pragma unroll
-          for (int u = 0; u < 8; ++u) {
-            const int r = rb + 2 * u + (lane >> 4);
-            *reinterpret_cast<uint4*>(dK + tile_off(r, chunk16)) = kv4[u];
-            *reinterpret_cast<uint4*>(dV + tile_off(r, chunk16)) = vv4[u];
-          }
+        const int full_pages = n_prefix >> 4;
+        const int tma_rows = full_pages << 4;
+        const uint32_t kf = smem_u32(&bars->k_full[s]), vf = smem_u32(&bars->v_full[s]);
+        if (lane == 0 && full_pages > 0) { mbar_expect_tx_only(kf, full_pages * 4096); mbar_expect_tx_only(vf, full_pages * 4096); }
+        __syncwarp();
+        if (lane < full_pages) {
+          const int page = ptab[(prefix_start >> 4) + lane];
+          tma_load_4d(smem_u32(dK) + lane * 2048, &tmK, 0, kvh, 0, page, kf);
+          tma_load_4d(smem_u32(dK) + HALF_BYTES + lane * 2048, &tmK, 64, kvh, 0, page, kf);
+          tma_load_4d(smem_u32(dV) + lane * 2048, &tmV, 0, kvh, 0, page, vf);
+          tma_load_4d(smem_u32(dV) + HALF_BYTES + lane * 2048, &tmV, 64, kvh, 0, page, vf);
         }
+        for (int idx = lane; idx < (KT - tma_rows) * 16; idx += 32) {
+          const int r = tma_rows + (idx >> 4), chunk16 = idx & 15;
+          const bool valid = r < n_prefix + n_block;
+          size_t off = 0;
+          const __nv_bfloat16 *srcK = a.k_pool, *srcV = a.v_pool;
+          if (r < n_prefix) {
+            const int p = prefix_start + r;
+            const int page = ptab[p >> 4];
+            off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
+          } else if (valid) {
+            srcK = a.kb; srcV = a.vb;
+            off = ((size_t(b) * a.k + (r - n_prefix)) * a.Hkv + kvh) * DH + chunk16 * 8;
+          }
+          cp_async16(smem_u32(dK) + tile_off(r, chunk16), srcK + off, valid);
+          cp_async16(smem_u32(dV) + tile_off(r, chunk16), srcV + off, valid);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
         fence_proxy_async();
         __syncwarp();
         if (lane == 0) { mbar_arrive(smem_u32(&bars->k_full[s])); mbar_arrive(smem_u32(&bars->v_full[s])); }
@@ -280,9 +288,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     if (lane == 0) {
       const uint32_t id_qk = idesc_bf16_128x128(false), id_pv = idesc_bf16_128x128(true);
       bool ok = mbar_wait(smem_u32(&bars->q_ready), 0);
+#ifdef HSPEC_ATTN_TIMING
+      long long w_k = 0, w_p = 0, w_v = 0, m0;
+#endif
       auto issue_s = [&](int t) -> bool {
         const int s = t % NS;
+#ifdef HSPEC_ATTN_TIMING
+        m0 = clock64();
+#endif
         if (!mbar_wait(smem_u32(&bars->k_full[s]), (t / NS) & 1)) return false;
+#ifdef HSPEC_ATTN_TIMING
+        w_k += clock64() - m0;
+#endif
         tc_fence_after();
         const uint32_t kbase = smem_u32(sKV + s * 2 * TILE_BYTES);
         const uint32_t qbase = smem_u32(sQ);
@@ -300,8 +317,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (t + 1 < g.T) ok = issue_s(t + 1);
         if (!ok) break;
         const int s = t % NS;
-        if (!mbar_wait(smem_u32(&bars->p_ready[t & 1]), (t >> 1) & 1) ||
-            !mbar_wait(smem_u32(&bars->v_full[s]), (t / NS) & 1)) { ok = false; break; }
+#ifdef HSPEC_ATTN_TIMING
+        m0 = clock64();
+#endif
+        if (!mbar_wait(smem_u32(&bars->p_ready[t & 1]), (t >> 1) & 1)) { ok = false; break; }
+#ifdef HSPEC_ATTN_TIMING
+        w_p += clock64() - m0; m0 = clock64();
+#endif
+        if (!mbar_wait(smem_u32(&bars->v_full[s]), (t / NS) & 1)) { ok = false; break; }
+#ifdef HSPEC_ATTN_TIMING
+        w_v += clock64() - m0;
+#endif
         tc_fence_after();
         const uint32_t vbase = smem_u32(sKV + s * 2 * TILE_BYTES + TILE_BYTES);
 #pragma unroll
@@ -313,6 +339,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         umma_commit(smem_u32(&bars->kv_empty[s]));
         umma_commit(smem_u32(&bars->pv_done[t & 1]));
       }
+#ifdef HSPEC_ATTN_TIMING
+      if ((blockIdx.x + blockIdx.y * 7 + blockIdx.z * 13) % 97 == 0)
+        printf("  mma (%d,%d,%d): wait_k=%lld wait_p=%lld wait_v=%lld\n", blockIdx.x, blockIdx.y, blockIdx.z, w_k, w_p, w_v);
+#endif
       if (ok) umma_commit(smem_u32(&bars->o_done));
       else {
         atomicExch(a.status, STATUS_TIMEOUT_MMA);
