@@ -16,6 +16,8 @@
 
 #include <cuda.h>
 
+#include <cstdlib>
+
 namespace hspec {
 
 namespace {
@@ -35,7 +37,7 @@ struct __align__(8) GemmSmemTail {
   int red_idx[4][256];
 };
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g) {
   extern __shared__ uint8_t smem_raw[];
   // 128-byte swizzle needs 1024-byte aligned tiles
@@ -142,11 +144,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __uint_as_float(r[j]);
         }
       } else if (g.mode == EPI_ACCUM_F32) {
+        // read-modify-write of the residual stream: issue the 16 loads together, then add and store
         float* out = reinterpret_cast<float*>(g.out);
+        float old[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const int m = m0 + c0 + j;
-          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] += __uint_as_float(r[j]);
+          old[j] = (n_ok && m < g.M) ? __ldcg(out + size_t(m) * g.ldo + n) : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const int m = m0 + c0 + j;
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = old[j] + __uint_as_float(r[j]);
         }
       } else if (g.mode == EPI_STORE_BF16) {
         __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(g.out);
@@ -308,6 +317,7 @@ int gemm_pick_bn(int M) {
 }
 
 int gemm_pick_splits(int M, int n_out, int K, int num_sms) {
+  if (gemm2_preferred(M, n_out)) return 1;
   // Weight streaming (few rows): keep every SM fed.  Many rows: one slice (tensor-bound, no reduction pass).
   const int k_tiles = (K + TILE_K - 1) / TILE_K;
   const int tiles = ((n_out + TILE_W - 1) / TILE_W) * ((M + 255) / 256);
@@ -325,6 +335,7 @@ size_t gemm_splitk_bytes(int M, int n_out, int splits) {
 
 // Launches y = x W^T.  tmW must describe W with box rows 128; x is described here (box rows BN).
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
+  if (gemm2_preferred(c.M, c.n_out)) return gemm2_launch(c, stream, trk, err);
   if (g_smem_optin < 0) {
     int dev = 0;
     cudaGetDevice(&dev);
@@ -346,7 +357,10 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   g.tmem_cols = cols;
   const size_t stage_bytes = A_STAGE_BYTES + size_t(g.BN) * TILE_K * 2;
   const size_t fixed = sizeof(GemmSmemTail) + 1024;
-  int stages = int((size_t(g_smem_optin) - fixed) / stage_bytes);
+  // Weight streaming (narrow activation tile): size the ring so that TWO CTAs fit on an SM; one CTA's prologue and
+  // epilogue then overlap the other's stream.  Wide tiles take the whole SM.
+  const size_t budget = (g.BN <= 128) ? size_t(g_smem_optin) / 2 - 1024 : size_t(g_smem_optin);
+  int stages = int((budget - fixed) / stage_bytes);
   if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
   if (stages > g.k_tiles_per_split) stages = g.k_tiles_per_split < 2 ? 2 : g.k_tiles_per_split;
   if (stages < 2) { if (err) *err = "shared memory too small for the GEMM pipeline"; return cudaErrorInvalidValue; }

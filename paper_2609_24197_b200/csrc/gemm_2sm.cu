@@ -1,0 +1,365 @@
+// y = x W^T for many activation rows (M >= 256): the tensor-bound regime of the draft step.
+//
+// Two CTAs on two SMs form one MMA unit (tcgen05 cta_group::2): the pair owns a [256 weight rows x BNT
+// activation rows] tile of y^T.  Each CTA loads its own 128 weight rows and only HALF of the activation tile per
+// k-step (the MMA reads the B operand from both CTAs' shared memory), which halves the shared-memory fill per
+// flop compared with the one-CTA kernel; the accumulator lives in both CTAs' TMEM (128 lanes each).
+// The kernel is persistent: one cluster per SM pair walks a static list of tiles; two TMEM accumulators
+// alternate so the epilogue of one tile (tcgen05.ld -> global stores) overlaps the main loop of the next.
+//
+//   warp 0   TMA producer (both CTAs; both signal the LEADER CTA's "full" barrier)
+//   warp 1   TMEM allocation (both CTAs), MMA issue + commits (leader CTA only, one thread)
+//   warps 2..5  epilogue (both CTAs, their own 128 accumulator lanes)
+// No TMA load is multicast; the only cluster-wide signal is tcgen05.commit to both CTAs' barriers.
+#include "common.cuh"
+#include "kernels.h"
+
+#include <cstdlib>
+
+namespace hspec {
+
+namespace {
+
+constexpr int TILE_K = 64;
+constexpr uint32_t A_BYTES = 128 * TILE_K * 2;     // 16 KiB: this CTA's 128 weight rows
+
+struct Gemm2Args {
+  int M, N_out, K;
+  int BNT;                 // activation rows per cluster tile (128 or 256); each CTA stages BNT/2
+  int k_tiles, stages;
+  int n_tiles_w, n_tiles_m;
+  int f16, mode;
+  void* out;
+  long long ldo;
+  float* logits;
+  float* part_val;
+  int* part_idx;
+  uint32_t* status;
+};
+
+struct __align__(8) Tail2 {
+  uint64_t full[GEMM_MAX_STAGES];
+  uint64_t empty[GEMM_MAX_STAGES];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+  float red_val[4][256];
+  int red_idx[4][256];
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t mapa_rank(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_2sm(uint32_t smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_2sm() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_2sm(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// TMA load issued by either CTA of the pair; the byte count is credited to the barrier at the same offset in
+// the leader CTA (rank bit of the shared::cluster address cleared).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap, int c0, int c1, uint32_t bar_local,
+                                                 uint64_t policy) {
+  const uint32_t bar_leader = bar_local & 0xFEFFFFFFu;
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%2, %3}], [%4], %5;"
+      ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(bar_leader), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void umma_2sm(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives (once every MMA issued so far has finished) on the barrier at this offset in BOTH CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t idesc_m256(uint32_t n, bool f16) {
+  const uint32_t fmt = f16 ? 0u : 1u;
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n >> 3) << 17) | ((256u >> 4) << 24);
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, Gemm2Args g) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const uint32_t b_bytes = uint32_t(g.BNT / 2) * TILE_K * 2;
+  const uint32_t stage_bytes = A_BYTES + b_bytes;
+  Tail2* tail = reinterpret_cast<Tail2*>(smem + size_t(g.stages) * stage_bytes);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  const int total_tiles = g.n_tiles_w * g.n_tiles_m;
+  const uint32_t tmem_cols = 2u * uint32_t(g.BNT);           // two accumulators (256 or 512 columns)
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmA);
+    tma_prefetch_desc(&tmB);
+    for (int s = 0; s < g.stages; ++s) {
+      mbar_init(smem_u32(&tail->full[s]), 1);
+      mbar_init(smem_u32(&tail->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&tail->tmem_full[a]), 1);
+      mbar_init(smem_u32(&tail->tmem_empty[a]), 256);        // 128 epilogue threads of each CTA (leader's copy is used)
+    }
+    tail->abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_2sm(smem_u32(&tail->tmem_base), tmem_cols);
+    tmem_relinquish_2sm();
+  }
+  tc_fence_before();
+  cluster_sync_all();
+  tc_fence_after();
+  const uint32_t tmem_base = tail->tmem_base;
+  volatile uint32_t* abort_flag = &tail->abort_flag;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+        const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
+        for (int kt = 0; kt < g.k_tiles; ++kt, ++it) {
+          const int s = it % g.stages;
+          const uint32_t round = it / g.stages;
+          if (round > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (round - 1) & 1)) {
+            atomicExch(g.status, STATUS_TIMEOUT_PRODUCER);
+            *abort_flag = 1;
+            ok = false;
+            break;
+          }
+          const uint32_t full = smem_u32(&tail->full[s]);
+          if (rank == 0) mbar_expect_tx(full, 2 * stage_bytes);       // both CTAs' bytes land on the leader's barrier
+          uint8_t* sa = smem + size_t(s) * stage_bytes;
+          tma_load_2d_pair(smem_u32(sa), &tmA, kt * TILE_K, tn * 256 + int(rank) * 128, full, pol_w);
+          tma_load_2d_pair(smem_u32(sa + A_BYTES), &tmB, kt * TILE_K, tm * g.BNT + int(rank) * (g.BNT / 2), full, pol_x);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = idesc_m256(uint32_t(g.BNT), g.f16 != 0);
+      uint32_t it = 0, tile_count = 0;
+      bool ok = true;
+      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++tile_count) {
+        const uint32_t acc = tile_count & 1, use = tile_count >> 1;
+        if (use > 0 && !mbar_wait(smem_u32(&tail->tmem_empty[acc]), (use - 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT);
+        for (int kt = 0; kt < g.k_tiles; ++kt, ++it) {
+          const int s = it % g.stages;
+          const uint32_t round = it / g.stages;
+          if (!mbar_wait(smem_u32(&tail->full[s]), round & 1)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes);
+          const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < TILE_K / 16; ++kk)
+            umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+          umma_commit_pair(smem_u32(&tail->empty[s]));
+        }
+        if (ok) umma_commit_pair(smem_u32(&tail->tmem_full[acc]));
+      }
+      if (!ok) { atomicExch(g.status, STATUS_TIMEOUT_MMA); *abort_flag = 1; }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue (both CTAs)
+    const int q = warp & 3;
+    uint32_t tile_count = 0;
+    bool ok = true;
+    const uint32_t empty_leader0 = mapa_rank(smem_u32(&tail->tmem_empty[0]), 0);
+    const uint32_t empty_leader1 = mapa_rank(smem_u32(&tail->tmem_empty[1]), 0);
+    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++tile_count) {
+      const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
+      const uint32_t acc = tile_count & 1, use = tile_count >> 1;
+      if (!mbar_wait(smem_u32(&tail->tmem_full[acc]), use & 1)) {
+        atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
+        ok = false;
+        break;
+      }
+      tc_fence_after();
+      const int tile_n128 = tn * 2 + int(rank);               // 128-row weight tile of this CTA
+      const int n = tile_n128 * 128 + q * 32 + lane;
+      const bool n_ok = n < g.N_out;
+      const int m0 = tm * g.BNT;
+      const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT) + (uint32_t(q * 32) << 16);
+      for (int c0 = 0; c0 < g.BNT; c0 += 16) {
+        if (m0 + c0 >= g.M && g.mode != EPI_ARGMAX) break;    // rows past M: nothing to store
+        uint32_t r[16];
+        tmem_ld16(tmem_acc + uint32_t(c0), r);
+        tmem_ld_wait();
+        if (g.mode == EPI_STORE_F32) {
+          float* out = reinterpret_cast<float*>(g.out);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __uint_as_float(r[j]);
+          }
+        } else if (g.mode == EPI_ACCUM_F32) {
+          // read-modify-write of the residual stream: issue the 16 loads together, then add and store
+          float* out = reinterpret_cast<float*>(g.out);
+          float old[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            old[j] = (n_ok && m < g.M) ? __ldcg(out + size_t(m) * g.ldo + n) : 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = old[j] + __uint_as_float(r[j]);
+          }
+        } else if (g.mode == EPI_STORE_F16) {
+          __half* out = reinterpret_cast<__half*>(g.out);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2half_rn(__uint_as_float(r[j]));
+          }
+        } else if (g.mode == EPI_STORE_BF16) {
+          __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(g.out);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
+          }
+        } else {  // EPI_ARGMAX
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            float v = n_ok ? __uint_as_float(r[j]) : -INFINITY;
+            if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v;
+            int idx = n;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+              const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+              const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+              if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+            }
+            if (lane == 0) { tail->red_val[q][c0 + j] = v; tail->red_idx[q][c0 + j] = idx; }
+          }
+        }
+      }
+      // accumulator drained: hand it back to the MMA issuer in the leader CTA
+      tc_fence_before();
+      mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
+      if (g.mode == EPI_ARGMAX) {
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const int t = threadIdx.x - 64;
+        for (int c = t; c < g.BNT; c += 128) {
+          const int m = m0 + c;
+          if (m >= g.M || tile_n128 * 128 >= g.N_out) continue;   // the pair's second half may lie wholly past V
+          float v = tail->red_val[0][c];
+          int idx = tail->red_idx[0][c];
+#pragma unroll
+          for (int qq = 1; qq < 4; ++qq) {
+            const float ov = tail->red_val[qq][c];
+            const int oi = tail->red_idx[qq][c];
+            if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+          }
+          g.part_val[size_t(tile_n128) * g.M + m] = v;
+          g.part_idx[size_t(tile_n128) * g.M + m] = idx;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");        // red_* is reused by the next tile
+      }
+    }
+  }
+  tc_fence_before();
+  cluster_sync_all();           // neither CTA may leave while its pair still reads its shared memory or TMEM
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_2sm(tmem_base, tmem_cols);
+  }
+}
+
+int g_smem_optin2 = -1;
+
+}  // namespace
+
+bool gemm2_preferred(int M, int n_out) {
+  static const bool off = [] { const char* e = getenv("HSPEC_GEMM_1SM"); return e && e[0] == '1'; }();
+  if (off || M < 256) return false;
+  const int bnt = gemm2_pick_bnt(M, n_out);
+  return ((n_out + 255) / 256) * ((M + bnt - 1) / bnt) >= 74;
+}
+
+// Tile width (activation rows per cluster tile) that wastes the fewest cluster rounds.
+int gemm2_pick_bnt(int M, int n_out) {
+  const int tw = (n_out + 255) / 256;
+  double best_cost = 1e30;
+  int best = 256;
+  for (int bnt : {256, 128}) {
+    const int tiles = tw * ((M + bnt - 1) / bnt);
+    const int rounds = (tiles + 73) / 74;
+    // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
+    // measured, the narrow tile runs ~1.5x slower per flop
+    const double cost = double(rounds) * bnt * (bnt == 128 ? 1.5 : 1.0);
+    if (cost < best_cost) { best_cost = cost; best = bnt; }
+  }
+  return best;
+}
+
+cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
+  if (g_smem_optin2 < 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_smem_optin2, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cudaError_t e = cudaFuncSetAttribute(gemm_2sm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin2);
+    if (e != cudaSuccess) return e;
+  }
+  Gemm2Args g{};
+  g.M = c.M; g.N_out = c.n_out; g.K = c.K;
+  g.BNT = gemm2_pick_bnt(c.M, c.n_out);
+  g.k_tiles = (c.K + TILE_K - 1) / TILE_K;
+  g.n_tiles_w = (c.n_out + 255) / 256;
+  g.n_tiles_m = (c.M + g.BNT - 1) / g.BNT;
+  g.f16 = c.f16 ? 1 : 0; g.mode = c.mode; g.out = c.out; g.ldo = c.ldo;
+  g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
+  const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
+  const size_t fixed = sizeof(Tail2) + 1024;
+  int stages = int((size_t(g_smem_optin2) - fixed) / stage_bytes);
+  if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
+  if (stages < 2) { if (err) *err = "shared memory too small for the 2-SM GEMM pipeline"; return cudaErrorInvalidValue; }
+  g.stages = stages;
+  CUtensorMap tmB;
+  if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BNT / 2, c.f16, err)) return cudaErrorInvalidValue;
+  const int total = g.n_tiles_w * g.n_tiles_m;
+  const int clusters = total < 74 ? total : 74;
+  const size_t smem = size_t(stages) * stage_bytes + fixed;
+  trk_begin(trk, c.label ? c.label : "gemm", 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
+  gemm_2sm_kernel<<<2 * clusters, 192, smem, stream>>>(*c.tmW, tmB, g);
+  trk_end(trk);
+  return cudaGetLastError();
+}
+
+}  // namespace hspec

@@ -82,6 +82,9 @@ int gemm_pick_bn(int M);
 int gemm_pick_splits(int M, int n_out, int K, int num_sms);
 size_t gemm_splitk_bytes(int M, int n_out, int splits);
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
+bool gemm2_preferred(int M, int n_out);        // many rows and at least one full round of cluster tiles
+int gemm2_pick_bnt(int M, int n_out);
+cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk);
 

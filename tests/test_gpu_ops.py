@@ -44,6 +44,8 @@ def test_gather_kv_bit_exact(hs, ctx):
 GEMM_CASES = [
     (1, 256, 64), (8, 1064, 256), (16, 1024, 256), (48, 300, 16), (5, 128, 4096), (200, 384, 4096),
     (256, 640, 128), (257, 130, 1024), (513, 256, 320), (33, 17536 // 8, 520),
+    # many rows and enough tiles for the 2-SM persistent kernel (ragged in every dimension)
+    (2048, 5120, 512), (600, 19000, 192), (300, 40000, 72), (2048, 2500, 4096),
 ]
 
 
@@ -88,7 +90,7 @@ def test_gemm_strided_output_and_exact_small_integers(hs):
     assert (big[:, n_out:] == -1.0).all()
 
 
-@pytest.mark.parametrize("M,V,K", [(8, 1024, 256), (40, 1000, 256), (300, 2500, 128)])
+@pytest.mark.parametrize("M,V,K", [(8, 1024, 256), (40, 1000, 256), (300, 2500, 128), (700, 30001, 64), (2048, 20000, 128)])
 def test_lm_head_argmax(hs, M, V, K):
     x = _randn((M, K), 7, 1.0, torch.float16)
     W = _randn((V, K), 8, 0.05, torch.float16)
