@@ -198,11 +198,14 @@ int hspec_op_rmsnorm(const float* x, const float* w, void* y_f16, int32_t M, int
  * k rows started from s_init, the D skip, and the SiLU(z) gate.
  *   zxbcdt fp32 [B*k, ld_in]: columns z [Di] | xBC [Di + 2GN] (| dt [H] when dt_raw is NULL)
  *   dt_raw fp32 [B*k, H] or NULL;  s_init fp16 [B, H, P, N] or NULL (zero state)
- *   y_gated fp32 [B*k, Di] = (scan output) * SiLU(z). */
+ *   y_gated fp32 [B*k, Di] = (scan output) * SiLU(z).
+ *   workspace: optional device scratch of hspec_scan_workspace_bytes(...) bytes (256-byte aligned); with it the serving
+ *   shapes (P = 64, N = 128) run as three kernels (conv, C.B table, state stream), without it as one fused kernel. */
 int hspec_op_mamba_scan(const float* zxbcdt, int64_t ld_in, const float* dt_raw, const void* s_init,
                         const float* conv_w, const float* conv_b, const float* dt_bias, const float* A_log,
                         const float* Dskip, float* y_gated, int32_t B, int32_t k, int32_t Di, int32_t P,
-                        int32_t N, int32_t G, int32_t d_conv, void* stream);
+                        int32_t N, int32_t G, int32_t d_conv, void* workspace, size_t workspace_bytes, void* stream);
+size_t hspec_scan_workspace_bytes(int32_t B, int32_t k, int32_t Di, int32_t N, int32_t G);
 /* Per-head RMSNorm (optional) + rotate-half RoPE at positions ctx_lens[b] + i (Sec. 3.3.2, positional alignment).
  * qkv fp32 [B*k, (Hq+2Hkv)*dh] (q | k | v) -> q bf16 [B*k, Hq, dh], kb bf16 [B*k, Hkv, dh], vb bf16 [B*k, Hkv, dh]. */
 int hspec_op_qk_norm_rope(const float* qkv, const float* q_norm_w, const float* k_norm_w, const int32_t* ctx_lens,

@@ -19,7 +19,7 @@ _DT = {torch.bfloat16: 0, torch.float32: 1, torch.int32: 2, torch.float16: 3}
 EXPORTS = [
     "hspec_init", "hspec_workspace_bytes", "hspec_load_weights", "hspec_draft_block", "hspec_destroy",
     "hspec_last_error", "hspec_get_stats", "hspec_set_profiling", "hspec_get_profile", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
-    "hspec_op_lm_head_argmax", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_op_qk_norm_rope",
+    "hspec_op_lm_head_argmax", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
 ]
 
@@ -96,7 +96,9 @@ def load_library(path=None):
     lib.hspec_gemm_workspace_bytes.restype = sz
     lib.hspec_op_lm_head_argmax.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp, sz, vp]
     lib.hspec_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, f32, vp]
-    lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
+    lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
+    lib.hspec_scan_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
+    lib.hspec_scan_workspace_bytes.restype = sz
     lib.hspec_op_qk_norm_rope.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, f32, f32, i32, vp]
     lib.hspec_op_attention.argtypes = [vp, vp, vp, vp, vp, i64, vp, i32, vp, i32, vp, i32, i32, i32, i32, i32, i32, i32,
                                        i32, vp, sz, vp]
@@ -255,13 +257,18 @@ def hspec_op_rmsnorm(x, w, y, eps):
                                            x.shape[0], x.shape[1], float(eps), _stream()), None, "hspec_op_rmsnorm")
 
 
+def hspec_scan_workspace_bytes(B, k, Di, N, G):
+    return int(load_library().hspec_scan_workspace_bytes(B, k, Di, N, G))
+
+
 def hspec_op_mamba_scan(zxbcdt, dt_raw, s_init, conv_w, conv_b, dt_bias, A_log, Dskip, y_gated, B, k, Di, P, N, G,
-                        d_conv):
+                        d_conv, workspace=None):
     _check(load_library().hspec_op_mamba_scan(
         _ptr(zxbcdt, torch.float32), zxbcdt.stride(0), _ptr(dt_raw, torch.float32), _ptr(s_init, torch.float16),
         _ptr(conv_w, torch.float32), _ptr(conv_b, torch.float32), _ptr(dt_bias, torch.float32),
         _ptr(A_log, torch.float32), _ptr(Dskip, torch.float32), _ptr(y_gated, torch.float32),
-        B, k, Di, P, N, G, d_conv, _stream()), None, "hspec_op_mamba_scan")
+        B, k, Di, P, N, G, d_conv, _ptr(workspace), workspace.numel() * workspace.element_size() if workspace is not None else 0,
+        _stream()), None, "hspec_op_mamba_scan")
 
 
 def hspec_op_qk_norm_rope(qkv, q_norm_w, k_norm_w, ctx_lens, q, kb, vb, B, k, Hq, Hkv, dh, theta, eps, qk_norm=1):

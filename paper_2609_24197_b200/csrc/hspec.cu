@@ -49,7 +49,7 @@ int imax(int a, int b) { return a > b ? a : b; }
 
 // Offsets of the step's scratch buffers inside the caller's workspace.
 struct Plan {
-  size_t X, U, BIG, LH, Fv, SINIT, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
+  size_t X, U, BIG, LH, Fv, SINIT, SCAN, scan_bytes, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
   size_t att_bytes, splitk_bytes;
   int attn_chunk, max_ctx;
 };
@@ -73,6 +73,8 @@ Plan make_plan(const hspec_config& c, int B, int k, int max_ctx) {
   p.DTL = take(M * size_t(imax(c.dt_rank, 8)) * 2);
   p.DT = take(M * size_t(d.H) * 4);
   p.YG = take(M * size_t(c.Di) * 4);
+  p.scan_bytes = scan_workspace_bytes(B, k, c.Di, c.N, c.G);
+  p.SCAN = take(p.scan_bytes);
   p.Q = take(M * size_t(c.Hq) * c.dh * 2);
   p.KB = take(M * size_t(c.Hkv) * c.dh * 2);
   p.VB = take(M * size_t(c.Hkv) * c.dh * 2);
@@ -463,6 +465,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     sc.conv_w = fptr(pre + "mamba.conv_w"); sc.conv_b = fptr(pre + "mamba.conv_b");
     sc.dt_bias = fptr(pre + "mamba.dt_bias"); sc.A_log = fptr(pre + "mamba.A_log"); sc.Dskip = fptr(pre + "mamba.Dskip");
     sc.y_gated = YG; sc.B = B; sc.k = k; sc.Di = c.Di; sc.P = c.P; sc.N = c.N; sc.G = c.G; sc.d_conv = c.d_conv;
+    sc.ws = ws + p.SCAN; sc.ws_bytes = p.scan_bytes;
     CUDA_TRY(h, scan_launch(sc, st, trk, &errtxt));
     EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st));
     CUDA_TRY(h, gemm(pre + "mamba.out_proj", "gemm:out_proj", U, M, EPI_ACCUM_F32, X, c.D));
@@ -596,7 +599,8 @@ int hspec_op_rmsnorm(const float* x, const float* w, void* y, int32_t M, int32_t
 
 int hspec_op_mamba_scan(const float* zxbcdt, int64_t ld_in, const float* dt_raw, const void* s_init, const float* conv_w,
                         const float* conv_b, const float* dt_bias, const float* A_log, const float* Dskip, float* y_gated,
-                        int32_t B, int32_t k, int32_t Di, int32_t P, int32_t N, int32_t G, int32_t d_conv, void* stream) {
+                        int32_t B, int32_t k, int32_t Di, int32_t P, int32_t N, int32_t G, int32_t d_conv, void* workspace,
+                        size_t workspace_bytes, void* stream) {
   if (!zxbcdt || !conv_w || !conv_b || !dt_bias || !A_log || !Dskip || !y_gated || B < 1 || P < 1 || P > 128 || N < 1 ||
       N > 256 || d_conv < 1 || d_conv > 4)
     return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_mamba_scan: bad argument");
@@ -605,8 +609,13 @@ int hspec_op_mamba_scan(const float* zxbcdt, int64_t ld_in, const float* dt_raw,
   sc.zxbcdt = zxbcdt; sc.ld_in = ld_in; sc.dt_raw = dt_raw; sc.s_init = s_init; sc.conv_w = conv_w; sc.conv_b = conv_b;
   sc.dt_bias = dt_bias; sc.A_log = A_log; sc.Dskip = Dskip; sc.y_gated = y_gated;
   sc.B = B; sc.k = k; sc.Di = Di; sc.P = P; sc.N = N; sc.G = G; sc.d_conv = d_conv;
+  sc.ws = workspace; sc.ws_bytes = workspace_bytes;
   OP_TRY(scan_launch(sc, reinterpret_cast<cudaStream_t>(stream), nullptr, &errtxt));
   return HSPEC_OK;
+}
+
+size_t hspec_scan_workspace_bytes(int32_t B, int32_t k, int32_t Di, int32_t N, int32_t G) {
+  return scan_workspace_bytes(B, k, Di, N, G);
 }
 
 int hspec_op_qk_norm_rope(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q, void* kb,

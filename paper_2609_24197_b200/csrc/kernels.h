@@ -120,7 +120,10 @@ struct ScanCall {
   const float *conv_w, *conv_b, *dt_bias, *A_log, *Dskip;
   float* y_gated;                   // [B*k, Di]
   int B, k, Di, P, N, G, d_conv;
+  void* ws;                         // optional scratch (scan_workspace_bytes): enables the three-kernel fast path
+  size_t ws_bytes;
 };
+size_t scan_workspace_bytes(int B, int k, int Di, int N, int G);
 cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 
 // ---- element-wise kernels (elementwise.cu)

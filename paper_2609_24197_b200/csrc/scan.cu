@@ -318,6 +318,198 @@ mamba_scan_mma_kernel(ScanArgs a) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Three-kernel form of the fast path (used when the caller provides scratch): the small per-position
+// operands are prepared once per request and group, so the kernel that streams S_init has no
+// block-wide phases in front of its loads.
+//   scan_conv_kernel   causal depthwise conv + SiLU of every xBC channel (thread = channel, taps in registers);
+//                      C is also written as fp16 head + fp16 remainder for the tensor-core contraction
+//   scan_cb_kernel     CB[b, g, t, s] = C_t . B_s for s <= t
+//   mamba_scan_stream_kernel  one warp per head: everything it needs is fetched up front (cp.async for the
+//                      shared operands, 16-byte loads of S_init straight into the MMA fragments)
+__global__ void scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* __restrict__ c16) {
+  const int ch = blockIdx.x * blockDim.x + threadIdx.x;
+  const int b = blockIdx.y;
+  if (ch >= a.d_xBC) return;
+  float w[4] = {0.f, 0.f, 0.f, 0.f};
+  for (int j = 0; j < a.d_conv; ++j) w[4 - a.d_conv + j] = a.conv_w[ch * a.d_conv + j];   // right-aligned taps
+  const float bias = a.conv_b[ch];
+  float h0 = 0.f, h1 = 0.f, h2 = 0.f;                        // the three rows before the current one (zero left context)
+  const size_t row0 = size_t(b) * a.k;
+  const int GN = a.G * a.N;
+  const int c_col = ch - a.Di - GN;                          // >= 0 for C channels
+  for (int i = 0; i < a.k; ++i) {
+    const float cur = a.zxbcdt[(row0 + i) * a.ld_in + a.Di + ch];
+    const float v = silu_f(bias + w[0] * h0 + w[1] * h1 + w[2] * h2 + w[3] * cur);
+    h0 = h1; h1 = h2; h2 = cur;
+    xact[(row0 + i) * a.d_xBC + ch] = v;
+    if (c_col >= 0) {
+      const __half hi = __float2half_rn(v);
+      c16[((row0 + i) * 2 + 0) * GN + c_col] = hi;
+      c16[((row0 + i) * 2 + 1) * GN + c_col] = __float2half_rn(v - __half2float(hi));
+    }
+  }
+}
+
+__global__ void scan_cb_kernel(ScanArgs a, const float* __restrict__ xact, float* __restrict__ cb) {
+  const int g = blockIdx.x, b = blockIdx.y;
+  const int k = a.k, N = a.N;
+  const size_t row0 = size_t(b) * k;
+  const int GN = a.G * N;
+  for (int idx = threadIdx.x; idx < k * k; idx += blockDim.x) {
+    const int t = idx / k, s2 = idx % k;
+    float dot = 0.f;
+    if (s2 <= t) {
+      const float* cr = xact + (row0 + t) * a.d_xBC + a.Di + GN + g * N;
+      const float* br = xact + (row0 + s2) * a.d_xBC + a.Di + g * N;
+      for (int n = 0; n < N; ++n) dot += cr[n] * br[n];
+    }
+    cb[((size_t(b) * a.G + g) * KMAX + t) * KMAX + s2] = dot;
+  }
+}
+
+template <int P, int N, int MT>
+__global__ void __launch_bounds__(128)
+mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __half* __restrict__ c16,
+                         const float* __restrict__ cb) {
+  constexpr int HPC = 4, NT = P / 8, KP = N / 32, ROWS = MT * 16;
+  extern __shared__ __align__(16) float sm[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int h0 = blockIdx.x * HPC, b = blockIdx.y;
+  const int hpg = a.H / a.G, g = h0 / hpg, k = a.k, GN = a.G * N;
+  const int h = h0 + warp;
+  const size_t row0 = size_t(b) * k;
+  __half* C16 = reinterpret_cast<__half*>(sm);                 // [ROWS][2][N]  (hi, lo), rows >= k zero
+  float* CB = sm + ROWS * N;                                   // [ROWS][ROWS]
+  float* xs = CB + ROWS * ROWS + warp * (ROWS * P);            // per warp [ROWS][P]
+  float* Wh = CB + ROWS * ROWS + HPC * ROWS * P + warp * ROWS * (ROWS + 1);   // per warp [ROWS][ROWS+1]
+
+  // ---- state fragments of the first two k-step pairs: issued before anything else
+  const int gq = lane >> 2, tq = lane & 3;
+  const __half* S = a.s_init ? a.s_init + (size_t(b) * a.H + h) * P * N : nullptr;
+  uint4 sv0[NT], sv1[NT];
+  if (S != nullptr) {
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      sv0[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + 0 * 32 + tq * 8));
+      sv1[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + 1 * 32 + tq * 8));
+    }
+  }
+  // ---- shared operands (C halves, CB) and this head's x rows: cp.async, zero fill for the padding rows
+  for (int idx = tid; idx < ROWS * 2 * N / 8; idx += 128) {
+    const int r = idx / (2 * N / 8), rest = idx % (2 * N / 8), half = rest / (N / 8), c8 = rest % (N / 8);
+    cp_async16(smem_u32(C16 + (r * 2 + half) * N + c8 * 8), c16 + ((row0 + min(r, k - 1)) * 2 + half) * GN + g * N + c8 * 8, r < k);
+  }
+  for (int idx = tid; idx < ROWS * ROWS / 4; idx += 128) {
+    const int r = idx / (ROWS / 4), c4 = idx % (ROWS / 4);
+    cp_async16(smem_u32(CB + r * ROWS + c4 * 4), cb + ((size_t(b) * a.G + g) * KMAX + r) * KMAX + c4 * 4, true);
+  }
+  for (int idx = lane; idx < ROWS * P / 4; idx += 32) {
+    const int r = idx / (P / 4), c4 = idx % (P / 4);
+    cp_async16(smem_u32(xs + r * P + c4 * 4), xact + (row0 + min(r, k - 1)) * a.d_xBC + h * P + c4 * 4, r < k);
+  }
+  cp_async_commit();
+  // ---- dt, inclusive prefix sum of dt * A over the block positions (one warp shuffle scan per head)
+  float dt = 0.f, dA = 0.f;
+  if (lane < k) {
+    const float raw = a.dt_raw ? a.dt_raw[(row0 + lane) * a.H + h] : a.zxbcdt[(row0 + lane) * a.ld_in + a.Di + a.d_xBC + h];
+    dt = softplus_f(raw + a.dt_bias[h]);
+    dA = dt * (-expf(a.A_log[h]));
+  }
+  float cum = dA;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const float up = __shfl_up_sync(0xffffffffu, cum, off);
+    if (lane >= off) cum += up;
+  }
+  cp_async_wait<0>();
+  __syncthreads();
+  // ---- W[t][s] = exp(c_t - c_s) dt_s CB[t][s]: lane s owns column s
+  for (int t = 0; t < k; ++t) {
+    const float ct = __shfl_sync(0xffffffffu, cum, t);
+    float w = 0.f;
+    if (lane <= t) w = expf(ct - cum) * dt * CB[t * ROWS + lane];
+    if (lane < ROWS) Wh[t * (ROWS + 1) + lane] = w;
+  }
+  __syncwarp();
+  // ---- state term on the tensor cores
+  float acc[MT][NT][4];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+    for (int j = 0; j < NT; ++j) { acc[mt][j][0] = acc[mt][j][1] = acc[mt][j][2] = acc[mt][j][3] = 0.f; }
+  if (S != nullptr) {
+#pragma unroll
+    for (int kp = 0; kp < KP; ++kp) {
+      uint4 sv[NT];
+      if (kp >= 2) {
+#pragma unroll
+        for (int j = 0; j < NT; ++j) sv[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + kp * 32 + tq * 8));
+      } else {
+#pragma unroll
+        for (int j = 0; j < NT; ++j) sv[j] = kp == 0 ? sv0[j] : sv1[j];
+      }
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        const __half* c0 = C16 + ((mt * 16 + gq) * 2) * N + kp * 32 + tq * 8;
+        const __half* c1 = C16 + ((mt * 16 + gq + 8) * 2) * N + kp * 32 + tq * 8;
+        const uint4 c_lo = *reinterpret_cast<const uint4*>(c0), c_hi = *reinterpret_cast<const uint4*>(c1);
+        const uint4 r_lo = *reinterpret_cast<const uint4*>(c0 + N), r_hi = *reinterpret_cast<const uint4*>(c1 + N);
+        const uint32_t a0[4] = {c_lo.x, c_hi.x, c_lo.y, c_hi.y}, a1[4] = {c_lo.z, c_hi.z, c_lo.w, c_hi.w};
+        const uint32_t e0[4] = {r_lo.x, r_hi.x, r_lo.y, r_hi.y}, e1[4] = {r_lo.z, r_hi.z, r_lo.w, r_hi.w};
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          mma_f16_16816(acc[mt][j], a0, sv[j].x, sv[j].y);
+          mma_f16_16816(acc[mt][j], a1, sv[j].z, sv[j].w);
+          mma_f16_16816(acc[mt][j], e0, sv[j].x, sv[j].y);
+          mma_f16_16816(acc[mt][j], e1, sv[j].z, sv[j].w);
+        }
+      }
+    }
+  }
+  // ---- epilogue: decay, intra-block term, D skip, gate
+  const float Dh = a.Dskip[h];
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int t = mt * 16 + gq + half * 8;
+      const float dec = expf(__shfl_sync(0xffffffffu, cum, t & 31));
+      if (t >= k) continue;
+      const size_t row = row0 + t;
+      float2 z[NT];
+#pragma unroll
+      for (int j = 0; j < NT; ++j) z[j] = *reinterpret_cast<const float2*>(a.zxbcdt + row * a.ld_in + h * P + j * 8 + tq * 2);
+      float y[NT][2];
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        const float2 xv = *reinterpret_cast<const float2*>(xs + t * P + j * 8 + tq * 2);
+        y[j][0] = dec * acc[mt][j][half * 2] + Dh * xv.x;
+        y[j][1] = dec * acc[mt][j][half * 2 + 1] + Dh * xv.y;
+      }
+      for (int s2 = 0; s2 <= t; ++s2) {
+        const float w = Wh[t * (ROWS + 1) + s2];
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          const float2 xv = *reinterpret_cast<const float2*>(xs + s2 * P + j * 8 + tq * 2);
+          y[j][0] += w * xv.x;
+          y[j][1] += w * xv.y;
+        }
+      }
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+        *reinterpret_cast<float2*>(a.y + row * a.Di + h * P + j * 8 + tq * 2) =
+            make_float2(y[j][0] * silu_f(z[j].x), y[j][1] * silu_f(z[j].y));
+    }
+  }
+}
+
+template <int MT>
+size_t scan_stream_smem() {
+  constexpr int P = 64, N = 128, HPC = 4, ROWS = MT * 16;
+  return sizeof(__half) * ROWS * 2 * N + sizeof(float) * (ROWS * ROWS + HPC * ROWS * P + HPC * ROWS * (ROWS + 1));
+}
+
 template <int MT>
 size_t scan_mma_smem() {
   constexpr int P = 64, N = 128, HPC = 4, ROWS = MT * 16;
@@ -326,6 +518,11 @@ size_t scan_mma_smem() {
 }
 
 }  // namespace
+
+size_t scan_workspace_bytes(int B, int k, int Di, int N, int G) {
+  const size_t M = size_t(B) * k, d_xBC = size_t(Di) + 2 * size_t(G) * N;
+  return M * d_xBC * 4 + size_t(B) * G * KMAX * KMAX * 4 + M * 2 * size_t(G) * N * 2 + 256;
+}
 
 cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (c.k < 1 || c.k > KMAX) { if (err) *err = "scan: k out of range"; return cudaErrorInvalidValue; }
@@ -338,6 +535,35 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
   a.NP = c.N + 1;                                    // odd pitch: threads of a warp own consecutive p
   if (a.H % c.G) { if (err) *err = "scan: heads must divide into groups"; return cudaErrorInvalidValue; }
   // serving shapes: tensor-core path (needs 8-byte aligned rows for the float2 accesses)
+  if (c.P == 64 && c.N == 128 && (a.H / c.G) % 4 == 0 && c.ld_in % 2 == 0 && c.Di % 4 == 0 && c.ws != nullptr &&
+      c.ws_bytes >= scan_workspace_bytes(c.B, c.k, c.Di, c.N, c.G)) {
+    const bool two = c.k > 16;
+    const size_t M = size_t(c.B) * c.k;
+    float* xact = reinterpret_cast<float*>(c.ws);
+    float* cbw = xact + M * a.d_xBC;
+    __half* c16 = reinterpret_cast<__half*>(cbw + size_t(c.B) * c.G * KMAX * KMAX);
+    trk_begin(trk, "scan_conv", 0, double(M) * a.d_xBC * 8);
+    scan_conv_kernel<<<dim3((a.d_xBC + 255) / 256, c.B), 256, 0, stream>>>(a, xact, c16);
+    trk_end(trk);
+    trk_begin(trk, "scan_cb", 0, 0);
+    scan_cb_kernel<<<dim3(c.G, c.B), 256, 0, stream>>>(a, xact, cbw);
+    trk_end(trk);
+    const size_t smem_s = two ? scan_stream_smem<2>() : scan_stream_smem<1>();
+    static bool sset1 = false, sset2 = false;
+    bool& was = two ? sset2 : sset1;
+    if (!was) {
+      cudaError_t e = two ? cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s))
+                          : cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s));
+      if (e != cudaSuccess) return e;
+      was = true;
+    }
+    dim3 grid_s(a.H / 4, c.B);
+    trk_begin(trk, "mamba_scan", 2.0 * c.B * c.k * a.H * c.P * c.N, double(c.B) * a.H * c.P * c.N * 2);
+    if (two) mamba_scan_stream_kernel<64, 128, 2><<<grid_s, 128, smem_s, stream>>>(a, xact, c16, cbw);
+    else mamba_scan_stream_kernel<64, 128, 1><<<grid_s, 128, smem_s, stream>>>(a, xact, c16, cbw);
+    trk_end(trk);
+    return cudaGetLastError();
+  }
   if (c.P == 64 && c.N == 128 && (a.H / c.G) % 4 == 0 && c.ld_in % 2 == 0 && c.Di % 2 == 0) {
     const bool two = c.k > 16;
     const size_t smem_f = two ? scan_mma_smem<2>() : scan_mma_smem<1>();

@@ -62,8 +62,9 @@ def scan(reps):
     cw, cb = _randn((Di + 2 * G * N, 4), 8, 0.3, torch.float32), _randn((Di + 2 * G * N,), 9, 0.02, torch.float32)
     dtb, Al, Ds = _randn((H,), 10, 1.0, torch.float32) - 4, torch.rand(H, device="cuda") * 2, torch.ones(H, device="cuda")
     y = torch.empty((B * k, Di), dtype=torch.float32, device="cuda")
+    ws = torch.empty(hs.hspec_scan_workspace_bytes(B, k, Di, N, G), dtype=torch.uint8, device="cuda")
     for _ in range(reps):
-        hs.hspec_op_mamba_scan(zx, None, s0, cw, cb, dtb, Al, Ds, y, B, k, Di, P, N, G, 4)
+        hs.hspec_op_mamba_scan(zx, None, s0, cw, cb, dtb, Al, Ds, y, B, k, Di, P, N, G, 4, ws)
     torch.cuda.synchronize()
     print(f"scan: B={B} H={H} S_init bytes per launch={B * H * P * N * 2}")
 

@@ -164,8 +164,10 @@ def test_qk_norm_rope(hs, dh, Hq, Hkv, theta, qk_norm):
 @pytest.mark.parametrize("B,k,Di,P,N,G,dtr,zero_state", [
     (2, 8, 512, 64, 16, 1, True, False), (3, 5, 256, 64, 128, 2, False, False), (1, 16, 8192, 64, 128, 4, False, False),
     (2, 1, 128, 64, 128, 1, False, False), (2, 32, 192, 64, 4, 1, False, False), (2, 7, 128, 32, 24, 2, False, True),
+    (2, 32, 512, 64, 128, 2, False, False), (3, 11, 1024, 64, 128, 4, True, True),
 ])
-def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state):
+@pytest.mark.parametrize("with_scratch", [False, True])
+def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state, with_scratch):
     H, d_conv = Di // P, 4
     d_xBC = Di + 2 * G * N
     ld = Di + d_xBC + (0 if dtr else H)
@@ -178,7 +180,8 @@ def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state):
     dt_bias = _randn((H,), 37, 1.0) - 4.0
     Dskip = 1 + _randn((H,), 38, 0.1)
     y = torch.full((B * k, Di), float("nan"), dtype=torch.float32, device="cuda")
-    hs.hspec_op_mamba_scan(zx, dt_raw, s_init, conv_w, conv_b, dt_bias, A_log, Dskip, y, B, k, Di, P, N, G, d_conv)
+    ws = torch.empty(hs.hspec_scan_workspace_bytes(B, k, Di, N, G), dtype=torch.uint8, device="cuda") if with_scratch else None
+    hs.hspec_op_mamba_scan(zx, dt_raw, s_init, conv_w, conv_b, dt_bias, A_log, Dskip, y, B, k, Di, P, N, G, d_conv, ws)
     torch.cuda.synchronize()
     f64 = lambda t: t.cpu().numpy().astype(np.float64)
     zxn = f64(zx)
