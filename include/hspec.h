@@ -191,6 +191,18 @@ size_t hspec_gemm_workspace_bytes(int32_t M, int32_t n_out, int32_t K);
  * x and W are both bf16 or both fp16 (in_dtype). */
 int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M, int32_t V,
                             int32_t K, void* workspace, size_t workspace_bytes, void* stream);
+/* The same LM head + arg-max for callers that cannot allocate device memory at the point where they draft: an engine
+ * whose KV-cache pool already owns every free byte of HBM (a later cudaMalloc fails), a decode loop that cannot take the
+ * device synchronisation and driver lock of an allocation, a plug-in that is handed pointers but no allocator.  (The
+ * paper has no counterpart; this is a deployment aid.)  The per-tile (max, index) partials and the status word live in
+ * a fixed array inside the library's device image: 8 MiB + 256 B on every GPU that loads the library, held until the
+ * process exits.  Limits: M <= 512 rows, V <= 262144; larger sizes are rejected with HSPEC_ERR_BAD_SHAPE.
+ * The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).  Its FIRST call on a device
+ * resolves the array's device address (cudaGetSymbolAddress, with that device current); make that first call before
+ * any stream capture begins.  All calls share the array: calls that overlap on the GPU (e.g. on two streams) race.
+ * Inputs and outputs are the caller's, as in hspec_op_lm_head_argmax; results are identical to it. */
+int hspec_op_lm_head_argmax_noalloc(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M,
+                                    int32_t V, int32_t K, void* stream);
 /* RMSNorm over the last axis: y fp16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
 int hspec_op_rmsnorm(const float* x, const float* w, void* y_f16, int32_t M, int32_t n, float eps, void* stream);
 /* Mamba-2 mixer core for B requests x k rows (Sec. 3.3.1): causal depthwise conv + SiLU on xBC (zero left

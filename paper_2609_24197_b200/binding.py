@@ -19,7 +19,7 @@ _DT = {torch.bfloat16: 0, torch.float32: 1, torch.int32: 2, torch.float16: 3}
 EXPORTS = [
     "hspec_init", "hspec_workspace_bytes", "hspec_load_weights", "hspec_draft_block", "hspec_destroy",
     "hspec_last_error", "hspec_get_stats", "hspec_set_profiling", "hspec_get_profile", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
-    "hspec_op_lm_head_argmax", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
+    "hspec_op_lm_head_argmax", "hspec_op_lm_head_argmax_noalloc", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
 ]
 
@@ -95,6 +95,7 @@ def load_library(path=None):
     lib.hspec_gemm_workspace_bytes.argtypes = [i32, i32, i32]
     lib.hspec_gemm_workspace_bytes.restype = sz
     lib.hspec_op_lm_head_argmax.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp, sz, vp]
+    lib.hspec_op_lm_head_argmax_noalloc.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp]
     lib.hspec_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, f32, vp]
     lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.hspec_scan_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
@@ -250,6 +251,15 @@ def hspec_op_lm_head_argmax(x, W, ids, logits, workspace):
         _ptr(x), _ptr(W, x.dtype), _DT[x.dtype], _ptr(ids, torch.int32), _ptr(logits, torch.float32),
         M, W.shape[0], K, _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()),
         None, "hspec_op_lm_head_argmax")
+
+
+def hspec_op_lm_head_argmax_noalloc(x, W, ids, logits=None):
+    """LM head + arg-max without any device allocation: the scratch is a fixed array inside the library (M <= 512 rows,
+    V <= 262144).  For hosts that cannot allocate while drafting (pre-reserved HBM, no allocator handle)."""
+    M, K = x.shape
+    _check(load_library().hspec_op_lm_head_argmax_noalloc(
+        _ptr(x), _ptr(W, x.dtype), _DT[x.dtype], _ptr(ids, torch.int32), _ptr(logits, torch.float32), M, W.shape[0], K,
+        _stream()), None, "hspec_op_lm_head_argmax_noalloc")
 
 
 def hspec_op_rmsnorm(x, w, y, eps):

@@ -140,6 +140,8 @@ int fail(hspec_handle* h, int code, const std::string& msg);
 
 namespace hspec {
 
+void set_last_error(const std::string& msg) { g_err = msg; }
+
 void Tracker::begin(const char* name, double flops, double bytes) {
   ++launches;
   if (!profiling) return;

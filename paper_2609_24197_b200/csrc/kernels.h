@@ -11,6 +11,9 @@ namespace hspec {
 
 constexpr int GEMM_MAX_STAGES = 8;
 
+// Records the message hspec_last_error(NULL) returns (calling thread).
+void set_last_error(const std::string& msg);
+
 // Counts kernel launches and, when profiling is on, brackets each launch with a pair of CUDA events
 // recorded on the launching stream (read back with elapsed() after the stream is synchronised).
 struct Tracker {
