@@ -161,6 +161,25 @@ __device__ __forceinline__ uint32_t umma_idesc_m128(uint32_t n, bool f16) {
   return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// SwiGLU epilogue for 16 accumulator columns (activation rows m0 + c0 .. +15).  Weight rows are interleaved in blocks
+// of 16: lanes 0..15 of a warp hold the gate pre-activation of 16 features, lanes 16..31 the up projection of the same
+// features.  Columns are handled in pairs: the lower half-warp finishes the even column, the upper half the odd one,
+// so all 32 lanes compute and store.  `f` is the feature index of this lane (same for lane and lane ^ 16).
+__device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], __half* out, long long ldo, int m_first, int M, int f,
+                                               bool f_ok, int lane) {
+  const bool upper = lane >= 16;
+#pragma unroll
+  for (int j = 0; j < 16; j += 2) {
+    const float mine_even = __uint_as_float(r[j]), mine_odd = __uint_as_float(r[j + 1]);
+    const float send = upper ? mine_even : mine_odd;           // what the partner needs from me
+    const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
+    const float gate = upper ? recv : mine_even;               // upper half: partner's gate of the odd column
+    const float up = upper ? mine_odd : recv;                  // lower half: partner's up of the even column
+    const int m = m_first + j + (upper ? 1 : 0);
+    if (f_ok && m < M) out[size_t(m) * ldo + f] = __float2half_rn(silu_f(gate) * up);
+  }
+}
+
 // ------------------------------------------------------------------ warp-level mma (attention)
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"

@@ -214,7 +214,7 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = tm * g.BNT;
       const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT) + (uint32_t(q * 32) << 16);
       for (int c0 = 0; c0 < g.BNT; c0 += 16) {
-        if (m0 + c0 >= g.M && g.mode != EPI_ARGMAX) break;    // rows past M: nothing to store
+        if (m0 + c0 >= g.M && g.mode != EPI_ARGMAX) break;    // rows past M: nothing to store (warp-uniform)
         uint32_t r[16];
         tmem_ld16(tmem_acc + uint32_t(c0), r);
         tmem_ld_wait();
@@ -239,6 +239,9 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int m = m0 + c0 + j;
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = old[j] + __uint_as_float(r[j]);
           }
+        } else if (g.mode == EPI_SWIGLU_F16) {
+          const int f = tile_n128 * 64 + q * 16 + (lane & 15);
+          swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane);
         } else if (g.mode == EPI_STORE_F16) {
           __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll

@@ -49,7 +49,7 @@ int imax(int a, int b) { return a > b ? a : b; }
 
 // Offsets of the step's scratch buffers inside the caller's workspace.
 struct Plan {
-  size_t X, U, BIG, LH, Fv, SINIT, SCAN, scan_bytes, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
+  size_t X, U, U2, BIG, LH, Fv, SINIT, SCAN, scan_bytes, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
   size_t att_bytes, splitk_bytes;
   int attn_chunk, max_ctx;
 };
@@ -65,7 +65,8 @@ Plan make_plan(const hspec_config& c, int B, int k, int max_ctx) {
   size_t at = 0;
   auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 1024); return o; };
   p.X = take(M * c.D * 4);
-  p.U = take(M * size_t(imax(imax(c.D, c.Di), imax(c.Hq * c.dh, c.F))) * 2);
+  p.U = take(M * size_t(imax(imax(c.D, c.Di), c.Hq * c.dh)) * 2);
+  p.U2 = take(M * size_t(c.F) * 2);
   p.BIG = take(M * size_t(imax(imax(d.d_in_proj, d.d_qkv), 2 * c.F)) * 4);
   p.LH = take(size_t(B) * c.n_fuse * c.D * 2);
   p.Fv = take(size_t(B) * c.r * 2);
@@ -254,6 +255,18 @@ __global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half
     dst[i] = __float2half_rn(__bfloat162float(src[i]));
 }
 
+// w_gate_up [2F, K] bf16 (rows gate | up) -> fp16 with rows interleaved in blocks of 16:
+// dst rows [32j, 32j+16) = gate rows [16j, 16j+16), dst rows [32j+16, 32j+32) = up rows [16j, 16j+16).
+__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int F, int K) {
+  const size_t total = size_t(2) * F * K;
+  for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < total; i += size_t(gridDim.x) * blockDim.x) {
+    const size_t r = i / K, c = i % K;
+    const size_t blk = r >> 5, w = r & 31;
+    const size_t src_row = (w < 16) ? blk * 16 + w : size_t(F) + blk * 16 + (w - 16);
+    dst[i] = __float2half_rn(__bfloat162float(src[src_row * K + c]));
+  }
+}
+
 __global__ void cvt_cols_f16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
                                     __half* __restrict__ dst) {
   const int total = M * ncols;
@@ -316,8 +329,12 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
     if (gemm) {
       // bf16 -> fp16: exact for every value with |w| in [2^-17, 65504]; smaller ones lose at most 2^-25
       const int blocks = int(std::min<size_t>((count + 255) / 256, 148 * 32));
-      bf16_to_f16_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
-                                          reinterpret_cast<__half*>(w.data), count);
+      if (name.size() >= 13 && name.compare(name.size() - 13, 13, "mlp.w_gate_up") == 0 && h->cfg.F % 16 == 0)
+        interleave_gate_up_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
+                                                   reinterpret_cast<__half*>(w.data), h->cfg.F, int(cols));
+      else
+        bf16_to_f16_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
+                                            reinterpret_cast<__half*>(w.data), count);
       CUDA_TRY(h, cudaGetLastError());
       if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, true, &errtxt)) {
         cudaFree(w.data);
@@ -405,6 +422,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   uint8_t* ws = reinterpret_cast<uint8_t*>(in->workspace);
   float* X = reinterpret_cast<float*>(ws + p.X);
   void* U = ws + p.U;
+  void* U2 = ws + p.U2;
   float* BIG = reinterpret_cast<float*>(ws + p.BIG);
   void* LH = ws + p.LH;
   void* Fv = ws + p.Fv;
@@ -491,9 +509,15 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     }
     // ---- SwiGLU MLP
     EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st));
-    CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
-    EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U, M, c.F, st));
-    CUDA_TRY(h, gemm(pre + "mlp.w_down", "gemm:down", U, M, EPI_ACCUM_F32, X, c.D));
+    if (c.F % 16 == 0) {
+      // gate/up rows were interleaved at load: the GEMM epilogue applies SiLU(gate) * up and writes h directly.
+      // U is both the GEMM's input (D columns) and h's home (F columns), so h goes to a second fp16 buffer.
+      CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_SWIGLU_F16, U2, c.F));
+    } else {
+      CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
+      EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U2, M, c.F, st));
+    }
+    CUDA_TRY(h, gemm(pre + "mlp.w_down", "gemm:down", U2, M, EPI_ACCUM_F32, X, c.D));
   }
   if (out->hidden) EW("copy_hidden", Md * c.D * 8, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st));
   // ---- final norm, LM head fused with the per-row arg-max

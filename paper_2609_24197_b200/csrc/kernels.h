@@ -41,7 +41,8 @@ enum GemmEpilogue : int {
   EPI_ACCUM_F32 = 2,    // y fp32 += acc   (residual)
   EPI_PARTIAL_F32 = 3,  // K-slice partial (internal)
   EPI_ARGMAX = 4,
-  EPI_STORE_F16 = 5,    // y fp16 = acc       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
+  EPI_STORE_F16 = 5,    // y fp16 = acc
+  EPI_SWIGLU_F16 = 6,   // weight rows interleaved in blocks of 16 (gate | up): h fp16 [M, n_out/2] = SiLU(gate) * up       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
 };
 
 struct GemmArgs {       // kernel argument block
