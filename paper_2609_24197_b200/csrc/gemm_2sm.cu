@@ -144,6 +144,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (warp == 0) {
     if (lane == 0) {
+      // evict-first on the weights measured faster than evict-normal (1.25 vs 1.15 PFLOP/s on 2048 x 51200 x 5120)
+      // although ncu shows 2.4x the algorithmic DRAM reads: the activation tile must not be pushed out of L2
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
