@@ -450,7 +450,8 @@ def main():
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=HEADLINE, choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default=HEADLINE,
+                    help="one of %s, or a sweep cell sweep_8b_B<B>_k<k>" % ", ".join(sorted(synth.CONFIGS)))
     ap.add_argument("--headline-only", action="store_true", help="skip the concurrency-1 and -32 workloads")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lean", action="store_true", help="only warm-up + timed steps (for profiler launch lists)")

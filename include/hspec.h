@@ -78,7 +78,9 @@ typedef struct {
   int32_t window;            /* sliding window in tokens, 0 = full context */
   int32_t qk_norm;           /* 1: per-head RMSNorm on q and the block's k before RoPE */
   int32_t F;                 /* SwiGLU width */
-  int32_t V;                 /* vocabulary (rows of the LM head) */
+  int32_t V;                 /* target vocabulary (rows of `embed`; of `lm_head` too unless V_draft > 0) */
+  int32_t V_draft;           /* 0, or the size of a pruned drafter vocabulary (App. B.2 "Pruned drafter vocabulary"): the LM
+                                head then has V_draft rows and `vocab_map` translates a row index into a target token id */
   int32_t mask_id;           /* token id whose embedding fills block rows 1..k-1 */
   float rms_eps;
   int32_t page_size;         /* tokens per KV page (16) */
@@ -89,7 +91,8 @@ typedef struct {
 
 /* A named tensor in DEVICE memory.  hspec_load_weights copies it (converting GEMM matrices to fp16), so
  * the caller may free or reuse it afterwards.  Names (l = layer index):
- *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D]
+ *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D] (or [V_draft,D])
+ *   vocab_map [V_draft] int32 (only if V_draft > 0: target token id of each LM-head row, ascending)
  *   layers.l.mamba.{norm [D], in_proj [Di + (Di+2GN) + (dt_rank or H), D] (rows z | xBC | dt),
  *                   dt_up [H, dt_rank] (only if dt_rank>0), conv_w [Di+2GN, d_conv], conv_b [Di+2GN],
  *                   dt_bias [H], A_log [H], Dskip [H], gnorm [Di], out_proj [D, Di]}
@@ -129,8 +132,9 @@ typedef struct {
 
 /* Outputs of one step, device memory owned by the caller. */
 typedef struct {
-  int32_t* draft_ids;   /* int32 [B, k], required: arg-max of the logits, lowest index on ties */
-  float* logits;        /* fp32 [B, k, V] or NULL (then the logits are never materialised) */
+  int32_t* draft_ids;   /* int32 [B, k], required: arg-max of the logits, lowest row index on ties; target token ids
+                           (mapped through vocab_map when the drafter vocabulary is pruned) */
+  float* logits;        /* fp32 [B, k, V] ([B, k, V_draft] when pruned) or NULL (then the logits are never materialised) */
   float* hidden;        /* fp32 [B, k, D] or NULL: the residual stream before the final norm */
 } hspec_out;
 
@@ -166,6 +170,12 @@ int hspec_destroy(hspec_handle* h);
 /* Message of the last failure on this handle (or of the last failed hspec_init if h is NULL). */
 const char* hspec_last_error(const hspec_handle* h);
 int hspec_get_stats(hspec_handle* h, hspec_stats* out);
+/* Failure-path self-test: enqueues a one-thread kernel that waits, for at most limit_ms (1..2000), on a barrier nothing
+ * completes; it then gives up, writes a code to the handle's device status word and returns normally (no trap: the
+ * context stays usable).  hspec_get_stats afterwards reports HSPEC_ERR_TIMEOUT with device_status != 0, which is how
+ * a bounded in-kernel wait that gave up inside a real step surfaces.  hspec_clear_status resets the word. */
+int hspec_debug_wait_selftest(hspec_handle* h, int32_t limit_ms, void* stream);
+int hspec_clear_status(hspec_handle* h);
 /* Measurement aid: when on, every kernel launch of a step is bracketed by CUDA events on the step's stream. */
 int hspec_set_profiling(hspec_handle* h, int32_t on);
 /* Per-launch times of the LAST step (synchronises its stream).  Returns the number of entries written (<= max_entries)

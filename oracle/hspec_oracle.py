@@ -343,13 +343,15 @@ def draft_block(cfg, weights, k_pools, v_pools, page_table, ctx_lens, last_hidde
       block rows X[0] = E[last_token], X[i>0] = E[mask] (no positional embedding);
       for each layer: X += Mamba(RMSNorm(X)); X += Attn(RMSNorm(X)) if the layer has
       attention (target KV of slot kv_slot[l]); X += MLP(RMSNorm(X));
-      logits = RMSNorm(X) W_lm^T; draft ids = argmax (lowest index on ties).
+      logits = RMSNorm(X) W_lm^T; draft ids = argmax (lowest index on ties), translated through
+      `vocab_map` when the drafter predicts over a pruned vocabulary (the LM head then holds only those rows).
     Returns dict: draft_ids [n, k], logits [n, k, V], hidden [n, k, D], margin [n, k],
     s_init [n, H, P, N] and, if asked, per-request intermediates.
     """
     B = len(ctx_lens)
     requests = list(range(B)) if requests is None else list(requests)
-    D, V = cfg["D"], cfg["V"]
+    D = cfg["D"]
+    V = int(np.asarray(weights["lm_head"]).shape[0])      # the target vocabulary, or a pruned drafter vocabulary
     eps = cfg["rms_eps"]
     out = dict(draft_ids=np.empty((len(requests), k), np.int32),
                logits=np.empty((len(requests), k, V), dtype),
@@ -386,6 +388,8 @@ def draft_block(cfg, weights, k_pools, v_pools, page_table, ctx_lens, last_hidde
                 inter[f"x_after_mlp.{l}"] = X.copy()
         logits = gemm(rmsnorm(X, widen(weights["final_norm"], dtype), eps), weights["lm_head"], dtype)
         ids, margin = argmax_margin(logits)
+        if "vocab_map" in weights:        # pruned drafter vocabulary: LM-head row index -> target token id
+            ids = np.asarray(weights["vocab_map"])[ids].astype(np.int32)
         out["draft_ids"][n], out["logits"][n], out["hidden"][n] = ids, logits, X
         out["margin"][n], out["s_init"][n] = margin, S_init
         out["intermediates"].append(inter)

@@ -18,7 +18,8 @@ _DT = {torch.bfloat16: 0, torch.float32: 1, torch.int32: 2, torch.float16: 3}
 
 EXPORTS = [
     "hspec_init", "hspec_workspace_bytes", "hspec_load_weights", "hspec_draft_block", "hspec_destroy",
-    "hspec_last_error", "hspec_get_stats", "hspec_set_profiling", "hspec_get_profile", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
+    "hspec_last_error", "hspec_get_stats", "hspec_set_profiling", "hspec_get_profile",
+    "hspec_debug_wait_selftest", "hspec_clear_status", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
     "hspec_op_lm_head_argmax", "hspec_op_lm_head_argmax_noalloc", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
 ]
@@ -35,7 +36,7 @@ class hspec_config(C.Structure):
         ("n_slots", C.c_int32), ("Di", C.c_int32), ("P", C.c_int32), ("N", C.c_int32), ("G", C.c_int32),
         ("d_conv", C.c_int32), ("dt_rank", C.c_int32), ("Hq", C.c_int32), ("Hkv", C.c_int32), ("dh", C.c_int32),
         ("rope_theta", C.c_float), ("window", C.c_int32), ("qk_norm", C.c_int32), ("F", C.c_int32),
-        ("V", C.c_int32), ("mask_id", C.c_int32), ("rms_eps", C.c_float), ("page_size", C.c_int32),
+        ("V", C.c_int32), ("V_draft", C.c_int32), ("mask_id", C.c_int32), ("rms_eps", C.c_float), ("page_size", C.c_int32),
         ("max_batch", C.c_int32), ("max_k", C.c_int32), ("max_pages_per_req", C.c_int32),
     ]
 
@@ -89,6 +90,8 @@ def load_library(path=None):
     lib.hspec_last_error.restype = C.c_char_p
     lib.hspec_get_stats.argtypes = [C.c_void_p, C.POINTER(hspec_stats)]
     lib.hspec_set_profiling.argtypes = [C.c_void_p, C.c_int32]
+    lib.hspec_debug_wait_selftest.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+    lib.hspec_clear_status.argtypes = [C.c_void_p]
     lib.hspec_get_profile.argtypes = [C.c_void_p, C.POINTER(hspec_prof_entry), C.c_int32]
     vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
     lib.hspec_op_gemm.argtypes = [vp, vp, i32, vp, i32, i32, i32, i64, i32, i32, i32, vp, sz, vp]
@@ -138,6 +141,7 @@ def make_config(cfg, max_batch=None, max_k=None, max_pages_per_req=None):
     for name in ("D", "n_fuse", "r", "L", "n_slots", "Di", "P", "N", "G", "d_conv", "dt_rank", "Hq", "Hkv", "dh",
                  "window", "qk_norm", "F", "V", "mask_id", "page_size"):
         setattr(c, name, int(cfg[name]))
+    c.V_draft = int(cfg.get("V_draft", 0))
     c.rope_theta = float(cfg["rope_theta"])
     c.rms_eps = float(cfg["rms_eps"])
     for l in range(int(cfg["L"])):
@@ -170,7 +174,7 @@ def hspec_load_weights(handle, tensors):
         keep.append(bname)
         arr[i].name = bname
         arr[i].data = t.data_ptr()
-        arr[i].dtype = {torch.bfloat16: HSPEC_BF16, torch.float32: HSPEC_F32}[t.dtype]
+        arr[i].dtype = {torch.bfloat16: HSPEC_BF16, torch.float32: HSPEC_F32, torch.int32: HSPEC_I32}[t.dtype]
         arr[i].ndim = t.dim()
         for j in range(t.dim()):
             arr[i].shape[j] = t.shape[j]
@@ -213,6 +217,14 @@ def hspec_get_stats(handle):
     rc = load_library().hspec_get_stats(handle, C.byref(s))
     return dict(kernel_launches=int(s.kernel_launches), device_status=int(s.device_status),
                 launches_last_step=int(s.launches_last_step), rc=rc)
+
+
+def hspec_debug_wait_selftest(handle, limit_ms=100):
+    _check(load_library().hspec_debug_wait_selftest(handle, int(limit_ms), _stream()), handle, "hspec_debug_wait_selftest")
+
+
+def hspec_clear_status(handle):
+    _check(load_library().hspec_clear_status(handle), handle, "hspec_clear_status")
 
 
 def hspec_set_profiling(handle, on):
@@ -337,7 +349,8 @@ class Drafter:
         B = batch["ctx_lens"].shape[0]
         dev = batch["ctx_lens"].device
         ids = torch.empty((B, k), dtype=torch.int32, device=dev)
-        logits = torch.empty((B, k, self.cfg["V"]), dtype=torch.float32, device=dev) if want_logits else None
+        v_out = self.cfg.get("V_draft", 0) or self.cfg["V"]
+        logits = torch.empty((B, k, v_out), dtype=torch.float32, device=dev) if want_logits else None
         hidden = torch.empty((B, k, self.cfg["D"]), dtype=torch.float32, device=dev) if want_hidden else None
         hspec_draft_block(self.handle, batch["page_table"], batch["ctx_lens"], batch["last_hidden"],
                           batch["last_token"], k, batch["k_pools"], batch["v_pools"], self.workspace, ids, logits,

@@ -13,6 +13,7 @@ enum : uint32_t {
   STATUS_TIMEOUT_PRODUCER = 0x101,
   STATUS_TIMEOUT_MMA = 0x102,
   STATUS_TIMEOUT_EPILOGUE = 0x103,
+  STATUS_TIMEOUT_SELFTEST = 0x1ff,
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -64,14 +65,14 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 }
 // Bounded wait: polls the barrier and gives up after about two seconds of wall time (checked every
 // 1024 polls).  Returns false on give-up; the caller records a status code and unwinds.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_t limit_ns = 2000000000ull) {
   uint64_t t0 = 0;
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u) {
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > 2000000000ull) return false;
+      else if (now - t0 > limit_ns) return false;
     }
   }
 }

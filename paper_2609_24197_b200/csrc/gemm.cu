@@ -246,7 +246,7 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
 
 // ids[m] = lowest index among the per-tile maxima (tiles are in ascending vocabulary order).
 __global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
-                                     int* __restrict__ ids) {
+                                     int* __restrict__ ids, const int* __restrict__ id_map) {
   const int m = blockIdx.x;
   float v = -INFINITY;
   int idx = 0x7fffffff;
@@ -273,7 +273,7 @@ __global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __
       const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
       if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
     }
-    if (threadIdx.x == 0) ids[m] = idx;
+    if (threadIdx.x == 0) ids[m] = id_map ? id_map[idx] : idx;   // pruned drafter vocabulary: row index -> token id
   }
 }
 
@@ -414,9 +414,9 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
 }
 
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
-                                 Tracker* trk) {
+                                 Tracker* trk, const int* id_map) {
   trk_begin(trk, "argmax_reduce", 0, double(n_tiles) * M * 8);
-  argmax_reduce_kernel<<<M, 256, 0, stream>>>(pv, pi, n_tiles, M, ids);
+  argmax_reduce_kernel<<<M, 256, 0, stream>>>(pv, pi, n_tiles, M, ids, id_map);
   trk_end(trk);
   return cudaGetLastError();
 }

@@ -12,6 +12,7 @@
 #include <unordered_map>
 #include <vector>
 
+#include "common.cuh"
 #include "kernels.h"
 
 using namespace hspec;
@@ -31,6 +32,7 @@ struct Weight {
 
 struct Dims {
   int H, d_S, d_xBC, d_dt, d_in_proj, d_qkv;
+  int Vd;   // rows of the LM head: the target vocabulary, or the pruned drafter vocabulary
 };
 
 Dims dims_of(const hspec_config& c) {
@@ -41,6 +43,7 @@ Dims dims_of(const hspec_config& c) {
   d.d_dt = c.dt_rank > 0 ? c.dt_rank : d.H;
   d.d_in_proj = c.Di + d.d_xBC + d.d_dt;
   d.d_qkv = (c.Hq + 2 * c.Hkv) * c.dh;
+  d.Vd = c.V_draft > 0 ? c.V_draft : c.V;
   return d;
 }
 
@@ -96,7 +99,7 @@ Plan make_plan(const hspec_config& c, int B, int k, int max_ctx) {
   upd(splitk_need(int(M), c.D, c.F));
   p.splitk_bytes = sk;
   p.SPLITK = take(sk);
-  const size_t vt = (size_t(c.V) + 127) / 128;
+  const size_t vt = 2 * ((size_t(d.Vd) + 255) / 256);   // 128-row tiles, in pairs (the 2-SM kernel's indexing)
   p.AMAXV = take(vt * M * 4);
   p.AMAXI = take(vt * M * 4);
   p.total = at;
@@ -116,6 +119,7 @@ const char* check_config(const hspec_config& c) {
   if (c.Hkv < 1 || c.Hq < c.Hkv || c.Hq % c.Hkv) return "Hq must be a multiple of Hkv";
   if (c.F < 8 || c.F % 8) return "F must be a multiple of 8";
   if (c.V < 2 || c.mask_id < 0 || c.mask_id >= c.V) return "V / mask_id out of range";
+  if (c.V_draft < 0 || c.V_draft > c.V) return "V_draft must be 0 or at most V";
   if (c.page_size < 1 || c.max_batch < 1 || c.max_pages_per_req < 1) return "page_size, max_batch, max_pages_per_req must be positive";
   if (c.max_k < 1 || c.max_k > HSPEC_MAX_K) return "max_k out of range";
   if (c.max_k * (c.Hq / c.Hkv) > 1024) return "k * Hq/Hkv too large";
@@ -211,7 +215,8 @@ bool expected_shape(const hspec_config& c, const Dims& d, const std::string& nam
   if (name == "proj_r") return mat(c.r, int64_t(c.n_fuse) * c.D, true);
   if (name == "proj_ds") return mat(d.d_S, c.r, true);
   if (name == "final_norm") return vec(c.D);
-  if (name == "lm_head") return mat(c.V, c.D, true);
+  if (name == "lm_head") return mat(d.Vd, c.D, true);
+  if (name == "vocab_map") { if (c.V_draft <= 0) return false; *rows = c.V_draft; *cols = 0; *dtype = HSPEC_I32; return true; }
   if (name.rfind("layers.", 0) != 0) return false;
   const size_t dot = name.find('.', 7);
   if (dot == std::string::npos) return false;
@@ -238,6 +243,7 @@ bool expected_shape(const hspec_config& c, const Dims& d, const std::string& nam
 
 std::vector<std::string> required_names(const hspec_config& c) {
   std::vector<std::string> n = {"embed", "proj_r", "proj_ds", "final_norm", "lm_head"};
+  if (c.V_draft > 0) n.push_back("vocab_map");
   for (int l = 0; l < c.L; ++l) {
     const std::string p = "layers." + std::to_string(l) + ".";
     for (const char* s : {"mamba.norm", "mamba.in_proj", "mamba.conv_w", "mamba.conv_b", "mamba.dt_bias", "mamba.A_log",
@@ -264,6 +270,17 @@ __global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src,
     const size_t blk = r >> 5, w = r & 31;
     const size_t src_row = (w < 16) ? blk * 16 + w : size_t(F) + blk * 16 + (w - 16);
     dst[i] = __float2half_rn(__bfloat162float(src[src_row * K + c]));
+  }
+}
+
+// Self-test of the bounded-wait path: waits on a barrier that nothing will ever complete, for a short limit, then
+// records the give-up in the status word and returns normally (no trap, the context stays usable).
+__global__ void wait_selftest_kernel(uint32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    fence_mbar_init();
+    if (!mbar_wait(smem_u32(&bar), 0, limit_ns)) atomicExch(status, STATUS_TIMEOUT_SELFTEST);
   }
 }
 
@@ -324,7 +341,7 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
     Weight w;
     w.dtype = dtype; w.rows = rows; w.cols = cols;
     const size_t count = size_t(rows) * size_t(cols ? cols : 1);
-    const size_t bytes = count * (dtype == HSPEC_F32 ? 4 : 2);
+    const size_t bytes = count * ((dtype == HSPEC_F32 || dtype == HSPEC_I32) ? 4 : 2);
     CUDA_TRY(h, cudaMalloc(&w.data, bytes));
     if (gemm) {
       // bf16 -> fp16: exact for every value with |w| in [2^-17, 65504]; smaller ones lose at most 2^-25
@@ -525,15 +542,40 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   {
     const Weight& w = W("lm_head");
     GemmCall g{};
-    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = c.V; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
-    g.logits = out->logits; g.ldo = c.V;
+    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
+    g.logits = out->logits; g.ldo = d.Vd;
     g.part_val = reinterpret_cast<float*>(ws + p.AMAXV); g.part_idx = reinterpret_cast<int*>(ws + p.AMAXI);
     g.status = h->d_status; g.label = "gemm:lm_head_argmax";
     CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
-    CUDA_TRY(h, argmax_reduce_launch(g.part_val, g.part_idx, (c.V + 127) / 128, M, out->draft_ids, st, trk));
+    const int* id_map = c.V_draft > 0 ? reinterpret_cast<const int*>(W("vocab_map").data) : nullptr;
+    CUDA_TRY(h, argmax_reduce_launch(g.part_val, g.part_idx, (d.Vd + 127) / 128, M, out->draft_ids, st, trk, id_map));
   }
 #undef EW
   h->launches_last_step = uint32_t(trk->launches - launches0);
+  return HSPEC_OK;
+}
+
+int hspec_debug_wait_selftest(hspec_handle* h, int32_t limit_ms, void* stream) {
+  if (!h || limit_ms < 1 || limit_ms > 2000) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_debug_wait_selftest: bad argument");
+  std::string errtxt;
+  if (!h->d_status) {
+    CUDA_TRY(h, cudaMalloc(&h->d_status, 256));
+    CUDA_TRY(h, cudaMemset(h->d_status, 0, 256));
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  h->last_stream = st;
+  wait_selftest_kernel<<<1, 32, 0, st>>>(h->d_status, (unsigned long long)limit_ms * 1000000ull);
+  CUDA_TRY(h, cudaGetLastError());
+  return HSPEC_OK;
+}
+
+int hspec_clear_status(hspec_handle* h) {
+  if (!h) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_clear_status: NULL handle");
+  std::string errtxt;
+  if (h->d_status) {
+    CUDA_TRY(h, cudaStreamSynchronize(h->last_stream));
+    CUDA_TRY(h, cudaMemset(h->d_status, 0, 256));
+  }
   return HSPEC_OK;
 }
 

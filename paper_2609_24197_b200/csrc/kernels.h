@@ -90,7 +90,7 @@ bool gemm2_preferred(int M, int n_out);        // many rows and at least one ful
 int gemm2_pick_bnt(int M, int n_out);
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
-                                 Tracker* trk);
+                                 Tracker* trk, const int* id_map = nullptr);
 
 // ---- attention (attention.cu)
 struct AttnCall {

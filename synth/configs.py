@@ -42,6 +42,8 @@ CONFIGS = {
     "latency_8b": dict(_MODEL_8B, name="latency_8b", B=1, k=16, ctx=("const", 2048, 2048)),
     "serving_8b": dict(_MODEL_8B, name="serving_8b", B=32, k=16, ctx=("uniform", 512, 8192)),
     "conc128_32b": dict(_MODEL_32B, name="conc128_32b", B=128, k=16, ctx=("loguniform", 1024, 32768)),
+    # the concurrency-128 workload with the drafter predicting over a pruned 32 000-token vocabulary (App. B.2)
+    "conc128_32b_v32k": dict(_MODEL_32B, name="conc128_32b_v32k", V_draft=32000, B=128, k=16, ctx=("loguniform", 1024, 32768)),
     "paper_8b": dict(_MODEL_PAPER_8B, name="paper_8b", B=32, k=8, ctx=("uniform", 512, 8192)),
 }
 
@@ -52,6 +54,12 @@ def sweep_config(B, k):
 
 
 def get_config(name, **overrides):
+    """Config by name: one of CONFIGS, or a sweep cell 'sweep_8b_B<B>_k<k>'."""
+    if name.startswith("sweep_8b_B"):
+        B, k = name[len("sweep_8b_B"):].split("_k")
+        cfg = sweep_config(int(B), int(k))
+        cfg.update(overrides)
+        return derived(cfg)
     cfg = copy.deepcopy(CONFIGS[name])
     cfg.update(overrides)
     return derived(cfg)

@@ -68,8 +68,10 @@ def weight_shapes(cfg):
         "proj_r": ((cfg["r"], cfg["n_fuse"] * D), "mat"),
         "proj_ds": ((cfg["d_S"], cfg["r"]), "mat"),
         "final_norm": ((D,), "gain"),
-        "lm_head": ((cfg["V"], D), "mat"),
+        "lm_head": ((cfg.get("V_draft", 0) or cfg["V"], D), "mat"),
     }
+    if cfg.get("V_draft", 0):
+        sh["vocab_map"] = ((cfg["V_draft"],), "vocab_map")   # drafter row -> target token id (pruned vocabulary)
     for l in range(L):
         p = f"layers.{l}."
         sh[p + "mamba.norm"] = ((D,), "gain")
@@ -114,6 +116,11 @@ def make_weights(cfg, device="cpu", only=None):
         elif kind == "dt_bias":
             dt = torch.exp(_uniform(shape, math.log(1e-3), math.log(1e-1), name, device).double())
             t = (dt + torch.log(-torch.expm1(-dt))).float()      # inverse softplus
+        elif kind == "vocab_map":
+            # a seeded random subset of the target vocabulary, ascending (the real list is "most frequent tokens in
+            # the training corpus", which is not available here)
+            g = _gen("cpu", tensor_seed(name))
+            t = torch.sort(torch.randperm(cfg["V"], generator=g)[:shape[0]])[0].to(torch.int32).to(device)
         elif kind == "Dskip":
             t = torch.ones(shape, dtype=torch.float32, device=device)
         else:

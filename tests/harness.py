@@ -67,7 +67,10 @@ def check_step(cfg, drafter, weights, batch, k, requests=None, dtype=np.float64,
     ref = oracle_step(cfg, weights, batch, k, requests, dtype)
     ids, logits, hidden = ids.cpu().numpy(), logits.cpu().numpy(), hidden.cpu().numpy()
     # the fused arg-max must agree with the library's own logits exactly (lowest index on ties)
-    np.testing.assert_array_equal(ids, np.argmax(logits, axis=-1).astype(np.int32))
+    own = np.argmax(logits, axis=-1).astype(np.int32)
+    if "vocab_map" in weights:
+        own = weights["vocab_map"].cpu().numpy()[own]
+    np.testing.assert_array_equal(ids, own)
     e_h = assert_close(hidden[requests], ref["hidden"], what + " hidden")
     e_l = assert_close(logits[requests], ref["logits"], what + " logits")
     sure = ref["margin"] > MARGIN

@@ -121,3 +121,41 @@ def test_serving_8b_full_size_sampled_requests():
 
 def test_conc128_32b_full_size_sampled_request():
     _full_size("conc128_32b", 1)
+
+
+def test_paper_shape_drafter_sampled_requests():
+    # the paper's own drafter shape (App. B.1): 48 Mamba heads x 64 with state = groups = conv = 4, five fused target
+    # layers, three attention layers + one Mamba-MLP layer, 2048-token window
+    _full_size("paper_8b", 2)
+
+
+def test_sweep_cell_8b_B128_k8_sampled_request():
+    _full_size("sweep_8b_B128_k8", 1)
+
+
+def test_mid_config_pruned_drafter_vocabulary():
+    cfg = synth.derived(dict(MID, V_draft=700, B=2))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[300, 41])
+    r = check_step(cfg, drafter, w, batch, 9, what="mid pruned vocab")
+    assert r["ids_compared"] > 0
+    drafter.close()
+
+
+def test_bounded_wait_gives_up_and_reports_without_killing_the_context():
+    # failure detection without a GPU fault: a wait nobody satisfies runs out, the kernel records a status code and
+    # returns; the host sees HSPEC_ERR_TIMEOUT, clears it, and the same handle then drafts correctly
+    import paper_2609_24197_b200 as hs
+    cfg = synth.get_config("tiny")
+    drafter, w, batch = cuda_setup(cfg)
+    ids0, _, _ = drafter.draft(batch, cfg["k"])
+    torch.cuda.synchronize()
+    assert drafter.stats()["device_status"] == 0
+    hs.hspec_debug_wait_selftest(drafter.handle, 50)
+    st = drafter.stats()
+    assert st["rc"] == -7 and st["device_status"] == 0x1FF            # HSPEC_ERR_TIMEOUT, the self-test's code
+    hs.hspec_clear_status(drafter.handle)
+    assert drafter.stats()["device_status"] == 0
+    ids1, _, _ = drafter.draft(batch, cfg["k"])
+    torch.cuda.synchronize()
+    assert torch.equal(ids0, ids1) and drafter.stats()["device_status"] == 0
+    drafter.close()

@@ -150,3 +150,17 @@ def test_tiny_config_runs_and_has_expected_scale():
     assert out["draft_ids"].shape == (1, 8) and np.isfinite(out["logits"]).all()
     # logits std ~ 0.02 * sqrt(D) = 0.32 for unit-RMS final-norm output
     assert 0.2 < out["logits"].std() < 0.45
+
+
+def test_pruned_vocabulary_is_a_row_subset_with_an_id_map():
+    cfg, w, batch = _setup([19])
+    full = _run(cfg, w, batch, 4)
+    keep = np.array([1, 2, 5, 6, 9], dtype=np.int32)                     # ascending subset of the 11 target tokens
+    cfg_p = synth.derived(dict(cfg, V_draft=5))
+    w_p = dict(w)
+    w_p["lm_head"] = np.asarray(w["lm_head"])[keep]
+    w_p["vocab_map"] = keep
+    pruned = _run(cfg_p, w_p, batch, 4)
+    np.testing.assert_array_equal(pruned["logits"], full["logits"][:, :, keep])
+    np.testing.assert_array_equal(pruned["draft_ids"], keep[np.argmax(full["logits"][:, :, keep], axis=-1)])
+    assert set(pruned["draft_ids"].ravel().tolist()) <= set(keep.tolist())
