@@ -499,8 +499,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 }
 
 // One block per (row of the block, query head): merge the chunk partials in chunk order (page-aligned chunk geometry).
-__global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o) {
-  const int m = blockIdx.x, hq = blockIdx.y;
+__global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n_pairs) {
+  // one warp per (row, head): each lane merges four adjacent head-dim columns with 16-byte loads
+  const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pair >= n_pairs) return;
+  const int m = pair / a.Hq, hq = pair % a.Hq;
   const int b = m / a.k, i = m % a.k;
   const int kvh = hq / a.rep, r = i * a.rep + hq % a.rep;
   const Range g = make_range(a.ctx_lens[b], a.window, a.chunk, 0, a.k);
@@ -508,15 +511,22 @@ __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o) {
   float m_tot = -INFINITY;
   for (int c = 0; c < g.n_chunks; ++c) m_tot = fmaxf(m_tot, a.ws_ml[((slab0 + c) * a.R + r) * 2]);
   const float ref = (m_tot == -INFINITY) ? 0.f : m_tot;
-  const int d = threadIdx.x;
-  float acc = 0.f, L = 0.f;
+  const int d4 = threadIdx.x & 31;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float L = 0.f;
   for (int c = 0; c < g.n_chunks; ++c) {
     const float* ml = a.ws_ml + ((slab0 + c) * a.R + r) * 2;
     const float w = exp2f(ml[0] - ref);
     L += ml[1] * w;
-    acc += a.ws_o[((slab0 + c) * a.R + r) * DH + d] * w;
+    const float4 v = reinterpret_cast<const float4*>(a.ws_o + ((slab0 + c) * a.R + r) * DH)[d4];
+    acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
   }
-  o[(size_t(m) * a.Hq + hq) * DH + d] = __float2half_rn(acc / L);
+  const float inv = 1.f / L;
+  __half2 lo = __floats2half2_rn(acc.x * inv, acc.y * inv), hi = __floats2half2_rn(acc.z * inv, acc.w * inv);
+  uint2 out;
+  out.x = *reinterpret_cast<uint32_t*>(&lo);
+  out.y = *reinterpret_cast<uint32_t*>(&hi);
+  reinterpret_cast<uint2*>(o + (size_t(m) * a.Hq + hq) * DH)[d4] = out;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -583,9 +593,9 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  dim3 mgrid(c.B * c.k, c.Hq);
+  const int n_pairs = c.B * c.k * c.Hq;
   trk_begin(trk, "attn_merge");
-  attn_tc_merge_kernel<<<mgrid, DH, 0, stream>>>(a, reinterpret_cast<__half*>(c.o));
+  attn_tc_merge_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(a, reinterpret_cast<__half*>(c.o), n_pairs);
   trk_end(trk);
   return cudaGetLastError();
 }

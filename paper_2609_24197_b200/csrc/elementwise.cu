@@ -40,24 +40,55 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
                                int n, float eps) {
   __shared__ float red[32];
   const float* xr = x + size_t(blockIdx.x) * n;
+  __half* yr = y + size_t(blockIdx.x) * n;
+  if ((n & 3) == 0 && n <= 4 * 6 * int(blockDim.x)) {
+    // 16-byte loads, the row stays in registers between the two passes
+    float4 v[6];
+    const int nv = n >> 2;
+    float ss = 0.f;
+#pragma unroll
+    for (int i = 0; i < 6; ++i) {
+      const int d4 = threadIdx.x + i * blockDim.x;
+      v[i] = d4 < nv ? reinterpret_cast<const float4*>(xr)[d4] : make_float4(0.f, 0.f, 0.f, 0.f);
+      ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
+    }
+    const float inv = rsqrtf(block_sum(ss, red) / float(n) + eps);
+#pragma unroll
+    for (int i = 0; i < 6; ++i) {
+      const int d4 = threadIdx.x + i * blockDim.x;
+      if (d4 < nv) {
+        const float4 g = reinterpret_cast<const float4*>(w)[d4];
+        __half2 lo = __floats2half2_rn(v[i].x * inv * g.x, v[i].y * inv * g.y);
+        __half2 hi = __floats2half2_rn(v[i].z * inv * g.z, v[i].w * inv * g.w);
+        uint2 out;
+        out.x = *reinterpret_cast<uint32_t*>(&lo);
+        out.y = *reinterpret_cast<uint32_t*>(&hi);
+        reinterpret_cast<uint2*>(yr)[d4] = out;
+      }
+    }
+    return;
+  }
   float ss = 0.f;
   for (int d = threadIdx.x; d < n; d += blockDim.x) { const float v = xr[d]; ss += v * v; }
   const float tot = block_sum(ss, red);
   const float inv = rsqrtf(tot / float(n) + eps);
-  __half* yr = y + size_t(blockIdx.x) * n;
   for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = __float2half_rn(xr[d] * inv * w[d]);
 }
 
 // Per (row, head): optional RMSNorm over dh, then rotate-half RoPE at position ctx_len + i.
 // The angle is one fp32 product pos * inv_freq[j]; sin/cos are the accurate library versions.
-// blockIdx.x = row m, blockIdx.y = head index over q heads then k heads then v heads (v is only converted).
+// One warp per (row, head), eight warps per block; heads run over q heads, then k heads, then v heads (v is only
+// converted).
 __global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* __restrict__ qw,
                                     const float* __restrict__ kw, const float* __restrict__ inv_freq,
                                     const int32_t* __restrict__ ctx_lens, __nv_bfloat16* __restrict__ q,
                                     __nv_bfloat16* __restrict__ kb, __nv_bfloat16* __restrict__ vb, int k, int Hq,
-                                    int Hkv, int dh, float eps, int qk_norm) {
-  const int m = blockIdx.x, hh = blockIdx.y;
-  const int lane = threadIdx.x;                       // one warp per (row, head)
+                                    int Hkv, int dh, float eps, int qk_norm, int n_pairs) {
+  const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pair >= n_pairs) return;
+  const int heads = Hq + 2 * Hkv;
+  const int m = pair / heads, hh = pair % heads;
+  const int lane = threadIdx.x & 31;
   const float* src = qkv + size_t(m) * (Hq + 2 * Hkv) * dh + size_t(hh) * dh;
   const int half = dh / 2;
   if (hh >= Hq + Hkv) {                               // values: plain conversion
@@ -146,9 +177,10 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
   if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
   const float* tab = rope_table(theta, dh, stream);
   if (!tab) return cudaErrorMemoryAllocation;
-  dim3 grid(B * k, Hq + 2 * Hkv);
-  qk_norm_rope_kernel<<<grid, 32, 0, stream>>>(qkv, qw, kw, tab, ctx_lens, (__nv_bfloat16*)q, (__nv_bfloat16*)kb,
-                                               (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps, qk_norm);
+  const int n_pairs = B * k * (Hq + 2 * Hkv);
+  qk_norm_rope_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(qkv, qw, kw, tab, ctx_lens, (__nv_bfloat16*)q,
+                                                             (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps,
+                                                             qk_norm, n_pairs);
   return cudaGetLastError();
 }
 

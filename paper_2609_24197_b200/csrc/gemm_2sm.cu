@@ -313,9 +313,10 @@ int g_smem_optin2 = -1;
 
 bool gemm2_preferred(int M, int n_out) {
   static const bool off = [] { const char* e = getenv("HSPEC_GEMM_1SM"); return e && e[0] == '1'; }();
-  if (off || M < 256) return false;
-  const int bnt = gemm2_pick_bnt(M, n_out);
-  return ((n_out + 255) / 256) * ((M + bnt - 1) / bnt) >= 74;
+  // from 256 rows on the contractions are tensor-bound; even a partly filled round of pair tiles beats the one-CTA
+  // kernel with K-slices and its reduction pass
+  (void)n_out;
+  return !off && M >= 256;
 }
 
 // Tile width (activation rows per cluster tile) that wastes the fewest cluster rounds.
