@@ -3,13 +3,14 @@
 // Same decomposition as attention.cu — CTA = (request, KV head, context chunk[, 128-row tile]), partials
 // (m, l, O) per chunk merged afterwards — but both contractions run on the 5th-generation tensor cores:
 //
-//   warp 4      producer: K/V pages -> shared memory.  Full 128-key tiles are 32 TMA boxes (one
+//   warp 8      producer: K/V pages -> shared memory.  Full 128-key tiles are 32 TMA boxes (one
 //               [16 tokens x 64 dh] box per page and head-dim half, 128-byte swizzle: each box is the page's rows
 //               of this KV head exactly as the target stored them).  The ragged end of the context and the block's
 //               own keys/values go through plain 16-byte loads with zero fill, so no garbage row is ever multiplied.
-//   warp 5      issues S = Q K^T (A = Q, B = K tile, both K-major) into one of two TMEM S buffers, then
+//   warp 9      issues S = Q K^T (A = Q, B = K tile, both K-major) into one of two TMEM S buffers, then
 //               O += P V (A = P read from TMEM, B = V tile as an MN-major operand) into the TMEM O buffer.
-//   warps 0..3  softmax: thread = query row = TMEM lane.  Reads its S row (128 fp32), masks by selection, keeps a
+//   warps 0..7  softmax: two threads per query row (= TMEM lane), 64 key columns each; they exchange their half-row
+//               maxima through shared memory.  Each reads its S half-row, masks by selection, keeps a
 //               reference maximum that only moves when the row maximum outgrows it by 2^8 (then, rarely, rescales
 //               its O row in TMEM), writes P (bf16, two keys per 32-bit column) into one of two TMEM P buffers.
 //
@@ -51,7 +52,8 @@ struct __align__(8) AttnTcBars {
   uint64_t s_ready[2], p_ready[2], pv_done[2];
   uint32_t tmem_base;
   uint32_t abort_flag;
-  int32_t pages[256];      // physical page ids of this chunk's full tiles (chunk <= 4096 tokens)
+  __half xmax[2][2][128];  // [tile parity][column half][row]: half-row maxima exchanged between the two threads of a row
+                           // (1 KiB; reused as float [2][128] for the final row-sum exchange)
 };
 
 // byte offset of (row, 16-byte chunk 0..15) inside a [128 x 128] bf16 operand tile stored as two K-major halves
@@ -165,7 +167,7 @@ __device__ __forceinline__ void manual_tile(const Range& g, int mi, int k, int& 
   else { n_prefix = 0; n_block = k; }
 }
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -183,7 +185,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   if (tid == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
-    mbar_init(smem_u32(&bars->q_ready), 128);
+    mbar_init(smem_u32(&bars->q_ready), 8);            // one arrival per softmax warp
     mbar_init(smem_u32(&bars->o_done), 1);
     for (int s = 0; s < NS; ++s) {
       mbar_init(smem_u32(&bars->k_full[s]), 1);
@@ -192,13 +194,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->s_ready[i]), 1);
-      mbar_init(smem_u32(&bars->p_ready[i]), 128);
+      mbar_init(smem_u32(&bars->p_ready[i]), 8);
       mbar_init(smem_u32(&bars->pv_done[i]), 1);
     }
     bars->abort_flag = 0;
     fence_mbar_init();
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tmem_alloc(smem_u32(&bars->tmem_base), 512);
     tmem_relinquish();
   }
@@ -212,13 +214,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   volatile uint32_t* abort_flag = &bars->abort_flag;
   const int row0 = rt * 128;
 
-  if (warp == 4) {
+  if (warp == 8) {
     // ================================================================= producer
     const int32_t* ptab = a.page_table + size_t(b) * a.page_table_stride;
-    // page ids of all full tiles up front: no dependent global load on the per-tile issue path
-    for (int i = lane; i < g.n_full * 8; i += 32) bars->pages[i] = ptab[(g.p_begin >> 4) + i];
-    __syncwarp();
+    // page ids are fetched one tile ahead (lanes 0..7, one page each): no dependent global load on the issue path
+    int page_next = (lane < 8 && g.n_full > 0) ? ptab[(g.p_begin >> 4) + lane] : 0;
     for (int t = 0; t < g.T; ++t) {
+      const int page_cur = page_next;
+      if (lane < 8 && t + 1 < g.n_full) page_next = ptab[(g.p_begin >> 4) + (t + 1) * 8 + lane];
       const int s = t % NS;
       if (t >= NS && !mbar_wait(smem_u32(&bars->kv_empty[s]), ((t / NS) - 1) & 1)) {
         if (lane == 0) { atomicExch(a.status, STATUS_TIMEOUT_PRODUCER); *abort_flag = 1; }
@@ -232,13 +235,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (lane == 0) { mbar_expect_tx(kf, TILE_BYTES); mbar_expect_tx(vf, TILE_BYTES); }
         __syncwarp();
         if (lane < 8) {                                   // one lane per page: K first (the score MMA needs it first)
-          const int page = bars->pages[t * 8 + lane];
+          const int page = page_cur;
           tma_load_4d(smem_u32(dK) + lane * 2048, &tmK, 0, kvh, 0, page, kf);
           tma_load_4d(smem_u32(dK) + HALF_BYTES + lane * 2048, &tmK, 64, kvh, 0, page, kf);
         }
         __syncwarp();
         if (lane < 8) {
-          const int page = bars->pages[t * 8 + lane];
+          const int page = page_cur;
           tma_load_4d(smem_u32(dV) + lane * 2048, &tmV, 0, kvh, 0, page, vf);
           tma_load_4d(smem_u32(dV) + HALF_BYTES + lane * 2048, &tmV, 64, kvh, 0, page, vf);
         }
@@ -283,7 +286,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (lane == 0) { mbar_arrive(smem_u32(&bars->k_full[s])); mbar_arrive(smem_u32(&bars->v_full[s])); }
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ================================================================= MMA issuer
     if (lane == 0) {
       const uint32_t id_qk = idesc_bf16_128x128(false), id_pv = idesc_bf16_128x128(true);
@@ -351,26 +354,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
     }
   } else {
-    // ================================================================= softmax warps: thread = query row
-    const int r_local = tid;                         // TMEM lane
+    // ================================================================= softmax warps: two threads per query row
+    // warps 0..3 own key columns [0, 64) of the tile, warps 4..7 columns [64, 128); warp w reads TMEM lane quarter
+    // w % 4, so threads tid and tid + 128 share a row and exchange their half-row maxima through shared memory.
+    const int r_local = tid & 127;                   // TMEM lane = query row of the tile
+    const int hf = tid >> 7;                         // which half of the key columns
     const int rg = row0 + r_local;                   // row among the k * rep rows of this KV head
     const bool row_ok = rg < a.R;
     const int i_blk = rg / a.rep;                    // block position of the row
-    {   // Q row -> shared memory (zeros for padding rows)
+    {   // Q row -> shared memory (zeros for padding rows): each thread of the pair writes one head-dim half
       const __nv_bfloat16* src = a.q + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH;
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch) {
+      for (int c8 = 0; c8 < 8; ++c8) {
+        const int ch = hf * 8 + c8;
         const uint4 v = row_ok ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0, 0, 0, 0);
         *reinterpret_cast<uint4*>(sQ + tile_off(r_local, ch)) = v;
       }
       fence_proxy_async();
-      mbar_arrive(smem_u32(&bars->q_ready));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
     }
-    const uint32_t lane_base = uint32_t(warp * 32) << 16;
+    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
     float m_ref = NEG, l_sum = 0.f;
     bool ok = true;
 #ifdef HSPEC_ATTN_TIMING
-    long long t_wait_s = 0, t_wait_pv = 0, t_start = clock64(), t_mark;
+    long long t_wait_s = 0, t_wait_pv = 0, t_start = clock64(), t_mark, t_ld = 0, t_bar = 0, t_exp = 0, t_st = 0;
 #endif
     for (int t = 0; t < g.T && ok; ++t) {
 #ifdef HSPEC_ATTN_TIMING
@@ -381,27 +389,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       t_wait_s += clock64() - t_mark;
 #endif
       tc_fence_after();
-      float s[KT];
+#ifdef HSPEC_ATTN_TIMING
+      t_mark = clock64();
+#endif
+      float s[64];
+      const int col0 = hf * 64;                      // first key column of this thread
 #pragma unroll
-      for (int j = 0; j < KT / 32; ++j) tmem_ld32(tmem_s0 + (t & 1) * 128 + lane_base + j * 32, reinterpret_cast<uint32_t*>(s + j * 32));
+      for (int j = 0; j < 2; ++j) tmem_ld32(tmem_s0 + (t & 1) * 128 + lane_base + col0 + j * 32, reinterpret_cast<uint32_t*>(s + j * 32));
       tmem_ld_wait();
+#ifdef HSPEC_ATTN_TIMING
+      t_ld += clock64() - t_mark; t_mark = clock64();
+#endif
       // ---- mask by selection (raw scores; the positive scale is folded into the exponent below)
       if (t < g.n_full) {
-        const int key0 = g.p_begin + t * KT;
+        const int key0 = g.p_begin + t * KT + col0;
         if (a.window > 0 && key0 < g.base + 16 + a.k) {                   // leading edge of the window
 #pragma unroll
-          for (int j = 0; j < KT; ++j)
+          for (int j = 0; j < 64; ++j)
             if ((ctx + i_blk) - (key0 + j) >= a.window) s[j] = -INFINITY;
         }
       } else {
         int n_prefix, prefix_start, n_block;
         manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
 #pragma unroll
-        for (int j = 0; j < KT; ++j) {
+        for (int j = 0; j < 64; ++j) {
+          const int col = col0 + j;
           bool vis;
-          if (j < n_prefix) vis = a.window <= 0 || (ctx + i_blk) - (prefix_start + j) < a.window;
+          if (col < n_prefix) vis = a.window <= 0 || (ctx + i_blk) - (prefix_start + col) < a.window;
           else {
-            const int jb = j - n_prefix;
+            const int jb = col - n_prefix;
             vis = jb < n_block && jb <= i_blk && (a.window <= 0 || i_blk - jb < a.window);
           }
           if (!vis) s[j] = -INFINITY;
@@ -409,32 +425,40 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};         // four chains instead of one
 #pragma unroll
-      for (int j = 0; j < KT; j += 4) {
+      for (int j = 0; j < 64; j += 4) {
         mx4[0] = fmaxf(mx4[0], s[j]); mx4[1] = fmaxf(mx4[1], s[j + 1]);
         mx4[2] = fmaxf(mx4[2], s[j + 2]); mx4[3] = fmaxf(mx4[3], s[j + 3]);
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-      // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY
+      // exchanged as fp16 (rounded UP, so the reference never undershoots): both threads of the row then hold the
+      // same two values and take the same decision; the reference maximum need not be the exact maximum
+      const __half mx_own = __float2half_ru(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+      bars->xmax[t & 1][hf][r_local] = mx_own;
+      asm volatile("bar.sync 1, 256;" ::: "memory");                        // the eight softmax warps
+      const float mx = fmaxf(__half2float(mx_own), __half2float(bars->xmax[t & 1][hf ^ 1][r_local])) * a.scale_log2;
+#ifdef HSPEC_ATTN_TIMING
+      t_bar += clock64() - t_mark;
+#endif
+      // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY (same decision in both halves)
       float factor = 1.f;
       const bool grow = mx > m_ref + LAZY;
       if (grow) { factor = ex2_ftz(m_ref - mx); m_ref = mx; }
       if (t > 0 && __any_sync(0xffffffffu, grow)) {
-        // O of the tiles so far must be complete before it is rescaled
+        // O of the tiles so far must be complete before it is rescaled; each thread rescales its 64 columns
         if (!mbar_wait(smem_u32(&bars->pv_done[(t - 1) & 1]), ((t - 1) >> 1) & 1)) { ok = false; break; }
         tc_fence_after();
 #pragma unroll
-        for (int j = 0; j < DH / 32; ++j) {
+        for (int j = 0; j < 2; ++j) {
           uint32_t o[32];
-          tmem_ld32(tmem_o + lane_base + j * 32, o);
+          tmem_ld32(tmem_o + lane_base + col0 + j * 32, o);
           tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-          tmem_st32(tmem_o + lane_base + j * 32, o);
+          tmem_st32(tmem_o + lane_base + col0 + j * 32, o);
         }
         tmem_st_wait();
       }
       l_sum *= factor;
-      // ---- P = exp2(s - m_ref) -> bf16 -> shared memory (K-major swizzled A operand of the PV MMA)
+      // ---- P = exp2(s - m_ref) -> bf16 pairs -> this thread's half of the TMEM P buffer
 #ifdef HSPEC_ATTN_TIMING
       t_mark = clock64();
 #endif
@@ -442,40 +466,52 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #ifdef HSPEC_ATTN_TIMING
       t_wait_pv += clock64() - t_mark;
 #endif
+#ifdef HSPEC_ATTN_TIMING
+      t_mark = clock64();
+#endif
       const float neg_m = -m_ref;
       float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t w[32];
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {                 // 64 keys = 32 packed columns per TMEM store
-        uint32_t w[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          const float p0 = ex2_ftz(fmaf(s[hh * 64 + 2 * e], a.scale_log2, neg_m));
-          const float p1 = ex2_ftz(fmaf(s[hh * 64 + 2 * e + 1], a.scale_log2, neg_m));
-          ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
-          w[e] = pack_bf16(p0, p1);
-        }
-        tmem_st32(tmem_p0 + (t & 1) * 64 + lane_base + hh * 32, w);
+      for (int e = 0; e < 32; ++e) {
+        const float p0 = ex2_ftz(fmaf(s[2 * e], a.scale_log2, neg_m));
+        const float p1 = ex2_ftz(fmaf(s[2 * e + 1], a.scale_log2, neg_m));
+        ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
+        w[e] = pack_bf16(p0, p1);
       }
+#ifdef HSPEC_ATTN_TIMING
+      t_exp += clock64() - t_mark; t_mark = clock64();
+#endif
+      tmem_st32(tmem_p0 + (t & 1) * 64 + lane_base + hf * 32, w);
       l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
       tmem_st_wait();
+#ifdef HSPEC_ATTN_TIMING
+      t_st += clock64() - t_mark;
+#endif
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars->p_ready[t & 1]));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->p_ready[t & 1]));   // one arrival per warp, after all its lanes' stores
     }
 #ifdef HSPEC_ATTN_TIMING
     if (tid == 0 && (blockIdx.x + blockIdx.y * 7 + blockIdx.z * 13) % 97 == 0)
-      printf("attn cta (%d,%d,%d): T=%d total=%lld wait_s=%lld wait_pv=%lld clocks\n", blockIdx.x, blockIdx.y, blockIdx.z, g.T,
-             clock64() - t_start, t_wait_s, t_wait_pv);
+      printf("attn cta (%d,%d,%d): T=%d total=%lld wait_s=%lld wait_pv=%lld ld=%lld max+bar=%lld exp=%lld st=%lld clocks\n", blockIdx.x, blockIdx.y,
+             blockIdx.z, g.T, clock64() - t_start, t_wait_s, t_wait_pv, t_ld, t_bar, t_exp, t_st);
 #endif
     if (!ok) { atomicExch(a.status, STATUS_TIMEOUT_EPILOGUE); *abort_flag = 1; }
-    // ---- partial (m, l, O) of this chunk
+    // ---- partial (m, l, O) of this chunk: the row sum is the sum of the two halves
+    float* xl = reinterpret_cast<float*>(&bars->xmax[0][0][0]);            // [2][128] floats
+    asm volatile("bar.sync 1, 256;" ::: "memory");                          // everyone is done with the maxima
+    xl[hf * 128 + r_local] = l_sum;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const float l_row = l_sum + xl[(hf ^ 1) * 128 + r_local];
     if (ok && mbar_wait(smem_u32(&bars->o_done), 0) && !*abort_flag) {
       tc_fence_after();
       const size_t slab = (size_t(b) * a.Hkv + kvh) * a.max_chunks + c;
-      float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH;
+      float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH + hf * 64;
 #pragma unroll
-      for (int j = 0; j < DH / 32; ++j) {
+      for (int j = 0; j < 2; ++j) {
         uint32_t o[32];
-        tmem_ld32(tmem_o + lane_base + j * 32, o);
+        tmem_ld32(tmem_o + lane_base + hf * 64 + j * 32, o);
         tmem_ld_wait();
         if (row_ok) {
 #pragma unroll
@@ -483,16 +519,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             *reinterpret_cast<uint4*>(dst + j * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
         }
       }
-      if (row_ok) {
+      if (row_ok && hf == 0) {
         float* ml = a.ws_ml + (slab * a.R + rg) * 2;
         ml[0] = (m_ref == NEG) ? -INFINITY : m_ref;
-        ml[1] = l_sum;
+        ml[1] = l_row;
       }
     }
     tc_fence_before();
   }
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after();
     tmem_dealloc(tmem, 512);
   }
@@ -589,7 +625,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   }
   dim3 grid(max_chunks * a.n_row_tiles, c.Hkv, c.B);
   trk_begin(trk, "attn_partial");
-  attn_tc_kernel<<<grid, 192, smem, stream>>>(tmK, tmV, a);
+  attn_tc_kernel<<<grid, 320, smem, stream>>>(tmK, tmV, a);
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
