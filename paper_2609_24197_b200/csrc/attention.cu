@@ -285,7 +285,10 @@ int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms) {
   int chunk = (lmax + nsplit - 1) / nsplit;
   chunk = ((chunk + 127) / 128) * 128;
   if (chunk < 256) chunk = 256;
-  if (chunk > 4096) chunk = 4096;
+  // long chunks mean fewer partials to write and merge; they need enough (request, head) pairs to keep every SM's
+  // share of the work list even
+  const int cap = (B * Hkv >= 4 * num_sms) ? 8192 : 4096;
+  if (chunk > cap) chunk = cap;
   return chunk;
 }
 
@@ -299,7 +302,8 @@ static int max_chunks_of(int max_ctx, int window, int chunk) {
 size_t attn_workspace_bytes(int B, int k, int Hq, int Hkv, int dh, int max_ctx, int window, int chunk_tokens) {
   const int R = k * (Hq / Hkv);
   const size_t slabs = size_t(B) * Hkv * max_chunks_of(max_ctx, window, chunk_tokens);
-  return slabs * R * (dh + 2) * sizeof(float) + 256;
+  const size_t row_tiles = (size_t(R) + 127) / 128;
+  return slabs * R * (dh + 2) * sizeof(float) + 256 + slabs * row_tiles * 16 + 64;   // partials + the tcgen05 path's work list
 }
 
 cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {

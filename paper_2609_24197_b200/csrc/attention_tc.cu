@@ -1,21 +1,27 @@
 // Block-query GQA attention over the target's paged KV, tcgen05 version (dh = 128, 16-token pages).
 //
-// Same decomposition as attention.cu — CTA = (request, KV head, context chunk[, 128-row tile]), partials
-// (m, l, O) per chunk merged afterwards — but both contractions run on the 5th-generation tensor cores:
+// Same decomposition as attention.cu — work item = (request, KV head, context chunk[, 128-row tile]), partials
+// (m, l, O) per chunk merged afterwards — but both contractions run on the 5th-generation tensor cores, and the
+// kernel is persistent: a small plan kernel writes the work list (longest items first), one CTA per SM walks it.
 //
-//   warp 8      producer: K/V pages -> shared memory.  Full 128-key tiles are 32 TMA boxes (one
-//               [16 tokens x 64 dh] box per page and head-dim half, 128-byte swizzle: each box is the page's rows
-//               of this KV head exactly as the target stored them).  The ragged end of the context and the block's
-//               own keys/values go through plain 16-byte loads with zero fill, so no garbage row is ever multiplied.
-//   warp 9      issues S = Q K^T (A = Q, B = K tile, both K-major) into one of two TMEM S buffers, then
-//               O += P V (A = P read from TMEM, B = V tile as an MN-major operand) into the TMEM O buffer.
+//   warp 8      K producer, warp 10 V producer: pages -> their own rings of 32 KiB slots in shared memory (3 + 3
+//               slots).  Full 128-key tiles are 16 TMA boxes per operand (one [16 tokens x 64 dh] box per page and
+//               head-dim half, 128-byte swizzle: each box is the page's rows of this KV head exactly as the target
+//               stored them).  The ragged end of the context and the block's own keys/values go through plain
+//               16-byte loads with zero fill, so no garbage row is ever multiplied.  A K slot is released as soon as
+//               the tile's scores are computed, a V slot after the P V product; both producers run on into the next
+//               work item, so HBM keeps streaming while an item's result is read out.
+//   warp 9      issues S = Q K^T (A = Q from shared memory, B = K tile, both K-major) into one of two TMEM S buffers,
+//               then O += P V (A = P read from TMEM, B = V tile as an MN-major operand) into the TMEM O buffer.
 //   warps 0..7  softmax: two threads per query row (= TMEM lane), 64 key columns each; they exchange their half-row
 //               maxima through shared memory.  Each reads its S half-row, masks by selection, keeps a
 //               reference maximum that only moves when the row maximum outgrows it by 2^8 (then, rarely, rescales
-//               its O row in TMEM), writes P (bf16, two keys per 32-bit column) into one of two TMEM P buffers.
+//               its O row in TMEM), and writes P (bf16, two keys per 32-bit column) over the first half of the S
+//               buffer it came from.  At the end of an item they put the next item's Q tile into shared memory
+//               first (the tensor core starts on its scores), then read O out.
 //
 // The MMA warp issues S_{t+1} before it waits for P_t, so the tensor core works on the next tile's scores while
-// the softmax warps are busy, and the producer runs NS tiles ahead.  Every wait is bounded.
+// the softmax warps are busy.  Every wait is bounded; a timed-out role sets a status word and the CTA unwinds.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -27,9 +33,9 @@ namespace {
 
 constexpr int KT = 128;            // keys per tile
 constexpr int DH = 128;
-constexpr int NS = 3;              // K/V stages in shared memory
-constexpr int HALF_BYTES = 128 * 128;            // [128 rows x 64 bf16] = 16 KiB
-constexpr int TILE_BYTES = 2 * HALF_BYTES;       // one operand tile [128 x 128] bf16
+constexpr int NSK = 3, NSV = 3;    // slots of the K ring and of the V ring (7 x 32 KiB = all of shared memory)
+constexpr int KV_HALF = KT * 128;                // K or V tile: [128 keys x 64 bf16] = 16 KiB per head-dim half
+constexpr int KV_BYTES = 2 * KV_HALF;            // one K or V tile [128 keys x 128 dh] bf16 = 32 KiB
 constexpr float NEG = -1.0e30f;
 constexpr float LAZY = 8.0f;       // rescale only when the row maximum exceeds the reference by 2^8
 
@@ -47,19 +53,21 @@ struct AttnTcArgs {
 };
 
 struct __align__(8) AttnTcBars {
-  uint64_t q_ready, o_done;
-  uint64_t k_full[NS], v_full[NS], kv_empty[NS];
-  uint64_t s_ready[2], p_ready[2], pv_done[2];
+  uint64_t q_ready, o_done, o_free, l_ready;
+  uint64_t x_ready[2];
+  uint64_t k_full[NSK], k_empty[NSK], v_full[NSV], v_empty[NSV];
+  uint64_t s_ready[2], p_ready[2];
   uint32_t tmem_base;
   uint32_t abort_flag;
   __half xmax[2][2][128];  // [tile parity][column half][row]: half-row maxima exchanged between the two threads of a row
-                           // (1 KiB; reused as float [2][128] for the final row-sum exchange)
+                           // (1 KiB; one parity's 512 bytes are reused as a float per row for the final row-sum exchange)
 };
 
 // byte offset of (row, 16-byte chunk 0..15) inside a [128 x 128] bf16 operand tile stored as two K-major halves
 // with the 128-byte swizzle (the layout TMA writes and the UMMA descriptors read)
+template <int HALF>
 __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
-  return uint32_t((chunk >> 3) * HALF_BYTES + (row >> 3) * 1024 + (row & 7) * 128 + (((chunk & 7) ^ (row & 7)) << 4));
+  return uint32_t((chunk >> 3) * HALF + (row >> 3) * 1024 + (row & 7) * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
 // adds to the barrier's expected byte count without arriving on it
@@ -79,7 +87,7 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int 
 __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr) {
   uint64_t d = 0;
   d |= uint64_t((smem_addr & 0x3FFFF) >> 4);
-  d |= uint64_t(HALF_BYTES >> 4) << 16;
+  d |= uint64_t(KV_HALF >> 4) << 16;
   d |= uint64_t(1024 >> 4) << 32;
   d |= uint64_t(1) << 46;
   d |= uint64_t(2) << 61;
@@ -106,6 +114,17 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
         "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
+}
+// Waits for the outstanding tensor-memory loads; the 32 destination registers are operands, so no use of them can be
+// scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_wait_ld32(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]), "+r"(r[16]),
+                 "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]),
+                 "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 // 2^x by the special-function unit alone (flush-to-zero form: no range fix-up code around it)
 __device__ __forceinline__ float ex2_ftz(float x) {
@@ -167,35 +186,161 @@ __device__ __forceinline__ void manual_tile(const Range& g, int mi, int k, int& 
   else { n_prefix = 0; n_block = k; }
 }
 
-__global__ void __launch_bounds__(320, 1)
-attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a) {
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sQ = smem;                               // 32 KiB
-  uint8_t* sKV = sQ + TILE_BYTES;                   // NS x (K 32 KiB + V 32 KiB)
-  AttnTcBars* bars = reinterpret_cast<AttnTcBars*>(sKV + NS * 2 * TILE_BYTES);
+// Work item = (request, KV head, context chunk, 128-row tile); x = request, y = KV head | row tile << 16, z = chunk,
+// w = the request's context length (so that one 16-byte load tells a role everything about the item).
+struct Item { int b, kvh, rt, c, ctx; };
+__device__ __forceinline__ Item unpack_item(const int4 w) {
+  Item it;
+  it.b = w.x; it.kvh = w.y & 0xffff; it.rt = w.y >> 16; it.c = w.z; it.ctx = w.w;
+  return it;
+}
+
+// Work list: one item per (request, KV head, context chunk, 128-row tile), longest first (bucketed by tile count),
+// heads of one request and chunk next to each other so the CTAs that run them at the same time read neighbouring
+// bytes of the same pages.  The order inside a bucket depends on atomics; every item is computed independently, so
+// results do not.
+__global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4* __restrict__ items) {
+  __shared__ int bucket[64];
+  __shared__ int offset[64];
+  const int per_chunk = a.Hkv * a.n_row_tiles;
+  for (int i = threadIdx.x; i < 64; i += blockDim.x) bucket[i] = 0;
+  __syncthreads();
+  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+    const int ctx = a.ctx_lens[b];
+    const int n_chunks = make_range(ctx, a.window, a.chunk, 0, a.k).n_chunks;
+    for (int c = 0; c < n_chunks; ++c) atomicAdd(&bucket[min(make_range(ctx, a.window, a.chunk, c, a.k).T, 63)], per_chunk);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int off = 0;
+    for (int T = 63; T >= 0; --T) { offset[T] = off; off += bucket[T]; }
+    *count = off;
+  }
+  __syncthreads();
+  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+    const int ctx = a.ctx_lens[b];
+    const int n_chunks = make_range(ctx, a.window, a.chunk, 0, a.k).n_chunks;
+    for (int c = 0; c < n_chunks; ++c) {
+      int at = atomicAdd(&offset[min(make_range(ctx, a.window, a.chunk, c, a.k).T, 63)], per_chunk);
+      for (int kvh = 0; kvh < a.Hkv; ++kvh)
+        for (int rt = 0; rt < a.n_row_tiles; ++rt) items[at++] = make_int4(b, kvh | (rt << 16), c, ctx);
+    }
+  }
+}
+
+// One operand (K or V) of every tile of this CTA's items -> its own ring of 32 KiB slots.  K and V have separate
+// rings and separate producer warps because their slots are released at different times (K once the tile's scores
+// are computed, V only after the softmax of the tile and the P V product), and a single in-order producer would
+// hold the next K loads back behind a V slot that is still in use.
+//   Full 128-key tiles are 16 TMA boxes (one [16 tokens x 64 dh] box per page and head-dim half, 128-byte swizzle).
+//   The ragged end of the prefix and the block's own rows: whole pages still by TMA, the rest through 16-byte
+//   cp.async with zero fill for every unused row, so nothing that is not a real key or value is ever multiplied.
+__device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUtensorMap* tm, const __nv_bfloat16* pool,
+                                                const __nv_bfloat16* blk, uint8_t* ring, uint64_t* full, uint64_t* empty,
+                                                volatile uint32_t* abort_flag, const int4* __restrict__ items, int n_items,
+                                                int lane, int ns) {
+  uint32_t gt = 0;                                 // tiles issued so far, across items
+  int4 w_next = items[blockIdx.x];
+  for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
+    const Item wi = unpack_item(w_next);
+    if (it + int(gridDim.x) < n_items) w_next = items[it + gridDim.x];     // consumed one item later
+    const int b = wi.b, kvh = wi.kvh;
+    const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
+    const int32_t* ptab = a.page_table + size_t(b) * a.page_table_stride;
+    // page ids are fetched one tile ahead (lanes 0..3, one page each): no dependent global load on the issue path
+    int page_next = (lane < KT / 16 && g.n_full > 0) ? ptab[(g.p_begin >> 4) + lane] : 0;
+    for (int t = 0; t < g.T; ++t, ++gt) {
+      const int page_cur = page_next;
+      if (lane < KT / 16 && t + 1 < g.n_full) page_next = ptab[(g.p_begin >> 4) + (t + 1) * (KT / 16) + lane];
+      const int s = gt % ns;
+      if (gt >= uint32_t(ns) && !mbar_wait(smem_u32(&empty[s]), ((gt / ns) - 1) & 1)) {
+        if (lane == 0) { atomicExch(a.status, STATUS_TIMEOUT_PRODUCER); *abort_flag = 1; }
+        return;
+      }
+      if (*abort_flag) return;
+      uint8_t* dst = ring + s * KV_BYTES;
+      const uint32_t bar = smem_u32(&full[s]);
+      if (t < g.n_full) {
+        if (lane == 0) mbar_expect_tx(bar, KV_BYTES);
+        __syncwarp();
+        if (lane < KT / 16) {
+          tma_load_4d(smem_u32(dst) + lane * 2048, tm, 0, kvh, 0, page_cur, bar);
+          tma_load_4d(smem_u32(dst) + KV_HALF + lane * 2048, tm, 64, kvh, 0, page_cur, bar);
+        }
+      } else {
+        int n_prefix, prefix_start, n_block;
+        manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
+        const int full_pages = n_prefix >> 4;
+        const int tma_rows = full_pages << 4;
+        if (lane == 0 && full_pages > 0) mbar_expect_tx_only(bar, full_pages * 4096);
+        __syncwarp();
+        if (lane < full_pages) {
+          const int page = ptab[(prefix_start >> 4) + lane];
+          tma_load_4d(smem_u32(dst) + lane * 2048, tm, 0, kvh, 0, page, bar);
+          tma_load_4d(smem_u32(dst) + KV_HALF + lane * 2048, tm, 64, kvh, 0, page, bar);
+        }
+        for (int idx = lane; idx < (KT - tma_rows) * 16; idx += 32) {
+          const int r = tma_rows + (idx >> 4), chunk16 = idx & 15;
+          const bool valid = r < n_prefix + n_block;
+          size_t off = 0;
+          const __nv_bfloat16* src = pool;
+          if (r < n_prefix) {
+            const int p = prefix_start + r;
+            const int page = ptab[p >> 4];
+            off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
+          } else if (valid) {
+            src = blk;
+            off = ((size_t(b) * a.k + (r - n_prefix)) * a.Hkv + kvh) * DH + chunk16 * 8;
+          }
+          cp_async16(smem_u32(dst) + tile_off<KV_HALF>(r, chunk16), src + off, valid);
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar);
+      }
+    }
+  }
+}
+
+// Persistent: one CTA per SM walks the work list (item = blockIdx.x, + gridDim.x, ...).  All ring and buffer indices
+// count tiles across items (gt): K slot = gt % NSK, V slot = gt % NSV, S / P buffer = gt & 1.
+__global__ void __launch_bounds__(352, 1)
+attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a,
+               const int* __restrict__ count, const int4* __restrict__ items) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  uint8_t* sQ = smem;                               // Q tile, 32 KiB
+  uint8_t* sKV = smem + KV_BYTES;                   // K ring (NSK x 32 KiB), then V ring (NSV x 32 KiB)
+  AttnTcBars* bars = reinterpret_cast<AttnTcBars*>(sKV + (NSK + NSV) * KV_BYTES);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int b = blockIdx.z, kvh = blockIdx.y;
-  const int c = blockIdx.x / a.n_row_tiles, rt = blockIdx.x % a.n_row_tiles;
-  const int ctx = a.ctx_lens[b];
-  const Range g = make_range(ctx, a.window, a.chunk, c, a.k);
-  if (c >= g.n_chunks) return;                      // uniform for the whole CTA
+  const int n_items = *count;
+  if (int(blockIdx.x) >= n_items) return;           // uniform for the whole CTA
+  if (smem_u32(smem) & 1023) {                      // the swizzled operand tiles need a 1 KiB-aligned base
+    if (tid == 0) atomicExch(a.status, STATUS_BAD_SMEM_BASE);
+    return;
+  }
 
   if (tid == 0) {
     tma_prefetch_desc(&tmK);
     tma_prefetch_desc(&tmV);
     mbar_init(smem_u32(&bars->q_ready), 8);            // one arrival per softmax warp
+    mbar_init(smem_u32(&bars->o_free), 8);
+    mbar_init(smem_u32(&bars->l_ready), 4);            // the four warps that own the upper column half
     mbar_init(smem_u32(&bars->o_done), 1);
-    for (int s = 0; s < NS; ++s) {
+    for (int s = 0; s < NSK; ++s) {
       mbar_init(smem_u32(&bars->k_full[s]), 1);
+      mbar_init(smem_u32(&bars->k_empty[s]), 1);
+    }
+    for (int s = 0; s < NSV; ++s) {
       mbar_init(smem_u32(&bars->v_full[s]), 1);
-      mbar_init(smem_u32(&bars->kv_empty[s]), 1);
+      mbar_init(smem_u32(&bars->v_empty[s]), 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->s_ready[i]), 1);
       mbar_init(smem_u32(&bars->p_ready[i]), 8);
-      mbar_init(smem_u32(&bars->pv_done[i]), 1);
+      mbar_init(smem_u32(&bars->x_ready[i]), 8);
     }
     bars->abort_flag = 0;
     fence_mbar_init();
@@ -208,146 +353,92 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = bars->tmem_base;
-  const uint32_t tmem_o = tmem;                     // columns [0, 128)
-  const uint32_t tmem_s0 = tmem + 128;              // S buffers: columns [128, 256) and [256, 384)
-  const uint32_t tmem_p0 = tmem + 384;              // P buffers (bf16 pairs): columns [384, 448) and [448, 512)
+  // tensor memory: O in columns [0, 128), two S buffers in [128, 256) and [256, 384); P (bf16 pairs, 64 columns)
+  // overwrites the first half of the S buffer it was computed from
+  const uint32_t tmem_o = tmem, tmem_s0 = tmem + 128;
   volatile uint32_t* abort_flag = &bars->abort_flag;
-  const int row0 = rt * 128;
 
-  if (warp == 8) {
-    // ================================================================= producer
-    const int32_t* ptab = a.page_table + size_t(b) * a.page_table_stride;
-    // page ids are fetched one tile ahead (lanes 0..7, one page each): no dependent global load on the issue path
-    int page_next = (lane < 8 && g.n_full > 0) ? ptab[(g.p_begin >> 4) + lane] : 0;
-    for (int t = 0; t < g.T; ++t) {
-      const int page_cur = page_next;
-      if (lane < 8 && t + 1 < g.n_full) page_next = ptab[(g.p_begin >> 4) + (t + 1) * 8 + lane];
-      const int s = t % NS;
-      if (t >= NS && !mbar_wait(smem_u32(&bars->kv_empty[s]), ((t / NS) - 1) & 1)) {
-        if (lane == 0) { atomicExch(a.status, STATUS_TIMEOUT_PRODUCER); *abort_flag = 1; }
-        break;
-      }
-      if (*abort_flag) break;
-      uint8_t* dK = sKV + s * 2 * TILE_BYTES;
-      uint8_t* dV = dK + TILE_BYTES;
-      if (t < g.n_full) {
-        const uint32_t kf = smem_u32(&bars->k_full[s]), vf = smem_u32(&bars->v_full[s]);
-        if (lane == 0) { mbar_expect_tx(kf, TILE_BYTES); mbar_expect_tx(vf, TILE_BYTES); }
-        __syncwarp();
-        if (lane < 8) {                                   // one lane per page: K first (the score MMA needs it first)
-          const int page = page_cur;
-          tma_load_4d(smem_u32(dK) + lane * 2048, &tmK, 0, kvh, 0, page, kf);
-          tma_load_4d(smem_u32(dK) + HALF_BYTES + lane * 2048, &tmK, 64, kvh, 0, page, kf);
-        }
-        __syncwarp();
-        if (lane < 8) {
-          const int page = page_cur;
-          tma_load_4d(smem_u32(dV) + lane * 2048, &tmV, 0, kvh, 0, page, vf);
-          tma_load_4d(smem_u32(dV) + HALF_BYTES + lane * 2048, &tmV, 64, kvh, 0, page, vf);
-        }
-      } else {
-        // ragged end of the prefix and / or the block's own keys.  Whole pages of the ragged end still come by
-        // TMA; the last partial page and the block rows come through cp.async (zero fill for every unused row,
-        // so nothing that is not a real key or value is ever multiplied).
-        int n_prefix, prefix_start, n_block;
-        manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
-        const int full_pages = n_prefix >> 4;
-        const int tma_rows = full_pages << 4;
-        const uint32_t kf = smem_u32(&bars->k_full[s]), vf = smem_u32(&bars->v_full[s]);
-        if (lane == 0 && full_pages > 0) { mbar_expect_tx_only(kf, full_pages * 4096); mbar_expect_tx_only(vf, full_pages * 4096); }
-        __syncwarp();
-        if (lane < full_pages) {
-          const int page = ptab[(prefix_start >> 4) + lane];
-          tma_load_4d(smem_u32(dK) + lane * 2048, &tmK, 0, kvh, 0, page, kf);
-          tma_load_4d(smem_u32(dK) + HALF_BYTES + lane * 2048, &tmK, 64, kvh, 0, page, kf);
-          tma_load_4d(smem_u32(dV) + lane * 2048, &tmV, 0, kvh, 0, page, vf);
-          tma_load_4d(smem_u32(dV) + HALF_BYTES + lane * 2048, &tmV, 64, kvh, 0, page, vf);
-        }
-        for (int idx = lane; idx < (KT - tma_rows) * 16; idx += 32) {
-          const int r = tma_rows + (idx >> 4), chunk16 = idx & 15;
-          const bool valid = r < n_prefix + n_block;
-          size_t off = 0;
-          const __nv_bfloat16 *srcK = a.k_pool, *srcV = a.v_pool;
-          if (r < n_prefix) {
-            const int p = prefix_start + r;
-            const int page = ptab[p >> 4];
-            off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
-          } else if (valid) {
-            srcK = a.kb; srcV = a.vb;
-            off = ((size_t(b) * a.k + (r - n_prefix)) * a.Hkv + kvh) * DH + chunk16 * 8;
-          }
-          cp_async16(smem_u32(dK) + tile_off(r, chunk16), srcK + off, valid);
-          cp_async16(smem_u32(dV) + tile_off(r, chunk16), srcV + off, valid);
-        }
-        cp_async_commit();
-        cp_async_wait<0>();
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) { mbar_arrive(smem_u32(&bars->k_full[s])); mbar_arrive(smem_u32(&bars->v_full[s])); }
-      }
-    }
+  if (warp == 8 || warp == 10) {
+    // ================================================================= producers: warp 8 streams K, warp 10 streams V
+    const bool is_v = warp == 10;
+    produce_operand(a, is_v ? &tmV : &tmK, is_v ? a.v_pool : a.k_pool, is_v ? a.vb : a.kb, sKV + (is_v ? NSK * KV_BYTES : 0),
+                    is_v ? bars->v_full : bars->k_full, is_v ? bars->v_empty : bars->k_empty, abort_flag, items, n_items, lane,
+                    is_v ? NSV : NSK);
   } else if (warp == 9) {
     // ================================================================= MMA issuer
     if (lane == 0) {
+      // fp32 accumulate, bf16 x bf16, M = 128, N = 128; scores: A = Q, B = K tile, both K-major in shared memory;
+      // P V: A = P from tensor memory, B = V tile (MN-major)
       const uint32_t id_qk = idesc_bf16_128x128(false), id_pv = idesc_bf16_128x128(true);
-      bool ok = mbar_wait(smem_u32(&bars->q_ready), 0);
+      uint32_t gt = 0, n = 0;                        // tiles and items done so far
+      bool ok = true;
 #ifdef HSPEC_ATTN_TIMING
-      long long w_k = 0, w_p = 0, w_v = 0, m0;
+      long long mk[8] = {0, 0, 0, 0, 0, 0, 0, 0}, m_last = clock64(), m_start = m_last;
+#define MCLK(i) { const long long t_now = clock64(); mk[i] += t_now - m_last; m_last = t_now; }
+#else
+#define MCLK(i)
 #endif
-      auto issue_s = [&](int t) -> bool {
-        const int s = t % NS;
-#ifdef HSPEC_ATTN_TIMING
-        m0 = clock64();
-#endif
-        if (!mbar_wait(smem_u32(&bars->k_full[s]), (t / NS) & 1)) return false;
-#ifdef HSPEC_ATTN_TIMING
-        w_k += clock64() - m0;
-#endif
+      // S = Q K^T of tile g_t into S buffer g_t & 1.  The buffer last held P of tile g_t - 2, whose P V product this
+      // thread issued earlier; the tensor pipe runs one thread's MMAs in issue order.
+      auto issue_s = [&](uint32_t g_t) -> bool {
+        const int s = g_t % NSK;
+        MCLK(0)
+        if (!mbar_wait(smem_u32(&bars->k_full[s]), (g_t / NSK) & 1)) return false;
+        MCLK(1)
         tc_fence_after();
-        const uint32_t kbase = smem_u32(sKV + s * 2 * TILE_BYTES);
-        const uint32_t qbase = smem_u32(sQ);
+        const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks) {
-          const uint64_t da = umma_desc_kmajor_sw128(qbase + (ks >> 2) * HALF_BYTES) + uint64_t((ks & 3) * 2);
-          const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * HALF_BYTES) + uint64_t((ks & 3) * 2);
-          umma_bf16(tmem_s0 + (t & 1) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
+          const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+          const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+          umma_bf16(tmem_s0 + (g_t & 1) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
         }
-        umma_commit(smem_u32(&bars->s_ready[t & 1]));
+        umma_commit(smem_u32(&bars->k_empty[s]));
+        umma_commit(smem_u32(&bars->s_ready[g_t & 1]));
         return true;
       };
-      if (ok) ok = issue_s(0);
-      for (int t = 0; t < g.T && ok; ++t) {
-        if (t + 1 < g.T) ok = issue_s(t + 1);
-        if (!ok) break;
-        const int s = t % NS;
-#ifdef HSPEC_ATTN_TIMING
-        m0 = clock64();
-#endif
-        if (!mbar_wait(smem_u32(&bars->p_ready[t & 1]), (t >> 1) & 1)) { ok = false; break; }
-#ifdef HSPEC_ATTN_TIMING
-        w_p += clock64() - m0; m0 = clock64();
-#endif
-        if (!mbar_wait(smem_u32(&bars->v_full[s]), (t / NS) & 1)) { ok = false; break; }
-#ifdef HSPEC_ATTN_TIMING
-        w_v += clock64() - m0;
-#endif
+      int4 w_next = items[blockIdx.x];
+      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n) {
+        const Item wi = unpack_item(w_next);
+        if (it + int(gridDim.x) < n_items) w_next = items[it + gridDim.x];
+        const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
+        MCLK(0)
+        if (!mbar_wait(smem_u32(&bars->q_ready), n & 1)) { ok = false; break; }      // this item's Q tile is in place
+        MCLK(4)
         tc_fence_after();
-        const uint32_t vbase = smem_u32(sKV + s * 2 * TILE_BYTES + TILE_BYTES);
+        ok = issue_s(gt);
+        for (int t = 0; t < g.T && ok; ++t, ++gt) {
+          // the next tile's scores are computed while the softmax warps work on this tile
+          if (t + 1 < g.T) ok = issue_s(gt + 1);
+          if (!ok) break;
+          const int s = gt % NSV;
+          MCLK(0)
+          if (!mbar_wait(smem_u32(&bars->p_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
+          MCLK(2)
+          if (!mbar_wait(smem_u32(&bars->v_full[s]), (gt / NSV) & 1)) { ok = false; break; }
+          MCLK(3)
+          // the first P V product of an item overwrites O: the previous item's accumulator must have been read out
+          if (t == 0 && n > 0 && !mbar_wait(smem_u32(&bars->o_free), (n - 1) & 1)) { ok = false; break; }
+          MCLK(5)
+          tc_fence_after();
+          const uint32_t vbase = smem_u32(sKV + (NSK + s) * KV_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < KT / 16; ++ks) {
-          // A = 16 keys of P = 8 TMEM columns of the P buffer; B = the same 16 keys (rows) of V
-          const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
-          umma_bf16_ts(tmem_o, tmem_p0 + (t & 1) * 64 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < KT / 16; ++ks) {
+            // A = 16 keys of P = 8 TMEM columns; B = the same 16 keys (rows) of V
+            const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
+            umma_bf16_ts(tmem_o, tmem_s0 + (gt & 1) * 128 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bars->v_empty[s]));
         }
-        umma_commit(smem_u32(&bars->kv_empty[s]));
-        umma_commit(smem_u32(&bars->pv_done[t & 1]));
+        if (ok) umma_commit(smem_u32(&bars->o_done));
       }
 #ifdef HSPEC_ATTN_TIMING
-      if ((blockIdx.x + blockIdx.y * 7 + blockIdx.z * 13) % 97 == 0)
-        printf("  mma (%d,%d,%d): wait_k=%lld wait_p=%lld wait_v=%lld\n", blockIdx.x, blockIdx.y, blockIdx.z, w_k, w_p, w_v);
+      MCLK(0)
+      if (blockIdx.x == 0 || blockIdx.x == 147)
+        printf("cta %d mma: total %lld | issue %lld wait_k %lld wait_p %lld wait_v %lld wait_q %lld wait_ofree %lld\n",
+               blockIdx.x, clock64() - m_start, mk[0], mk[1], mk[2], mk[3], mk[4], mk[5]);
 #endif
-      if (ok) umma_commit(smem_u32(&bars->o_done));
-      else {
+      if (!ok) {
         atomicExch(a.status, STATUS_TIMEOUT_MMA);
         *abort_flag = 1;
         mbar_arrive(smem_u32(&bars->o_done));
@@ -359,172 +450,212 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     // w % 4, so threads tid and tid + 128 share a row and exchange their half-row maxima through shared memory.
     const int r_local = tid & 127;                   // TMEM lane = query row of the tile
     const int hf = tid >> 7;                         // which half of the key columns
-    const int rg = row0 + r_local;                   // row among the k * rep rows of this KV head
-    const bool row_ok = rg < a.R;
-    const int i_blk = rg / a.rep;                    // block position of the row
-    {   // Q row -> shared memory (zeros for padding rows): each thread of the pair writes one head-dim half
-      const __nv_bfloat16* src = a.q + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH;
-#pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) {
-        const int ch = hf * 8 + c8;
-        const uint4 v = row_ok ? *reinterpret_cast<const uint4*>(src + ch * 8) : make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(sQ + tile_off(r_local, ch)) = v;
-      }
-      fence_proxy_async();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
-    }
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
-    float m_ref = NEG, l_sum = 0.f;
+    const int col0 = hf * 64;                        // first key column of this thread
+    uint32_t gt = 0, n = 0;
     bool ok = true;
 #ifdef HSPEC_ATTN_TIMING
-    long long t_wait_s = 0, t_wait_pv = 0, t_start = clock64(), t_mark, t_ld = 0, t_bar = 0, t_exp = 0, t_st = 0;
+    long long tk[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t_last = clock64(), t_start = t_last;
+#define TCLK(i) { const long long t_now = clock64(); tk[i] += t_now - t_last; t_last = t_now; }
+#else
+#define TCLK(i)
 #endif
-    for (int t = 0; t < g.T && ok; ++t) {
-#ifdef HSPEC_ATTN_TIMING
-      t_mark = clock64();
-#endif
-      if (!mbar_wait(smem_u32(&bars->s_ready[t & 1]), (t >> 1) & 1)) { ok = false; break; }
-#ifdef HSPEC_ATTN_TIMING
-      t_wait_s += clock64() - t_mark;
-#endif
-      tc_fence_after();
-#ifdef HSPEC_ATTN_TIMING
-      t_mark = clock64();
-#endif
-      float s[64];
-      const int col0 = hf * 64;                      // first key column of this thread
+    // Each thread of a row pair owns one 64-element half (128 bytes) of the Q row.  The half is pulled into L2 an item
+    // ahead and read while the item's last P V product drains.
+    auto q_half = [&](const Item& wi, bool& row_ok) -> const __nv_bfloat16* {
+      const int rg = wi.rt * 128 + r_local;
+      row_ok = rg < a.R;
+      return a.q + ((size_t(wi.b) * a.k + (row_ok ? rg / a.rep : 0)) * a.Hq + wi.kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH + hf * 64;
+    };
+    auto prefetch_q = [&](const Item& wi) {
+      bool row_ok;
+      const __nv_bfloat16* src = q_half(wi, row_ok);
+      if (row_ok) asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
+    };
+    auto load_q = [&](const Item& wi, uint4 (&qv)[8]) {
+      bool row_ok;
+      const __nv_bfloat16* src = q_half(wi, row_ok);
 #pragma unroll
-      for (int j = 0; j < 2; ++j) tmem_ld32(tmem_s0 + (t & 1) * 128 + lane_base + col0 + j * 32, reinterpret_cast<uint32_t*>(s + j * 32));
-      tmem_ld_wait();
-#ifdef HSPEC_ATTN_TIMING
-      t_ld += clock64() - t_mark; t_mark = clock64();
-#endif
-      // ---- mask by selection (raw scores; the positive scale is folded into the exponent below)
-      if (t < g.n_full) {
-        const int key0 = g.p_begin + t * KT + col0;
-        if (a.window > 0 && key0 < g.base + 16 + a.k) {                   // leading edge of the window
+      for (int c8 = 0; c8 < 8; ++c8)
+        qv[c8] = row_ok ? __ldg(reinterpret_cast<const uint4*>(src + c8 * 8)) : make_uint4(0, 0, 0, 0);
+    };
+    // Q tile -> shared memory in the swizzled K-major operand layout (zeros for padding rows)
+    auto store_q = [&](const uint4 (&qv)[8]) {
 #pragma unroll
-          for (int j = 0; j < 64; ++j)
-            if ((ctx + i_blk) - (key0 + j) >= a.window) s[j] = -INFINITY;
-        }
-      } else {
-        int n_prefix, prefix_start, n_block;
-        manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
-#pragma unroll
-        for (int j = 0; j < 64; ++j) {
-          const int col = col0 + j;
-          bool vis;
-          if (col < n_prefix) vis = a.window <= 0 || (ctx + i_blk) - (prefix_start + col) < a.window;
-          else {
-            const int jb = col - n_prefix;
-            vis = jb < n_block && jb <= i_blk && (a.window <= 0 || i_blk - jb < a.window);
-          }
-          if (!vis) s[j] = -INFINITY;
-        }
-      }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};         // four chains instead of one
-#pragma unroll
-      for (int j = 0; j < 64; j += 4) {
-        mx4[0] = fmaxf(mx4[0], s[j]); mx4[1] = fmaxf(mx4[1], s[j + 1]);
-        mx4[2] = fmaxf(mx4[2], s[j + 2]); mx4[3] = fmaxf(mx4[3], s[j + 3]);
-      }
-      // exchanged as fp16 (rounded UP, so the reference never undershoots): both threads of the row then hold the
-      // same two values and take the same decision; the reference maximum need not be the exact maximum
-      const __half mx_own = __float2half_ru(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
-      bars->xmax[t & 1][hf][r_local] = mx_own;
-      asm volatile("bar.sync 1, 256;" ::: "memory");                        // the eight softmax warps
-      const float mx = fmaxf(__half2float(mx_own), __half2float(bars->xmax[t & 1][hf ^ 1][r_local])) * a.scale_log2;
-#ifdef HSPEC_ATTN_TIMING
-      t_bar += clock64() - t_mark;
-#endif
-      // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY (same decision in both halves)
-      float factor = 1.f;
-      const bool grow = mx > m_ref + LAZY;
-      if (grow) { factor = ex2_ftz(m_ref - mx); m_ref = mx; }
-      if (t > 0 && __any_sync(0xffffffffu, grow)) {
-        // O of the tiles so far must be complete before it is rescaled; each thread rescales its 64 columns
-        if (!mbar_wait(smem_u32(&bars->pv_done[(t - 1) & 1]), ((t - 1) >> 1) & 1)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-          uint32_t o[32];
-          tmem_ld32(tmem_o + lane_base + col0 + j * 32, o);
-          tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
-          tmem_st32(tmem_o + lane_base + col0 + j * 32, o);
-        }
-        tmem_st_wait();
-      }
-      l_sum *= factor;
-      // ---- P = exp2(s - m_ref) -> bf16 pairs -> this thread's half of the TMEM P buffer
-#ifdef HSPEC_ATTN_TIMING
-      t_mark = clock64();
-#endif
-      if (t >= 2 && !mbar_wait(smem_u32(&bars->pv_done[t & 1]), ((t >> 1) - 1) & 1)) { ok = false; break; }
-#ifdef HSPEC_ATTN_TIMING
-      t_wait_pv += clock64() - t_mark;
-#endif
-#ifdef HSPEC_ATTN_TIMING
-      t_mark = clock64();
-#endif
-      const float neg_m = -m_ref;
-      float ls4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t w[32];
-#pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const float p0 = ex2_ftz(fmaf(s[2 * e], a.scale_log2, neg_m));
-        const float p1 = ex2_ftz(fmaf(s[2 * e + 1], a.scale_log2, neg_m));
-        ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
-        w[e] = pack_bf16(p0, p1);
-      }
-#ifdef HSPEC_ATTN_TIMING
-      t_exp += clock64() - t_mark; t_mark = clock64();
-#endif
-      tmem_st32(tmem_p0 + (t & 1) * 64 + lane_base + hf * 32, w);
-      l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-      tmem_st_wait();
-#ifdef HSPEC_ATTN_TIMING
-      t_st += clock64() - t_mark;
-#endif
+      for (int c8 = 0; c8 < 8; ++c8) *reinterpret_cast<uint4*>(sQ + tile_off<KV_HALF>(r_local, hf * 8 + c8)) = qv[c8];
+      fence_proxy_async();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&bars->p_ready[t & 1]));   // one arrival per warp, after all its lanes' stores
+      if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
+    };
+    int4 w_cur = items[blockIdx.x];
+    int4 w_next = (int(blockIdx.x + gridDim.x) < n_items) ? items[blockIdx.x + gridDim.x] : w_cur;
+    {
+      uint4 qv[8];
+      load_q(unpack_item(w_cur), qv);
+      store_q(qv);
     }
-#ifdef HSPEC_ATTN_TIMING
-    if (tid == 0 && (blockIdx.x + blockIdx.y * 7 + blockIdx.z * 13) % 97 == 0)
-      printf("attn cta (%d,%d,%d): T=%d total=%lld wait_s=%lld wait_pv=%lld ld=%lld max+bar=%lld exp=%lld st=%lld clocks\n", blockIdx.x, blockIdx.y,
-             blockIdx.z, g.T, clock64() - t_start, t_wait_s, t_wait_pv, t_ld, t_bar, t_exp, t_st);
-#endif
-    if (!ok) { atomicExch(a.status, STATUS_TIMEOUT_EPILOGUE); *abort_flag = 1; }
-    // ---- partial (m, l, O) of this chunk: the row sum is the sum of the two halves
-    float* xl = reinterpret_cast<float*>(&bars->xmax[0][0][0]);            // [2][128] floats
-    asm volatile("bar.sync 1, 256;" ::: "memory");                          // everyone is done with the maxima
-    xl[hf * 128 + r_local] = l_sum;
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    const float l_row = l_sum + xl[(hf ^ 1) * 128 + r_local];
-    if (ok && mbar_wait(smem_u32(&bars->o_done), 0) && !*abort_flag) {
-      tc_fence_after();
+    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n) {
+      const Item wi = unpack_item(w_cur);
+      const int b = wi.b, kvh = wi.kvh, c = wi.c, ctx = wi.ctx;
+      const Range g = make_range(ctx, a.window, a.chunk, c, a.k);
+      const int rg = wi.rt * 128 + r_local;          // row among the k * rep rows of this KV head
+      const bool row_ok = rg < a.R;
+      const int i_blk = rg / a.rep;                  // block position of the row
+      const bool has_next = it + int(gridDim.x) < n_items;
+      int4 w_next2 = w_next;                         // the descriptor is fetched two items ahead
+      if (it + 2 * int(gridDim.x) < n_items) w_next2 = items[it + 2 * gridDim.x];
+      if (has_next) prefetch_q(unpack_item(w_next));
+      float m_ref = NEG, l_sum = 0.f;
+      TCLK(0)
+      for (int t = 0; t < g.T && ok; ++t, ++gt) {
+        const uint32_t t_s = tmem_s0 + (gt & 1) * 128 + lane_base;
+        if (!mbar_wait(smem_u32(&bars->s_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
+        tc_fence_after();
+        TCLK(1)
+        float s[64];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) tmem_ld32(t_s + col0 + j * 32, reinterpret_cast<uint32_t*>(s + j * 32));
+        tmem_wait_ld32(reinterpret_cast<uint32_t*>(s));
+        tmem_wait_ld32(reinterpret_cast<uint32_t*>(s + 32));
+        // ---- mask by selection (raw scores; the positive scale is folded into the exponent below)
+        if (t < g.n_full) {
+          const int key0 = g.p_begin + t * KT + col0;
+          if (a.window > 0 && key0 < g.base + 16 + a.k) {                 // leading edge of the window
+#pragma unroll
+            for (int j = 0; j < 64; ++j)
+              if ((ctx + i_blk) - (key0 + j) >= a.window) s[j] = -INFINITY;
+          }
+        } else {
+          int n_prefix, prefix_start, n_block;
+          manual_tile(g, t - g.n_full, a.k, n_prefix, prefix_start, n_block);
+#pragma unroll
+          for (int j = 0; j < 64; ++j) {
+            const int col = col0 + j;
+            bool vis;
+            if (col < n_prefix) vis = a.window <= 0 || (ctx + i_blk) - (prefix_start + col) < a.window;
+            else {
+              const int jb = col - n_prefix;
+              vis = jb < n_block && jb <= i_blk && (a.window <= 0 || i_blk - jb < a.window);
+            }
+            if (!vis) s[j] = -INFINITY;
+          }
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};       // four chains instead of one
+#pragma unroll
+        for (int j = 0; j < 64; j += 4) {
+          mx4[0] = fmaxf(mx4[0], s[j]); mx4[1] = fmaxf(mx4[1], s[j + 1]);
+          mx4[2] = fmaxf(mx4[2], s[j + 2]); mx4[3] = fmaxf(mx4[3], s[j + 3]);
+        }
+        // exchanged as fp16 (rounded UP, so the reference never undershoots): both threads of the row then hold the
+        // same two values and take the same decision; the reference maximum need not be the exact maximum
+        const __half mx_own = __float2half_ru(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+        TCLK(2)
+        bars->xmax[gt & 1][hf][r_local] = mx_own;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->x_ready[gt & 1]));       // bounded exchange between the eight softmax warps
+        if (!mbar_wait(smem_u32(&bars->x_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
+        // (past this barrier both threads of the row hold their scores in registers: P may overwrite the S columns)
+        const float mx = fmaxf(__half2float(mx_own), __half2float(bars->xmax[gt & 1][hf ^ 1][r_local])) * a.scale_log2;
+        TCLK(3)
+        // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY (same decision in both halves)
+        float factor = 1.f;
+        const bool grow = mx > m_ref + LAZY;
+        if (grow) { factor = ex2_ftz(m_ref - mx); m_ref = mx; }
+        if (t > 0 && __any_sync(0xffffffffu, grow)) {
+          // O of the tiles so far must be complete before it is rescaled (the barrier that releases the previous
+          // tile's V slot is committed behind its P V product); each thread rescales its 64 columns
+          if (!mbar_wait(smem_u32(&bars->v_empty[(gt - 1) % NSV]), ((gt - 1) / NSV) & 1)) { ok = false; break; }
+          tc_fence_after();
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            uint32_t o[32];
+            tmem_ld32(tmem_o + lane_base + col0 + j * 32, o);
+            tmem_wait_ld32(o);
+#pragma unroll
+            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * factor);
+            tmem_st32(tmem_o + lane_base + col0 + j * 32, o);
+          }
+          tmem_st_wait();
+        }
+        l_sum *= factor;
+        TCLK(4)
+        // ---- P = exp2(s * scale - m_ref) -> bf16 pairs -> this thread's 32 of the 64 P columns, which lie over the
+        // first half of the S buffer (both threads of the row took their scores into registers before the exchange)
+        const float neg_m = -m_ref;
+        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+        uint32_t pw[32];
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          const float p0 = ex2_ftz(fmaf(s[2 * e], a.scale_log2, neg_m));
+          const float p1 = ex2_ftz(fmaf(s[2 * e + 1], a.scale_log2, neg_m));
+          ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
+          pw[e] = pack_bf16(p0, p1);
+        }
+        tmem_st32(t_s + hf * 32, pw);
+        l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+        tmem_st_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->p_ready[gt & 1]));   // one arrival per warp, after all its lanes' stores
+        TCLK(5)
+      }
+      if (!ok) break;
+      // ---- partial (m, l, O) of this chunk: the row sum is the sum of the two halves.
+      // The exchange buffer of parity gt & 1 was last used two tiles ago and is not written again before every
+      // softmax warp has signalled q_ready for the next item, i.e. after this read: 512 bytes = one float per row.
+      float* xl = reinterpret_cast<float*>(&bars->xmax[gt & 1][0][0]);
+      float l_row = l_sum;
+      if (hf == 1) {
+        xl[r_local] = l_sum;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bars->l_ready));
+      } else {
+        if (!mbar_wait(smem_u32(&bars->l_ready), n & 1)) { ok = false; break; }
+        l_row += xl[r_local];
+      }
+      {
+        // every MMA of the item has finished (so has every read of Q): the next item's Q goes in at once and the
+        // tensor core starts on its scores during the read-out
+        uint4 qv[8];
+        if (has_next) load_q(unpack_item(w_next), qv);
+        if (!mbar_wait(smem_u32(&bars->o_done), n & 1) || *abort_flag) { ok = false; break; }
+        tc_fence_after();
+        TCLK(6)
+        if (has_next) store_q(qv);
+      }
       const size_t slab = (size_t(b) * a.Hkv + kvh) * a.max_chunks + c;
       float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH + hf * 64;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         uint32_t o[32];
         tmem_ld32(tmem_o + lane_base + hf * 64 + j * 32, o);
-        tmem_ld_wait();
+        tmem_wait_ld32(o);
         if (row_ok) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
             *reinterpret_cast<uint4*>(dst + j * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
         }
       }
+      // O has been read out: the next item's first P V product may overwrite it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->o_free));
       if (row_ok && hf == 0) {
         float* ml = a.ws_ml + (slab * a.R + rg) * 2;
         ml[0] = (m_ref == NEG) ? -INFINITY : m_ref;
         ml[1] = l_row;
       }
+      w_cur = w_next;
+      w_next = w_next2;
+      TCLK(7)
     }
+#ifdef HSPEC_ATTN_TIMING
+    if ((blockIdx.x == 0 || blockIdx.x == 147) && (tid == 0 || tid == 128))
+      printf("cta %d tid %d: items %u tiles %u total %lld | q %lld wait_s %lld max %lld xchg %lld rescale %lld exp %lld wait_o %lld item_end %lld\n",
+             blockIdx.x, tid, n, gt, clock64() - t_start, tk[0], tk[1], tk[2], tk[3], tk[4], tk[5], tk[6], tk[7]);
+#endif
+    if (!ok) { atomicExch(a.status, STATUS_TIMEOUT_EPILOGUE); *abort_flag = 1; }
     tc_fence_before();
   }
   __syncthreads();
@@ -616,18 +747,31 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   CUtensorMap tmK, tmV;
   if (!make_pool_tmap(&tmK, c.k_pool, c.num_pages, c.Hkv, err) || !make_pool_tmap(&tmV, c.v_pool, c.num_pages, c.Hkv, err))
     return cudaErrorInvalidValue;
-  const size_t smem = size_t(TILE_BYTES) * (1 + 2 * NS) + sizeof(AttnTcBars) + 1024;
+  const size_t smem = size_t(KV_BYTES) * (1 + NSK + NSV) + sizeof(AttnTcBars);
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  dim3 grid(max_chunks * a.n_row_tiles, c.Hkv, c.B);
-  trk_begin(trk, "attn_partial");
-  attn_tc_kernel<<<grid, 320, smem, stream>>>(tmK, tmV, a);
+  // work list (count + items) behind the partials in the workspace
+  int* count = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(a.ws_ml + slabs * a.R * 2) + 15) & ~uintptr_t(15));
+  int4* items = reinterpret_cast<int4*>(count + 4);
+  trk_begin(trk, "attn_plan");
+  attn_tc_plan_kernel<<<1, 256, 0, stream>>>(a, count, items);
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  static int n_sms = 0;
+  if (n_sms == 0) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
+      n_sms = 148;
+  }
+  trk_begin(trk, "attn_partial");
+  attn_tc_kernel<<<n_sms, 352, smem, stream>>>(tmK, tmV, a, count, items);
+  trk_end(trk);
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int n_pairs = c.B * c.k * c.Hq;
   trk_begin(trk, "attn_merge");

@@ -13,6 +13,7 @@ enum : uint32_t {
   STATUS_TIMEOUT_PRODUCER = 0x101,
   STATUS_TIMEOUT_MMA = 0x102,
   STATUS_TIMEOUT_EPILOGUE = 0x103,
+  STATUS_BAD_SMEM_BASE = 0x104,
   STATUS_TIMEOUT_SELFTEST = 0x1ff,
 };
 
