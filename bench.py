@@ -323,9 +323,9 @@ def summarize(res, peaks):
     roofs = [r for r in (gemm_roof("gemm_2sm_kernel", g2), gemm_roof("gemm_tcgen05_kernel", g1)) if r]
     if att_ms > 0:
         roofs.append(dict(kernel="attn_tc_kernel", bound="hbm", achieved=round(att_gbs, 1), peak=hbm, unit="GB/s",
-                          frac=round(att_gbs / hbm, 4), traffic=round(1.04 * a["kv_bytes"] / n_attn), ms_per_step=round(att_ms, 4),
+                          frac=round(att_gbs / hbm, 4), traffic=round(1.06 * a["kv_bytes"] / n_attn), ms_per_step=round(att_ms, 4),
                           note=f"visible target-KV bytes / CUDA-event time over its {n_attn} launches per step, of "
-                               f"{peaks['source']}; traffic per launch = 1.04 x algorithmic, scaled from the small-case ncu "
+                               f"{peaks['source']}; traffic per launch = 1.06 x algorithmic, scaled from the small-case ncu "
                                f"capture (profiles/attn_tc_32b_small.md)"))
     roof = max(roofs, key=lambda r: r["ms_per_step"])            # the dominant kernel of this workload
     return dict(
