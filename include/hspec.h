@@ -213,6 +213,31 @@ int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t in_dtype, int3
  * Inputs and outputs are the caller's, as in hspec_op_lm_head_argmax; results are identical to it. */
 int hspec_op_lm_head_argmax_noalloc(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M,
                                     int32_t V, int32_t K, void* stream);
+/* Acceptance rule of speculative decoding (App. A): draft i of request b is accepted if every earlier draft of b
+ * was and min(1, P_T / P_D) >= alpha.  p_target, p_draft, alpha: device fp32 [B, k] (probabilities of the drafted
+ * tokens under the target and under the drafter, and the caller's uniform draws); n_accept: device int32 [B], the
+ * number of leading accepted drafts (the iteration then emits n_accept + 1 tokens).  Ratio, minimum and comparison
+ * are fp32 with IEEE division; 0 / 0 rejects, P_D = 0 with P_T > 0 accepts. */
+int hspec_op_accept(const float* p_target, const float* p_draft, const float* alpha, int32_t* n_accept, int32_t B, int32_t k,
+                    void* stream);
+/* Draft probability P_D of App. A: p[m] = softmax(logits[m, 0..V))[ids[m]] for device fp32 logits with row pitch ld
+ * elements; ids index the logits' own vocabulary (the drafter's row index when its vocabulary is pruned). */
+int hspec_op_token_probs(const float* logits, int64_t ld, const int32_t* ids, float* p, int32_t M, int32_t V, void* stream);
+/* Causal correction after the backbone (Sec. 3.3.3; rank 256 in App. B.1): a first-order dependency between adjacent
+ * draft positions applied to the logits.  The paper prints no formula; the reading implemented is a low-rank bigram
+ * table, logits'[b, i, :] = logits[b, i, :] + W_out . W_in[prev(b, i), :], prev(b, 0) = last_token[b], prev(b, i) =
+ * the token chosen at position i - 1 from the adjusted logits (lowest index on ties), positions strictly in order.
+ *   logits   device fp32 [B*k, ld] (row b*k + i), adjusted in place when write_logits != 0, else left as they are
+ *   W_in     device [V, r]  fp16 or bf16 (w_dtype), one row per possible previous TOKEN id
+ *   W_out    device [Vd, r] same type, one row per drafter-vocabulary index; r % 8 == 0, both 16-byte aligned
+ *   id_map   device int32 [Vd] drafter-vocabulary index -> token id, or NULL (identity)
+ *   ids      device int32 [B*k] out: chosen token ids
+ *   workspace >= hspec_markov_workspace_bytes(B, Vd, r), 256-byte aligned.
+ * Runs 2k + 1 launches on `stream` (one rank-r product with arg-max per position). */
+int hspec_op_markov_head(float* logits, int64_t ld, const void* W_in, const void* W_out, int32_t w_dtype, const int32_t* last_token,
+                         const int32_t* id_map, int32_t* ids, int32_t B, int32_t k, int32_t Vd, int32_t r, int32_t write_logits,
+                         void* workspace, size_t workspace_bytes, void* stream);
+size_t hspec_markov_workspace_bytes(int32_t B, int32_t Vd, int32_t r);
 /* RMSNorm over the last axis: y fp16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
 int hspec_op_rmsnorm(const float* x, const float* w, void* y_f16, int32_t M, int32_t n, float eps, void* stream);
 /* Mamba-2 mixer core for B requests x k rows (Sec. 3.3.1): causal depthwise conv + SiLU on xBC (zero left

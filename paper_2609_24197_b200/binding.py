@@ -22,6 +22,7 @@ EXPORTS = [
     "hspec_debug_wait_selftest", "hspec_clear_status", "hspec_op_gemm", "hspec_gemm_workspace_bytes",
     "hspec_op_lm_head_argmax", "hspec_op_lm_head_argmax_noalloc", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
+    "hspec_op_accept", "hspec_op_token_probs", "hspec_op_markov_head", "hspec_markov_workspace_bytes",
 ]
 
 
@@ -100,6 +101,11 @@ def load_library(path=None):
     lib.hspec_op_lm_head_argmax.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp, sz, vp]
     lib.hspec_op_lm_head_argmax_noalloc.argtypes = [vp, vp, i32, vp, vp, i32, i32, i32, vp]
     lib.hspec_op_rmsnorm.argtypes = [vp, vp, vp, i32, i32, f32, vp]
+    lib.hspec_op_accept.argtypes = [vp, vp, vp, vp, i32, i32, vp]
+    lib.hspec_op_token_probs.argtypes = [vp, i64, vp, vp, i32, i32, vp]
+    lib.hspec_op_markov_head.argtypes = [vp, i64, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
+    lib.hspec_markov_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.hspec_markov_workspace_bytes.restype = sz
     lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.hspec_scan_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.hspec_scan_workspace_bytes.restype = sz
@@ -272,6 +278,33 @@ def hspec_op_lm_head_argmax_noalloc(x, W, ids, logits=None):
     _check(load_library().hspec_op_lm_head_argmax_noalloc(
         _ptr(x), _ptr(W, x.dtype), _DT[x.dtype], _ptr(ids, torch.int32), _ptr(logits, torch.float32), M, W.shape[0], K,
         _stream()), None, "hspec_op_lm_head_argmax_noalloc")
+
+
+def hspec_op_accept(p_target, p_draft, alpha, n_accept):
+    """App. A acceptance rule on device fp32 [B, k] arrays -> n_accept int32 [B]."""
+    B, k = p_target.shape
+    _check(load_library().hspec_op_accept(_ptr(p_target, torch.float32), _ptr(p_draft, torch.float32), _ptr(alpha, torch.float32),
+                                          _ptr(n_accept, torch.int32), B, k, _stream()), None, "hspec_op_accept")
+
+
+def hspec_op_token_probs(logits, ids, p):
+    """p[m] = softmax(logits[m])[ids[m]] for fp32 logits [M, V]."""
+    M, V = logits.shape
+    _check(load_library().hspec_op_token_probs(_ptr(logits, torch.float32), V, _ptr(ids, torch.int32), _ptr(p, torch.float32),
+                                               M, V, _stream()), None, "hspec_op_token_probs")
+
+
+def hspec_markov_workspace_bytes(B, Vd, r):
+    return int(load_library().hspec_markov_workspace_bytes(B, Vd, r))
+
+
+def hspec_op_markov_head(logits, W_in, W_out, last_token, id_map, ids, B, k, write_logits, workspace):
+    """Sequential first-order correction of the block's fp32 logits [B*k, Vd] (Sec. 3.3.3) -> token ids [B*k]."""
+    Vd, r = W_out.shape
+    _check(load_library().hspec_op_markov_head(
+        _ptr(logits, torch.float32), logits.shape[1], _ptr(W_in), _ptr(W_out, W_in.dtype), _DT[W_in.dtype],
+        _ptr(last_token, torch.int32), _ptr(id_map, torch.int32), _ptr(ids, torch.int32), B, k, Vd, r, int(write_logits),
+        _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()), None, "hspec_op_markov_head")
 
 
 def hspec_op_rmsnorm(x, w, y, eps):

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhspec.so")
-SOURCES = ["hspec.cu", "gemm.cu", "gemm_2sm.cu", "attention.cu", "attention_tc.cu", "scan.cu", "elementwise.cu", "noalloc.cu"]
+SOURCES = ["hspec.cu", "gemm.cu", "gemm_2sm.cu", "attention.cu", "attention_tc.cu", "scan.cu", "elementwise.cu", "noalloc.cu", "next_ops.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--shared"]
 

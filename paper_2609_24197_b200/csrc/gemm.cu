@@ -179,6 +179,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int j = 0; j < 16; ++j) {
           const int m = m0 + c0 + j;
           float v = n_ok ? __uint_as_float(r[j]) : -INFINITY;
+          if (g.addend != nullptr && n_ok && m < g.M) v += __ldcg(g.addend + size_t(m) * g.ld_add + n);
           if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v;
           int idx = n;
 #pragma unroll
@@ -347,7 +348,7 @@ size_t gemm_splitk_bytes(int M, int n_out, int splits) {
 
 // Launches y = x W^T.  tmW must describe W with box rows 128; x is described here (box rows BN).
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
-  if (gemm2_preferred(c.M, c.n_out)) return gemm2_launch(c, stream, trk, err);
+  if (c.addend == nullptr && gemm2_preferred(c.M, c.n_out)) return gemm2_launch(c, stream, trk, err);
   if (g_smem_optin < 0) {
     int dev = 0;
     cudaGetDevice(&dev);
@@ -379,7 +380,7 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   g.stages = stages;
   g.status = c.status;
   g.f16 = c.f16 ? 1 : 0;
-  g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx;
+  g.logits = c.logits; g.addend = c.addend; g.ld_add = c.ld_add; g.part_val = c.part_val; g.part_idx = c.part_idx;
   g.ldo = c.ldo;
   if (splits > 1) {
     if (c.mode == EPI_ARGMAX) { if (err) *err = "LM-head epilogue cannot be K-sliced"; return cudaErrorInvalidValue; }

@@ -351,6 +351,7 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.n_tiles_w = (c.n_out + 255) / 256;
   g.n_tiles_m = (c.M + g.BNT - 1) / g.BNT;
   g.f16 = c.f16 ? 1 : 0; g.mode = c.mode; g.out = c.out; g.ldo = c.ldo;
+  if (c.addend != nullptr) { if (err) *err = "the 2-SM kernel has no addend epilogue"; return cudaErrorInvalidValue; }
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
   const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
   const size_t fixed = sizeof(Tail2) + 1024;

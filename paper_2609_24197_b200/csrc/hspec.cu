@@ -658,6 +658,49 @@ int hspec_op_lm_head_argmax(const void* x, const void* Wt, int32_t in_dtype, int
   return HSPEC_OK;
 }
 
+int hspec_op_accept(const float* p_target, const float* p_draft, const float* alpha, int32_t* n_accept, int32_t B, int32_t k,
+                    void* stream) {
+  if (!p_target || !p_draft || !alpha || !n_accept || B < 1 || k < 1)
+    return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_accept: bad argument");
+  std::string errtxt;
+  OP_TRY(accept_launch(p_target, p_draft, alpha, n_accept, B, k, reinterpret_cast<cudaStream_t>(stream)));
+  return HSPEC_OK;
+}
+
+int hspec_op_token_probs(const float* logits, int64_t ld, const int32_t* ids, float* p, int32_t M, int32_t V, void* stream) {
+  if (!logits || !ids || !p || M < 1 || V < 1 || ld < V) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_token_probs: bad argument");
+  std::string errtxt;
+  OP_TRY(token_probs_launch(logits, ld, ids, p, M, V, reinterpret_cast<cudaStream_t>(stream)));
+  return HSPEC_OK;
+}
+
+size_t hspec_markov_workspace_bytes(int32_t B, int32_t Vd, int32_t r) {
+  if (B < 1 || Vd < 1 || r < 1) return 0;
+  return markov_workspace_bytes(B, Vd, r);
+}
+
+int hspec_op_markov_head(float* logits, int64_t ld, const void* W_in, const void* W_out, int32_t w_dtype, const int32_t* last_token,
+                         const int32_t* id_map, int32_t* ids, int32_t B, int32_t k, int32_t Vd, int32_t r, int32_t write_logits,
+                         void* workspace, size_t workspace_bytes, void* stream) {
+  if (!logits || !W_in || !W_out || !last_token || !ids || !workspace || B < 1 || k < 1 || Vd < 1 || r < 8 || r % 8 || ld < Vd ||
+      (w_dtype != HSPEC_F16 && w_dtype != HSPEC_BF16))
+    return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_markov_head: bad argument");
+  if (workspace_bytes < markov_workspace_bytes(B, Vd, r) || (reinterpret_cast<uintptr_t>(workspace) & 255))
+    return fail(nullptr, HSPEC_ERR_WORKSPACE_TOO_SMALL, "hspec_op_markov_head: workspace too small or not 256-byte aligned");
+  std::string errtxt;
+  CUtensorMap tm;
+  if (!make_tmap_16bit_2d(&tm, W_out, Vd, r, r, 128, w_dtype == HSPEC_F16, &errtxt))
+    return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_markov_head: " + errtxt);
+  MarkovCall mc{};
+  mc.logits = logits; mc.ld = ld; mc.W_in = W_in; mc.tmW_out = &tm; mc.f16 = (w_dtype == HSPEC_F16);
+  mc.last_token = last_token; mc.id_map = id_map; mc.ids = ids; mc.B = B; mc.k = k; mc.Vd = Vd; mc.r = r;
+  mc.write_logits = write_logits; mc.ws = workspace;
+  mc.status = global_status();
+  if (!mc.status) return fail(nullptr, HSPEC_ERR_CUDA, "hspec_op_markov_head: cannot allocate the status word");
+  OP_TRY(markov_launch(mc, reinterpret_cast<cudaStream_t>(stream), nullptr, &errtxt));
+  return HSPEC_OK;
+}
+
 int hspec_op_rmsnorm(const float* x, const float* w, void* y, int32_t M, int32_t n, float eps, void* stream) {
   if (!x || !w || !y || M < 1 || n < 1) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_rmsnorm: bad argument");
   std::string errtxt;

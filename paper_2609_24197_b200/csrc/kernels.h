@@ -56,6 +56,8 @@ struct GemmArgs {       // kernel argument block
   void* out;
   long long ldo;
   float* logits;
+  const float* addend;  // EPI_ARGMAX only (one-CTA kernel): value = acc + addend[m * ld_add + n] (may be null)
+  long long ld_add;
   float* part_val;
   int* part_idx;
   uint32_t* status;
@@ -74,6 +76,8 @@ struct GemmCall {       // host-side description of one y = x W^T
   void* splitk_ws;
   size_t splitk_ws_bytes;
   float* logits;            // EPI_ARGMAX only (may be null)
+  const float* addend;      // EPI_ARGMAX, one-CTA kernel only: fp32 [M, ld_add] added before the arg-max (may be null)
+  long long ld_add;
   float* part_val;
   int* part_idx;
   uint32_t* status;
@@ -91,6 +95,25 @@ int gemm2_pick_bnt(int M, int n_out);
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk, const int* id_map = nullptr);
+
+// ---- steps next to the draft block (next_ops.cu)
+struct MarkovCall {
+  float* logits;                    // fp32 [B*k, ld]: the block's logits (adjusted in place when write_logits)
+  long long ld;
+  const void *W_in;                 // [V, r] 16-bit: factor row of every possible previous token
+  const CUtensorMap* tmW_out;       // [Vd, r] 16-bit, box 128 x 64
+  bool f16;
+  const int* last_token;            // [B]
+  const int* id_map;                // [Vd] draft-vocabulary index -> token id, or null
+  int* ids;                         // [B*k] token ids out
+  int B, k, Vd, r, write_logits;
+  void* ws;                         // markov_workspace_bytes(B, Vd, r)
+  uint32_t* status;
+};
+cudaError_t accept_launch(const float* pt, const float* pd, const float* alpha, int* n_accept, int B, int k, cudaStream_t stream);
+cudaError_t token_probs_launch(const float* logits, long long ld, const int* ids, float* p, int M, int V, cudaStream_t stream);
+size_t markov_workspace_bytes(int B, int Vd, int r);
+cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 
 // ---- attention (attention.cu)
 struct AttnCall {

@@ -1,0 +1,189 @@
+// Steps next to the draft block: the acceptance rule of App. A, the draft probability it divides by, and the
+// causal correction of Sec. 3.3.3 (a first-order dependency between adjacent draft positions applied to the logits).
+#include "common.cuh"
+#include "kernels.h"
+
+namespace hspec {
+
+namespace {
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ------------------------------------------------------------------ acceptance rule (App. A)
+// One warp per request: n[b] = number of leading positions with min(1, P_T / P_D) >= alpha, all in fp32 with IEEE
+// division.  0 / 0 (NaN) rejects; P_D = 0 with P_T > 0 (+inf) accepts.
+__global__ void accept_kernel(const float* __restrict__ pt, const float* __restrict__ pd, const float* __restrict__ alpha,
+                              int* __restrict__ n_accept, int B, int k) {
+  const int b = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (b >= B) return;
+  int n = k;
+  for (int base = 0; base < k; base += 32) {
+    const int i = base + lane;
+    bool ok = true;
+    if (i < k) {
+      const float r = __fdiv_rn(pt[size_t(b) * k + i], pd[size_t(b) * k + i]);
+      ok = !(r != r) && fminf(1.0f, r) >= alpha[size_t(b) * k + i];
+    }
+    const unsigned bad = __ballot_sync(0xffffffffu, !ok);
+    if (bad != 0u) { n = base + __ffs(bad) - 1; break; }
+  }
+  if (lane == 0) n_accept[b] = n;
+}
+
+// ------------------------------------------------------------------ softmax probability of one token per row
+// One block per row, one pass over the fp32 logits: every thread keeps a running (max, sum of exp) over its
+// elements, the block merges them; p = exp(z[id] - max) / sum.
+__global__ void token_probs_kernel(const float* __restrict__ logits, long long ld, const int* __restrict__ ids,
+                                   float* __restrict__ p, int V) {
+  const int m = blockIdx.x;
+  const float* z = logits + size_t(m) * ld;
+  float mx = -INFINITY, sum = 0.f;
+  auto add = [&](float v) {                       // (-inf entries contribute nothing, also while the maximum is still -inf)
+    if (v > mx) { sum = sum * __expf(mx - v) + 1.f; mx = v; }
+    else if (v > -INFINITY) sum += __expf(v - mx);
+  };
+  const bool vec = ((reinterpret_cast<uintptr_t>(z) & 15) == 0);
+  const int V4 = vec ? (V >> 2) : 0;
+  for (int i = threadIdx.x; i < V4; i += blockDim.x) {
+    const float4 v = __ldcs(reinterpret_cast<const float4*>(z) + i);
+    // local maximum first: one rescale per four elements
+    const float m4 = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+    if (m4 > mx) { sum *= __expf(mx - m4); mx = m4; }
+    if (mx > -INFINITY) sum += __expf(v.x - mx) + __expf(v.y - mx) + __expf(v.z - mx) + __expf(v.w - mx);
+  }
+  for (int i = V4 * 4 + threadIdx.x; i < V; i += blockDim.x) add(z[i]);
+  auto merge = [&](float omx, float osum) {
+    const float nm = fmaxf(mx, omx);
+    if (nm == -INFINITY) return;
+    sum = (mx > -INFINITY ? sum * __expf(mx - nm) : 0.f) + (omx > -INFINITY ? osum * __expf(omx - nm) : 0.f);
+    mx = nm;
+  };
+  for (int off = 16; off > 0; off >>= 1) {
+    const float omx = __shfl_xor_sync(0xffffffffu, mx, off);
+    const float osum = __shfl_xor_sync(0xffffffffu, sum, off);
+    merge(omx, osum);
+  }
+  __shared__ float smx[32], ssum[32];
+  if ((threadIdx.x & 31) == 0) { smx[threadIdx.x >> 5] = mx; ssum[threadIdx.x >> 5] = sum; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int nw = blockDim.x >> 5;
+    mx = threadIdx.x < nw ? smx[threadIdx.x] : -INFINITY;
+    sum = threadIdx.x < nw ? ssum[threadIdx.x] : 0.f;
+    for (int off = 16; off > 0; off >>= 1) {
+      const float omx = __shfl_xor_sync(0xffffffffu, mx, off);
+      const float osum = __shfl_xor_sync(0xffffffffu, sum, off);
+      merge(omx, osum);
+    }
+    if (threadIdx.x == 0) p[m] = expf(z[ids[m]] - mx) / sum;
+  }
+}
+
+// ------------------------------------------------------------------ Markov head (Sec. 3.3.3)
+// x[b, :] = W_in[prev[b], :] (16-bit rows copied as they are): the predecessor's factor row, the activation of the
+// position's rank-r product with W_out.
+__global__ void markov_gather_kernel(const uint16_t* __restrict__ W_in, const int* __restrict__ prev, long long prev_stride,
+                                     uint16_t* __restrict__ x, int r) {
+  const int b = blockIdx.x;
+  const uint16_t* src = W_in + size_t(prev[size_t(b) * prev_stride]) * r;
+  for (int i = threadIdx.x; i < (r >> 3); i += blockDim.x)
+    reinterpret_cast<uint4*>(x + size_t(b) * r)[i] = reinterpret_cast<const uint4*>(src)[i];
+}
+
+// Position i of every request: lowest index among the per-tile maxima -> ids[b * k + i] (mapped to a token id when the
+// drafter's vocabulary is pruned), and the factor row of that token -> x[b, :] for position i + 1.
+__global__ void markov_reduce_gather_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int B,
+                                            int* __restrict__ ids, int k, int i, const int* __restrict__ id_map,
+                                            const uint16_t* __restrict__ W_in, uint16_t* __restrict__ x, int r, int gather) {
+  const int b = blockIdx.x;
+  float v = -INFINITY;
+  int idx = 0x7fffffff;
+  for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
+    const float ov = pv[size_t(t) * B + b];
+    const int oi = pi[size_t(t) * B + b];
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+  __shared__ float sv[32];
+  __shared__ int si[32];
+  __shared__ int token;
+  for (int off = 16; off > 0; off >>= 1) {
+    const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  }
+  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = v; si[threadIdx.x >> 5] = idx; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const int nw = blockDim.x >> 5;
+    v = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
+    idx = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
+    for (int off = 16; off > 0; off >>= 1) {
+      const float ov = __shfl_xor_sync(0xffffffffu, v, off);
+      const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+    }
+    if (threadIdx.x == 0) {
+      const int tok = id_map ? id_map[idx] : idx;
+      ids[size_t(b) * k + i] = tok;
+      token = tok;
+    }
+  }
+  __syncthreads();
+  if (gather) {
+    const uint16_t* src = W_in + size_t(token) * r;
+    for (int j = threadIdx.x; j < (r >> 3); j += blockDim.x)
+      reinterpret_cast<uint4*>(x + size_t(b) * r)[j] = reinterpret_cast<const uint4*>(src)[j];
+  }
+}
+
+}  // namespace
+
+cudaError_t accept_launch(const float* pt, const float* pd, const float* alpha, int* n_accept, int B, int k, cudaStream_t stream) {
+  accept_kernel<<<(B + 7) / 8, 256, 0, stream>>>(pt, pd, alpha, n_accept, B, k);
+  return cudaGetLastError();
+}
+
+cudaError_t token_probs_launch(const float* logits, long long ld, const int* ids, float* p, int M, int V, cudaStream_t stream) {
+  token_probs_kernel<<<M, 512, 0, stream>>>(logits, ld, ids, p, V);
+  return cudaGetLastError();
+}
+
+size_t markov_workspace_bytes(int B, int Vd, int r) {
+  const size_t vt = (size_t(Vd) + 127) / 128;
+  return round_up(size_t(B) * r * 2, 256) + 2 * round_up(vt * B * 4, 256) + 256;
+}
+
+cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
+  const size_t vt = (size_t(c.Vd) + 127) / 128;
+  uint8_t* ws = reinterpret_cast<uint8_t*>(c.ws);
+  uint16_t* x = reinterpret_cast<uint16_t*>(ws);
+  float* part_val = reinterpret_cast<float*>(ws + round_up(size_t(c.B) * c.r * 2, 256));
+  int* part_idx = reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(part_val) + round_up(vt * c.B * 4, 256));
+  trk_begin(trk, "markov_gather");
+  markov_gather_kernel<<<c.B, 32, 0, stream>>>(reinterpret_cast<const uint16_t*>(c.W_in), c.last_token, 1, x, c.r);
+  trk_end(trk);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  for (int i = 0; i < c.k; ++i) {
+    GemmCall g{};
+    g.tmW = c.tmW_out; g.x = x; g.ldx = c.r; g.f16 = c.f16; g.M = c.B; g.n_out = c.Vd; g.K = c.r; g.mode = EPI_ARGMAX; g.splits = 1;
+    g.addend = c.logits + size_t(i) * c.ld;                 // row b of this GEMM is row b * k + i of the block's logits
+    g.ld_add = (long long)c.k * c.ld;
+    g.logits = c.write_logits ? c.logits + size_t(i) * c.ld : nullptr;
+    g.ldo = (long long)c.k * c.ld;
+    g.part_val = part_val; g.part_idx = part_idx; g.status = c.status;
+    g.label = "markov";
+    e = gemm_launch(g, stream, trk, err);
+    if (e != cudaSuccess) return e;
+    trk_begin(trk, "markov_reduce");
+    markov_reduce_gather_kernel<<<c.B, 128, 0, stream>>>(part_val, part_idx, int(vt), c.B, c.ids, c.k, i, c.id_map,
+                                                         reinterpret_cast<const uint16_t*>(c.W_in), x, c.r, i + 1 < c.k);
+    trk_end(trk);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace hspec
