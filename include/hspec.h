@@ -87,6 +87,9 @@ typedef struct {
   int32_t max_batch;         /* largest B a step may carry */
   int32_t max_k;             /* largest k a step may carry, <= HSPEC_MAX_K */
   int32_t max_pages_per_req; /* largest page-table row length (bounds the context) */
+  int32_t markov_rank;       /* 0, or the rank of the causal-correction head applied after the LM head (Sec. 3.3.3; 256 in
+                                App. B.1): tensors `markov_in` [V, rank] and `markov_out` [V or V_draft, rank] are then
+                                required and the draft ids follow hspec_op_markov_head's rule */
 } hspec_config;
 
 /* A named tensor in DEVICE memory.  hspec_load_weights copies it (converting GEMM matrices to fp16), so

@@ -33,6 +33,8 @@ What pins each function (tests/test_oracle_*.py):
 """
 import numpy as np
 
+from .accept_oracle import markov_head
+
 # --------------------------------------------------------------------------- storage helpers
 
 
@@ -345,6 +347,8 @@ def draft_block(cfg, weights, k_pools, v_pools, page_table, ctx_lens, last_hidde
       attention (target KV of slot kv_slot[l]); X += MLP(RMSNorm(X));
       logits = RMSNorm(X) W_lm^T; draft ids = argmax (lowest index on ties), translated through
       `vocab_map` when the drafter predicts over a pruned vocabulary (the LM head then holds only those rows).
+      When `markov_in` / `markov_out` are among the weights the logits first go through the causal-correction
+      head (accept_oracle.markov_head), and `logits` / `margin` are the corrected ones.
     Returns dict: draft_ids [n, k], logits [n, k, V], hidden [n, k, D], margin [n, k],
     s_init [n, H, P, N] and, if asked, per-request intermediates.
     """
@@ -387,7 +391,12 @@ def draft_block(cfg, weights, k_pools, v_pools, page_table, ctx_lens, last_hidde
             if keep_intermediates:
                 inter[f"x_after_mlp.{l}"] = X.copy()
         logits = gemm(rmsnorm(X, widen(weights["final_norm"], dtype), eps), weights["lm_head"], dtype)
-        ids, margin = argmax_margin(logits)
+        if "markov_in" in weights:        # causal correction after the backbone (Sec. 3.3.3): sequential over positions
+            ids, logits, margin = markov_head(logits[None], weights["markov_in"], weights["markov_out"],
+                                              [int(last_token[b])], id_map=weights.get("vocab_map"), dtype=dtype)
+            ids, logits, margin = ids[0], logits[0], margin[0]
+        else:
+            ids, margin = argmax_margin(logits)
         if "vocab_map" in weights:        # pruned drafter vocabulary: LM-head row index -> target token id
             ids = np.asarray(weights["vocab_map"])[ids].astype(np.int32)
         out["draft_ids"][n], out["logits"][n], out["hidden"][n] = ids, logits, X

@@ -39,6 +39,7 @@ class hspec_config(C.Structure):
         ("rope_theta", C.c_float), ("window", C.c_int32), ("qk_norm", C.c_int32), ("F", C.c_int32),
         ("V", C.c_int32), ("V_draft", C.c_int32), ("mask_id", C.c_int32), ("rms_eps", C.c_float), ("page_size", C.c_int32),
         ("max_batch", C.c_int32), ("max_k", C.c_int32), ("max_pages_per_req", C.c_int32),
+        ("markov_rank", C.c_int32),
     ]
 
 
@@ -148,6 +149,7 @@ def make_config(cfg, max_batch=None, max_k=None, max_pages_per_req=None):
                  "window", "qk_norm", "F", "V", "mask_id", "page_size"):
         setattr(c, name, int(cfg[name]))
     c.V_draft = int(cfg.get("V_draft", 0))
+    c.markov_rank = int(cfg.get("markov_rank", 0))
     c.rope_theta = float(cfg["rope_theta"])
     c.rms_eps = float(cfg["rms_eps"])
     for l in range(int(cfg["L"])):

@@ -52,7 +52,7 @@ int imax(int a, int b) { return a > b ? a : b; }
 
 // Offsets of the step's scratch buffers inside the caller's workspace.
 struct Plan {
-  size_t X, U, U2, BIG, LH, Fv, SINIT, SCAN, scan_bytes, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, total;
+  size_t X, U, U2, BIG, LH, Fv, SINIT, SCAN, scan_bytes, DTL, DT, YG, Q, KB, VB, ATT, SPLITK, AMAXV, AMAXI, LOGITS, MARKOV, total;
   size_t att_bytes, splitk_bytes;
   int attn_chunk, max_ctx;
 };
@@ -102,6 +102,11 @@ Plan make_plan(const hspec_config& c, int B, int k, int max_ctx) {
   const size_t vt = 2 * ((size_t(d.Vd) + 255) / 256);   // 128-row tiles, in pairs (the 2-SM kernel's indexing)
   p.AMAXV = take(vt * M * 4);
   p.AMAXI = take(vt * M * 4);
+  if (c.markov_rank > 0) {
+    // the causal-correction head works on materialised fp32 logits of the whole block
+    p.LOGITS = take(M * size_t(d.Vd) * 4);
+    p.MARKOV = take(markov_workspace_bytes(B, d.Vd, c.markov_rank));
+  }
   p.total = at;
   return p;
 }
@@ -125,6 +130,7 @@ const char* check_config(const hspec_config& c) {
   if (c.max_k * (c.Hq / c.Hkv) > 1024) return "k * Hq/Hkv too large";
   if (c.n_slots < 0 || c.n_slots > HSPEC_MAX_SLOTS) return "n_slots out of range";
   if (c.window < 0) return "window must be >= 0";
+  if (c.markov_rank < 0 || c.markov_rank % 8) return "markov_rank must be 0 or a multiple of 8";
   for (int l = 0; l < c.L; ++l)
     if (c.has_attn[l] && (c.kv_slot[l] < 0 || c.kv_slot[l] >= c.n_slots)) return "kv_slot out of range";
   return nullptr;
@@ -216,6 +222,8 @@ bool expected_shape(const hspec_config& c, const Dims& d, const std::string& nam
   if (name == "proj_ds") return mat(d.d_S, c.r, true);
   if (name == "final_norm") return vec(c.D);
   if (name == "lm_head") return mat(d.Vd, c.D, true);
+  if (name == "markov_in") return c.markov_rank > 0 ? mat(c.V, c.markov_rank, true) : false;
+  if (name == "markov_out") return c.markov_rank > 0 ? mat(d.Vd, c.markov_rank, true) : false;
   if (name == "vocab_map") { if (c.V_draft <= 0) return false; *rows = c.V_draft; *cols = 0; *dtype = HSPEC_I32; return true; }
   if (name.rfind("layers.", 0) != 0) return false;
   const size_t dot = name.find('.', 7);
@@ -244,6 +252,7 @@ bool expected_shape(const hspec_config& c, const Dims& d, const std::string& nam
 std::vector<std::string> required_names(const hspec_config& c) {
   std::vector<std::string> n = {"embed", "proj_r", "proj_ds", "final_norm", "lm_head"};
   if (c.V_draft > 0) n.push_back("vocab_map");
+  if (c.markov_rank > 0) { n.push_back("markov_in"); n.push_back("markov_out"); }
   for (int l = 0; l < c.L; ++l) {
     const std::string p = "layers." + std::to_string(l) + ".";
     for (const char* s : {"mamba.norm", "mamba.in_proj", "mamba.conv_w", "mamba.conv_b", "mamba.dt_bias", "mamba.A_log",
@@ -539,7 +548,21 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   if (out->hidden) EW("copy_hidden", Md * c.D * 8, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st));
   // ---- final norm, LM head fused with the per-row arg-max
   EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st));
-  {
+  const int* id_map = c.V_draft > 0 ? reinterpret_cast<const int*>(W("vocab_map").data) : nullptr;
+  if (c.markov_rank > 0) {
+    // ---- LM head to fp32 logits, then the causal correction position by position (Sec. 3.3.3)
+    float* logits = out->logits ? out->logits : reinterpret_cast<float*>(ws + p.LOGITS);
+    const Weight& w = W("lm_head");
+    GemmCall g{};
+    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_STORE_F32; g.splits = 1;
+    g.out = logits; g.ldo = d.Vd; g.status = h->d_status; g.label = "gemm:lm_head";
+    CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
+    MarkovCall mc{};
+    mc.logits = logits; mc.ld = d.Vd; mc.W_in = W("markov_in").data; mc.tmW_out = &W("markov_out").tm; mc.f16 = true;
+    mc.last_token = in->last_token; mc.id_map = id_map; mc.ids = out->draft_ids; mc.B = B; mc.k = k; mc.Vd = d.Vd;
+    mc.r = c.markov_rank; mc.write_logits = out->logits != nullptr; mc.ws = ws + p.MARKOV; mc.status = h->d_status;
+    CUDA_TRY(h, markov_launch(mc, st, trk, &errtxt));
+  } else {
     const Weight& w = W("lm_head");
     GemmCall g{};
     g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
@@ -547,7 +570,6 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     g.part_val = reinterpret_cast<float*>(ws + p.AMAXV); g.part_idx = reinterpret_cast<int*>(ws + p.AMAXI);
     g.status = h->d_status; g.label = "gemm:lm_head_argmax";
     CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
-    const int* id_map = c.V_draft > 0 ? reinterpret_cast<const int*>(W("vocab_map").data) : nullptr;
     CUDA_TRY(h, argmax_reduce_launch(g.part_val, g.part_idx, (d.Vd + 127) / 128, M, out->draft_ids, st, trk, id_map));
   }
 #undef EW

@@ -33,7 +33,7 @@ _MODEL_PAPER_8B = dict(
     D=4096, n_fuse=5, r=4096, L=4, has_attn=[1, 1, 1, 0], kv_slot=[0, 1, 2, -1],
     n_slots=3, Di=3072, P=64, N=4, G=4, d_conv=4, dt_rank=0,
     Hq=32, Hkv=8, dh=128, rope_theta=1.0e6, window=2048, qk_norm=1,
-    F=12288, V=151936, rms_eps=1e-6, page_size=16,
+    F=12288, V=151936, rms_eps=1e-6, page_size=16, markov_rank=256,
 )
 
 CONFIGS = {
@@ -45,6 +45,9 @@ CONFIGS = {
     # the concurrency-128 workload with the drafter predicting over a pruned 32 000-token vocabulary (App. B.2)
     "conc128_32b_v32k": dict(_MODEL_32B, name="conc128_32b_v32k", V_draft=32000, B=128, k=16, ctx=("loguniform", 1024, 32768)),
     "paper_8b": dict(_MODEL_PAPER_8B, name="paper_8b", B=32, k=8, ctx=("uniform", 512, 8192)),
+    # the concurrency-128 workload with the rank-256 causal-correction head behind the LM head (Sec. 3.3.3, App. B.1)
+    "conc128_32b_markov": dict(_MODEL_32B, name="conc128_32b_markov", markov_rank=256, B=128, k=16,
+                               ctx=("loguniform", 1024, 32768)),
 }
 
 
@@ -77,4 +80,5 @@ def derived(cfg):
     cfg["d_in_proj"] = cfg["Di"] + cfg["d_xBC"] + cfg["d_dt"]
     cfg["d_qkv"] = (cfg["Hq"] + 2 * cfg["Hkv"]) * cfg["dh"]
     cfg.setdefault("mask_id", cfg["V"] - 1)
+    cfg.setdefault("markov_rank", 0)
     return cfg

@@ -72,6 +72,10 @@ def weight_shapes(cfg):
     }
     if cfg.get("V_draft", 0):
         sh["vocab_map"] = ((cfg["V_draft"],), "vocab_map")   # drafter row -> target token id (pruned vocabulary)
+    if cfg.get("markov_rank", 0):
+        rm = cfg["markov_rank"]
+        sh["markov_in"] = ((cfg["V"], rm), "markov")                                   # one row per previous token
+        sh["markov_out"] = ((cfg.get("V_draft", 0) or cfg["V"], rm), "markov")         # one row per drafter-vocabulary row
     for l in range(L):
         p = f"layers.{l}."
         sh[p + "mamba.norm"] = ((D,), "gain")
@@ -105,6 +109,9 @@ def make_weights(cfg, device="cpu", only=None):
             continue
         if kind == "mat":
             t = _normal(shape, 0.02, name, device, torch.bfloat16)
+        elif kind == "markov":
+            # factor entries sized so that the rank-r table has entries of about half a logit
+            t = _normal(shape, (0.25 / shape[1]) ** 0.25, name, device, torch.bfloat16)
         elif kind == "gain":
             t = _normal(shape, 0.02, name, device, torch.float32, mean=1.0)
         elif kind == "conv_w":

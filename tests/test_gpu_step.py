@@ -141,6 +141,33 @@ def test_mid_config_pruned_drafter_vocabulary():
     drafter.close()
 
 
+@pytest.mark.parametrize("over", [dict(markov_rank=64), dict(markov_rank=72, V_draft=700), dict(markov_rank=256, k=1)])
+def test_mid_config_markov_head(over):
+    """Causal-correction head behind the LM head (Sec. 3.3.3): the step's ids and corrected logits follow the oracle's
+    sequential rule; with a pruned vocabulary the predecessor is looked up by its target id."""
+    cfg = synth.derived(dict(MID, B=3, **over))
+    k = cfg["k"] if "k" in over else 11
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[300, 41, 1500])
+    r = check_step(cfg, drafter, w, batch, k, what=f"mid markov {over}")
+    assert r["ids_compared"] > 0
+    # the head changes the draft: ids differ from the plain arg-max of the uncorrected logits somewhere
+    if k > 1:
+        plain = dict(w)
+        del plain["markov_in"], plain["markov_out"]
+        cfg0 = synth.derived(dict(cfg, markov_rank=0))
+        d0, _, _ = cuda_setup(cfg0, ctx_lens=[300, 41, 1500], weights=plain)
+        ids0 = d0.draft(batch, k)[0]
+        ids1 = drafter.draft(batch, k)[0]
+        torch.cuda.synchronize()
+        assert (ids0 != ids1).any()
+        d0.close()
+    drafter.close()
+
+
+def test_conc128_32b_markov_full_size_sampled_request():
+    _full_size("conc128_32b_markov", 1)
+
+
 def test_bounded_wait_gives_up_and_reports_without_killing_the_context():
     # failure detection without a GPU fault: a wait nobody satisfies runs out, the kernel records a status code and
     # returns; the host sees HSPEC_ERR_TIMEOUT, clears it, and the same handle then drafts correctly
