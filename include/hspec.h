@@ -10,6 +10,8 @@
  *              in place, plus the block's causal keys/values              (Sec. 3.3.2)
  *              SwiGLU MLP                                                 (App. B.1 "MLP")
  *   final norm, the target's LM head, arg-max -> k draft tokens           (App. B.2 "Pruned drafter vocabulary": LM head is the target's)
+ *   optionally (markov_rank > 0) the causal-correction head between the LM head and the arg-max: a rank-r first-order
+ *   dependency between adjacent positions, applied position by position  (Sec. 3.3.3; see hspec_op_markov_head)
  * No drafter-side KV cache exists: the library never writes the KV pools (Sec. 3.2).
  *
  * Precision
@@ -96,6 +98,7 @@ typedef struct {
  * the caller may free or reuse it afterwards.  Names (l = layer index):
  *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D] (or [V_draft,D])
  *   vocab_map [V_draft] int32 (only if V_draft > 0: target token id of each LM-head row, ascending)
+ *   markov_in [V, markov_rank]  markov_out [V or V_draft, markov_rank]  (only if markov_rank > 0)
  *   layers.l.mamba.{norm [D], in_proj [Di + (Di+2GN) + (dt_rank or H), D] (rows z | xBC | dt),
  *                   dt_up [H, dt_rank] (only if dt_rank>0), conv_w [Di+2GN, d_conv], conv_b [Di+2GN],
  *                   dt_bias [H], A_log [H], Dskip [H], gnorm [Di], out_proj [D, Di]}
@@ -137,7 +140,9 @@ typedef struct {
 typedef struct {
   int32_t* draft_ids;   /* int32 [B, k], required: arg-max of the logits, lowest row index on ties; target token ids
                            (mapped through vocab_map when the drafter vocabulary is pruned) */
-  float* logits;        /* fp32 [B, k, V] ([B, k, V_draft] when pruned) or NULL (then the logits are never materialised) */
+  float* logits;        /* fp32 [B, k, V] ([B, k, V_draft] when pruned) or NULL (then the logits are never materialised,
+                           except in the workspace when markov_rank > 0); with the causal-correction head these are the
+                           corrected logits */
   float* hidden;        /* fp32 [B, k, D] or NULL: the residual stream before the final norm */
 } hspec_out;
 
