@@ -78,6 +78,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint64_
   }
 }
 
+// 16 rows x 32 lanes -> one (max, lowest index on ties) per row with 32 shuffles instead of 160: every round a lane
+// hands half of its rows to its partner and merges the partner's copy of the half it keeps.  After the rounds with
+// offsets 16, 8, 4, 2 and a last pairwise round, v[0] / idx[0] of every EVEN lane hold the result of row `row`.
+__device__ __forceinline__ void warp_argmax16(float (&v)[16], int (&idx)[16], int lane, int& row) {
+#define HSPEC_ARGMAX_ROUND(OFF, HALF)                                                  \
+  {                                                                                    \
+    const bool up = (lane & OFF) != 0;                                                 \
+    _Pragma("unroll") for (int t = 0; t < HALF; ++t) {                                 \
+      const float sv = up ? v[t] : v[t + HALF];                                        \
+      const int si = up ? idx[t] : idx[t + HALF];                                      \
+      const float ov = __shfl_xor_sync(0xffffffffu, sv, OFF);                          \
+      const int oi = __shfl_xor_sync(0xffffffffu, si, OFF);                            \
+      float kv = up ? v[t + HALF] : v[t];                                              \
+      int ki = up ? idx[t + HALF] : idx[t];                                            \
+      if (ov > kv || (ov == kv && oi < ki)) { kv = ov; ki = oi; }                      \
+      v[t] = kv; idx[t] = ki;                                                          \
+    }                                                                                  \
+  }
+  HSPEC_ARGMAX_ROUND(16, 8)
+  HSPEC_ARGMAX_ROUND(8, 4)
+  HSPEC_ARGMAX_ROUND(4, 2)
+  HSPEC_ARGMAX_ROUND(2, 1)
+#undef HSPEC_ARGMAX_ROUND
+  const float ov = __shfl_xor_sync(0xffffffffu, v[0], 1);
+  const int oi = __shfl_xor_sync(0xffffffffu, idx[0], 1);
+  if (ov > v[0] || (ov == v[0] && oi < idx[0])) { v[0] = ov; idx[0] = oi; }
+  row = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+}
+
 // ------------------------------------------------------------------ TMA (no multicast anywhere)
 __device__ __forceinline__ void tma_prefetch_desc(const void* tmap) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(tmap) : "memory");

@@ -195,38 +195,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           vi[j] = n;
           if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v[j];
         }
-        // 16 rows x 32 lanes -> one (max, lowest index) per row with 32 shuffles: every round a lane hands half of
-        // its rows to its partner and merges the partner's copy of the half it keeps; after the rounds with
-        // offsets 16, 8, 4, 2 lane l holds row (l >> 1) & 15 (bit-reversed order below), a last round joins the pairs
-#define HSPEC_ARGMAX_ROUND(OFF, HALF)                                                        \
-        {                                                                                    \
-          const bool up = (lane & OFF) != 0;                                                 \
-          _Pragma("unroll") for (int t = 0; t < HALF; ++t) {                                 \
-            const float sv = up ? v[t] : v[t + HALF];                                        \
-            const int si = up ? vi[t] : vi[t + HALF];                                        \
-            const float ov = __shfl_xor_sync(0xffffffffu, sv, OFF);                          \
-            const int oi = __shfl_xor_sync(0xffffffffu, si, OFF);                            \
-            float kv = up ? v[t + HALF] : v[t];                                              \
-            int ki = up ? vi[t + HALF] : vi[t];                                              \
-            if (ov > kv || (ov == kv && oi < ki)) { kv = ov; ki = oi; }                      \
-            v[t] = kv; vi[t] = ki;                                                           \
-          }                                                                                  \
-        }
-        HSPEC_ARGMAX_ROUND(16, 8)
-        HSPEC_ARGMAX_ROUND(8, 4)
-        HSPEC_ARGMAX_ROUND(4, 2)
-        HSPEC_ARGMAX_ROUND(2, 1)
-#undef HSPEC_ARGMAX_ROUND
-        {
-          const float ov = __shfl_xor_sync(0xffffffffu, v[0], 1);
-          const int oi = __shfl_xor_sync(0xffffffffu, vi[0], 1);
-          if (ov > v[0] || (ov == v[0] && oi < vi[0])) { v[0] = ov; vi[0] = oi; }
-        }
-        if ((lane & 1) == 0) {
-          const int row = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-          tail->red_val[q][c0 + row] = v[0];
-          tail->red_idx[q][c0 + row] = vi[0];
-        }
+        int row;
+        warp_argmax16(v, vi, lane, row);
+        if ((lane & 1) == 0) { tail->red_val[q][c0 + row] = v[0]; tail->red_idx[q][c0 + row] = vi[0]; }
       }
     }
     if (g.mode == EPI_ARGMAX) {

@@ -260,20 +260,18 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
           }
         } else {  // EPI_ARGMAX
+          float v[16];
+          int vi[16];
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
-            float v = n_ok ? __uint_as_float(r[j]) : -INFINITY;
-            if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v;
-            int idx = n;
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-              const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-              const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-              if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-            }
-            if (lane == 0) { tail->red_val[q][c0 + j] = v; tail->red_idx[q][c0 + j] = idx; }
+            v[j] = n_ok ? __uint_as_float(r[j]) : -INFINITY;
+            vi[j] = n;
+            if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v[j];
           }
+          int row;
+          warp_argmax16(v, vi, lane, row);
+          if ((lane & 1) == 0) { tail->red_val[q][c0 + row] = v[0]; tail->red_idx[q][c0 + row] = vi[0]; }
         }
       }
       // accumulator drained: hand it back to the MMA issuer in the leader CTA
