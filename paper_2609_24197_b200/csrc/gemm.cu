@@ -253,6 +253,27 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
   }
 }
 
+// The same for fp32 outputs whose row length and pitch are multiples of four: 16-byte loads and stores, one row
+// per blockIdx.y, every slice's load issued before the first add.
+template <int SPLITS>
+__global__ void splitk_reduce_f32x4_kernel(const float* __restrict__ part, int M, int N, float* __restrict__ out,
+                                           long long ldo, int accumulate) {
+  const int m = blockIdx.y;
+  const size_t slice = size_t(M) * N;
+  for (int n4 = blockIdx.x * blockDim.x + threadIdx.x; n4 < (N >> 2); n4 += gridDim.x * blockDim.x) {
+    float4 v[SPLITS];
+#pragma unroll
+    for (int s = 0; s < SPLITS; ++s) v[s] = __ldcs(reinterpret_cast<const float4*>(part + s * slice + size_t(m) * N) + n4);
+    float4* dst = reinterpret_cast<float4*>(out + size_t(m) * ldo) + n4;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 old = accumulate ? *dst : acc;
+#pragma unroll
+    for (int s = 0; s < SPLITS; ++s) { acc.x += v[s].x; acc.y += v[s].y; acc.z += v[s].z; acc.w += v[s].w; }
+    if (accumulate) { acc.x = old.x + acc.x; acc.y = old.y + acc.y; acc.z = old.z + acc.z; acc.w = old.w + acc.w; }
+    *dst = acc;
+  }
+}
+
 // ids[m] = lowest index among the per-tile maxima (tiles are in ascending vocabulary order).
 __global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
                                      int* __restrict__ ids, const int* __restrict__ id_map) {
@@ -337,8 +358,12 @@ int gemm_pick_bn(int M) {
   return ((M + 15) / 16) * 16;
 }
 
-int gemm_pick_splits(int M, int n_out, int K, int num_sms) {
-  if (gemm2_preferred(M, n_out)) return 1;
+int gemm_pick_splits(int M, int n_out, int K, int num_sms, int mode) {
+  if (gemm2_preferred(M, n_out)) {
+    int bnt = 256, s = 1;
+    gemm2_pick(M, n_out, K, mode, &bnt, &s);
+    return s;
+  }
   // Weight streaming (few rows): keep every SM fed.  Many rows: one slice (tensor-bound, no reduction pass).
   const int k_tiles = (K + TILE_K - 1) / TILE_K;
   const int tiles = ((n_out + TILE_W - 1) / TILE_W) * ((M + 255) / 256);
@@ -409,17 +434,31 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  if (splits > 1) {
-    const long long total = (long long)c.M * c.n_out;
+  if (splits > 1)
+    e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk);
+  return e;
+}
+
+cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, void* out, long long ldo, int mode,
+                                 cudaStream_t stream, Tracker* trk) {
+  const long long total = (long long)M * N;
+  trk_begin(trk, "splitk_reduce", 0, double(splits + 1) * M * N * 4);
+  const bool f32 = mode == EPI_STORE_F32 || mode == EPI_ACCUM_F32;
+  if (f32 && (N & 3) == 0 && (ldo & 3) == 0 && (reinterpret_cast<uintptr_t>(out) & 15) == 0 && splits >= 2 && splits <= 4) {
+    // (the sum order s = 0, 1, ... and "old + sum" match the generic kernel bit for bit)
+    dim3 grid((N / 4 + 255) / 256, M);
+    float* o = reinterpret_cast<float*>(out);
+    const int acc = mode == EPI_ACCUM_F32;
+    if (splits == 2) splitk_reduce_f32x4_kernel<2><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
+    else if (splits == 3) splitk_reduce_f32x4_kernel<3><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
+    else splitk_reduce_f32x4_kernel<4><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
+  } else {
     int blocks = int((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    trk_begin(trk, "splitk_reduce", 0, double(splits + 1) * c.M * c.n_out * 4);
-    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M,
-                                                     c.n_out, c.out, c.ldo, c.mode);
-    trk_end(trk);
-    e = cudaGetLastError();
+    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(part, splits, M, N, out, ldo, mode);
   }
-  return e;
+  trk_end(trk);
+  return cudaGetLastError();
 }
 
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,

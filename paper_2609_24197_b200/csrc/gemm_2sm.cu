@@ -29,6 +29,7 @@ struct Gemm2Args {
   int BNT;                 // activation rows per cluster tile (128 or 256); each CTA stages BNT/2
   int k_tiles, stages;
   int n_tiles_w, n_tiles_m;
+  int splits, k_tiles_per_split;   // K-slices per tile (work unit = tile x slice); > 1: fp32 partials to `out`
   int f16, mode;
   void* out;
   long long ldo;
@@ -116,7 +117,7 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-  const int total_tiles = g.n_tiles_w * g.n_tiles_m;
+  const int total_units = g.n_tiles_w * g.n_tiles_m * g.splits;   // unit u = tile u / splits, K-slice u % splits
   const uint32_t tmem_cols = 2u * uint32_t(g.BNT);           // two accumulators (256 or 512 columns)
 
   if (threadIdx.x == 0) {
@@ -150,9 +151,11 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters) {
+      for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters) {
+        const int tile = unit / g.splits, sp = unit % g.splits;
         const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
-        for (int kt = 0; kt < g.k_tiles; ++kt, ++it) {
+        const int kt_end = min(g.k_tiles, (sp + 1) * g.k_tiles_per_split);
+        for (int kt = sp * g.k_tiles_per_split; kt < kt_end; ++kt, ++it) {
           const int s = it % g.stages;
           const uint32_t round = it / g.stages;
           if (round > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (round - 1) & 1)) {
@@ -174,12 +177,14 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const uint32_t idesc = idesc_m256(uint32_t(g.BNT), g.f16 != 0);
       uint32_t it = 0, tile_count = 0;
       bool ok = true;
-      for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++tile_count) {
+      for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters, ++tile_count) {
+        const int sp = unit % g.splits;
+        const int kt_begin = sp * g.k_tiles_per_split, kt_end = min(g.k_tiles, (sp + 1) * g.k_tiles_per_split);
         const uint32_t acc = tile_count & 1, use = tile_count >> 1;
         if (use > 0 && !mbar_wait(smem_u32(&tail->tmem_empty[acc]), (use - 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT);
-        for (int kt = 0; kt < g.k_tiles; ++kt, ++it) {
+        for (int kt = kt_begin; kt < kt_end; ++kt, ++it) {
           const int s = it % g.stages;
           const uint32_t round = it / g.stages;
           if (!mbar_wait(smem_u32(&tail->full[s]), round & 1)) { ok = false; break; }
@@ -188,7 +193,7 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
 #pragma unroll
           for (int kk = 0; kk < TILE_K / 16; ++kk)
-            umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > 0 || kk > 0) ? 1u : 0u);
+            umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > kt_begin || kk > 0) ? 1u : 0u);
           umma_commit_pair(smem_u32(&tail->empty[s]));
         }
         if (ok) umma_commit_pair(smem_u32(&tail->tmem_full[acc]));
@@ -202,7 +207,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     bool ok = true;
     const uint32_t empty_leader0 = mapa_rank(smem_u32(&tail->tmem_empty[0]), 0);
     const uint32_t empty_leader1 = mapa_rank(smem_u32(&tail->tmem_empty[1]), 0);
-    for (int tile = cluster_id; tile < total_tiles && ok; tile += n_clusters, ++tile_count) {
+    for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters, ++tile_count) {
+      const int tile = unit / g.splits, sp = unit % g.splits;
       const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
       const uint32_t acc = tile_count & 1, use = tile_count >> 1;
       if (!mbar_wait(smem_u32(&tail->tmem_full[acc]), use & 1)) {
@@ -221,8 +227,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         uint32_t r[16];
         tmem_ld16(tmem_acc + uint32_t(c0), r);
         tmem_ld_wait();
-        if (g.mode == EPI_STORE_F32) {
-          float* out = reinterpret_cast<float*>(g.out);
+        if (g.mode == EPI_STORE_F32 || g.mode == EPI_PARTIAL_F32) {
+          float* out = reinterpret_cast<float*>(g.out) + (g.mode == EPI_PARTIAL_F32 ? size_t(sp) * g.M * g.ldo : 0);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
@@ -318,20 +324,32 @@ bool gemm2_preferred(int M, int n_out) {
   return !off && M >= 256;
 }
 
-// Tile width (activation rows per cluster tile) that wastes the fewest cluster rounds.
-int gemm2_pick_bnt(int M, int n_out) {
+// Tile width (activation rows per cluster tile) and number of K-slices per tile that finish soonest by a simple
+// model: rounds of the 74 SM pairs x k-steps per round x cost of a k-step, plus a fixed cost per round (pipeline fill,
+// the last epilogue) and, with slices, the pass that sums the fp32 partials.  One cost unit ~ 2.2 ns (a k-step of a
+// 256-wide pair tile = 256 units ~ 0.56 us).
+void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out) {
   const int tw = (n_out + 255) / 256;
+  const int k_tiles = (K + TILE_K - 1) / TILE_K;
+  const bool may_split = mode == EPI_STORE_F32 || mode == EPI_ACCUM_F32 || mode == EPI_STORE_F16 || mode == EPI_STORE_BF16;
   double best_cost = 1e30;
-  int best = 256;
+  int best_bnt = 256, best_s = 1;
   for (int bnt : {256, 128}) {
-    const int tiles = tw * ((M + bnt - 1) / bnt);
-    const int rounds = (tiles + 73) / 74;
-    // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
-    // measured, the narrow tile runs ~1.5x slower per flop
-    const double cost = double(rounds) * bnt * (bnt == 128 ? 1.5 : 1.0);
-    if (cost < best_cost) { best_cost = cost; best = bnt; }
+    for (int s : {1, 2, 3, 4, 6, 8}) {
+      if (s > 1 && (!may_split || k_tiles / s < 8)) continue;
+      const int kps = (k_tiles + s - 1) / s;
+      if (s > 1 && kps * (s - 1) >= k_tiles) continue;         // an empty last slice
+      const long long units = (long long)tw * ((M + bnt - 1) / bnt) * s;
+      const long long rounds = (units + 73) / 74;
+      // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
+      // measured, the narrow tile runs ~1.5x slower per flop
+      double cost = double(rounds) * kps * bnt * (bnt == 128 ? 1.5 : 1.0) + double(rounds) * 1500.0;
+      if (s > 1) cost += (double(s + 2) * M * n_out * 4.0 / 5.0e6 + 4.0) * 455.0;
+      if (cost < best_cost) { best_cost = cost; best_bnt = bnt; best_s = s; }
+    }
   }
-  return best;
+  *bnt_out = best_bnt;
+  *splits_out = best_s;
 }
 
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
@@ -344,11 +362,27 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   }
   Gemm2Args g{};
   g.M = c.M; g.N_out = c.n_out; g.K = c.K;
-  g.BNT = gemm2_pick_bnt(c.M, c.n_out);
+  int splits = 1;
+  gemm2_pick(c.M, c.n_out, c.K, c.mode, &g.BNT, &splits);
+  if (c.splits > 0) {                                     // the caller fixed the number of K-slices
+    splits = c.splits;
+    if (splits > 1 && (c.mode == EPI_ARGMAX || c.mode == EPI_SWIGLU_F16)) { if (err) *err = "this epilogue cannot be K-sliced"; return cudaErrorInvalidValue; }
+  }
   g.k_tiles = (c.K + TILE_K - 1) / TILE_K;
+  if (splits > g.k_tiles) splits = g.k_tiles;
+  g.k_tiles_per_split = (g.k_tiles + splits - 1) / splits;
+  splits = (g.k_tiles + g.k_tiles_per_split - 1) / g.k_tiles_per_split;   // no empty slice
+  g.splits = splits;
   g.n_tiles_w = (c.n_out + 255) / 256;
   g.n_tiles_m = (c.M + g.BNT - 1) / g.BNT;
   g.f16 = c.f16 ? 1 : 0; g.mode = c.mode; g.out = c.out; g.ldo = c.ldo;
+  if (splits > 1) {
+    if (c.splitk_ws == nullptr || c.splitk_ws_bytes < gemm_splitk_bytes(c.M, c.n_out, splits)) {
+      if (err) *err = "K-slice workspace too small";
+      return cudaErrorInvalidValue;
+    }
+    g.mode = EPI_PARTIAL_F32; g.out = c.splitk_ws; g.ldo = c.n_out;
+  }
   if (c.addend != nullptr) { if (err) *err = "the 2-SM kernel has no addend epilogue"; return cudaErrorInvalidValue; }
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
   const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
@@ -359,7 +393,7 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.stages = stages;
   CUtensorMap tmB;
   if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BNT / 2, c.f16, err)) return cudaErrorInvalidValue;
-  const int total = g.n_tiles_w * g.n_tiles_m;
+  const int total = g.n_tiles_w * g.n_tiles_m * splits;
   const int clusters = total < 74 ? total : 74;
   const size_t smem = size_t(stages) * stage_bytes + fixed;
   // profile name "gemm2:<what>" tells this kernel's launches from the one-CTA kernel's "gemm:<what>"
@@ -368,7 +402,10 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   trk_begin(trk, label.c_str(), 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
   gemm_2sm_kernel<<<2 * clusters, 192, smem, stream>>>(*c.tmW, tmB, g);
   trk_end(trk);
-  return cudaGetLastError();
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess && splits > 1)
+    e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk);
+  return e;
 }
 
 }  // namespace hspec

@@ -470,7 +470,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     GemmCall g{};
     g.tmW = &w.tm; g.x = x; g.f16 = true; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
     g.mode = mode; g.out = o; g.ldo = ldo;
-    g.splits = gemm_pick_splits(rows, g.n_out, g.K, kNumSMs);
+    g.splits = gemm_pick_splits(rows, g.n_out, g.K, kNumSMs, mode);
     g.splitk_ws = ws + p.SPLITK; g.splitk_ws_bytes = p.splitk_bytes;
     g.status = h->d_status; g.label = label;
     return gemm_launch(g, st, trk, &errtxt);

@@ -87,11 +87,13 @@ struct GemmCall {       // host-side description of one y = x W^T
 bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
                        int box_rows, bool f16, std::string* err);
 int gemm_pick_bn(int M);
-int gemm_pick_splits(int M, int n_out, int K, int num_sms);
+int gemm_pick_splits(int M, int n_out, int K, int num_sms, int mode = EPI_STORE_F32);
 size_t gemm_splitk_bytes(int M, int n_out, int splits);
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 bool gemm2_preferred(int M, int n_out);        // many rows and at least one full round of cluster tiles
-int gemm2_pick_bnt(int M, int n_out);
+void gemm2_pick(int M, int n_out, int K, int mode, int* bnt, int* splits);   // tile width and K-slices of the 2-SM kernel
+cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, void* out, long long ldo, int mode,
+                                 cudaStream_t stream, Tracker* trk);
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk, const int* id_map = nullptr);

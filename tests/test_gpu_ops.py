@@ -46,6 +46,8 @@ GEMM_CASES = [
     (256, 640, 128), (257, 130, 1024), (513, 256, 320), (33, 17536 // 8, 520),
     # many rows and enough tiles for the 2-SM persistent kernel (ragged in every dimension)
     (2048, 5120, 512), (600, 19000, 192), (300, 40000, 72), (2048, 2500, 4096),
+    # few tiles and a long contraction: the 2-SM kernel slices K on its own
+    (512, 4096, 4096), (256, 1024, 14336), (384, 700, 9000),
 ]
 
 
