@@ -146,9 +146,11 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
   if (warp == 0) {
     if (lane == 0) {
-      // evict-first on the weights measured faster than evict-normal (1.25 vs 1.15 PFLOP/s on 2048 x 51200 x 5120)
-      // although ncu shows 2.4x the algorithmic DRAM reads: the activation tile must not be pushed out of L2
-      const uint64_t pol_w = policy_evict_first(), pol_x = policy_evict_last();
+      // Weights at normal L2 priority, activations evict-last.  Evict-first weights ran a few percent faster in
+      // short isolated runs, but ncu showed 2.4x the algorithmic DRAM reads (the clusters that share a weight tile
+      // drift apart and fetch it again), and in a long power-capped step the extra DRAM traffic costs clock:
+      // 13.5 vs 13.75 ms per step at conc128_32b.
+      const uint64_t pol_w = policy_evict_normal(), pol_x = policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters) {
@@ -157,8 +159,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int kt_end = min(g.k_tiles, (sp + 1) * g.k_tiles_per_split);
         for (int kt = sp * g.k_tiles_per_split; kt < kt_end; ++kt, ++it) {
           const int s = it % g.stages;
-          const uint32_t round = it / g.stages;
-          if (round > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (round - 1) & 1)) {
+          const uint32_t lap = it / g.stages;
+          if (lap > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (lap - 1) & 1)) {
             atomicExch(g.status, STATUS_TIMEOUT_PRODUCER);
             *abort_flag = 1;
             ok = false;
@@ -186,8 +188,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT);
         for (int kt = kt_begin; kt < kt_end; ++kt, ++it) {
           const int s = it % g.stages;
-          const uint32_t round = it / g.stages;
-          if (!mbar_wait(smem_u32(&tail->full[s]), round & 1)) { ok = false; break; }
+          const uint32_t lap = it / g.stages;
+          if (!mbar_wait(smem_u32(&tail->full[s]), lap & 1)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes);
           const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
@@ -318,14 +320,14 @@ int g_smem_optin2 = -1;
 
 bool gemm2_preferred(int M, int n_out) {
   static const bool off = [] { const char* e = getenv("HSPEC_GEMM_1SM"); return e && e[0] == '1'; }();
-  // from 256 rows on the contractions are tensor-bound; even a partly filled round of pair tiles beats the one-CTA
+  // from 256 rows on the contractions are tensor-bound; even a partly filled wave of pair tiles beats the one-CTA
   // kernel with K-slices and its reduction pass
   (void)n_out;
   return !off && M >= 256;
 }
 
 // Tile width (activation rows per cluster tile) and number of K-slices per tile that finish soonest by a simple
-// model: rounds of the 74 SM pairs x k-steps per round x cost of a k-step, plus a fixed cost per round (pipeline fill,
+// model: waves of the 74 SM pairs x k-steps per wave x cost of a k-step, plus a fixed cost per wave (pipeline fill,
 // the last epilogue) and, with slices, the pass that sums the fp32 partials.  One cost unit ~ 2.2 ns (a k-step of a
 // 256-wide pair tile = 256 units ~ 0.56 us).
 void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out) {
@@ -340,10 +342,10 @@ void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out
       const int kps = (k_tiles + s - 1) / s;
       if (s > 1 && kps * (s - 1) >= k_tiles) continue;         // an empty last slice
       const long long units = (long long)tw * ((M + bnt - 1) / bnt) * s;
-      const long long rounds = (units + 73) / 74;
+      const long long waves = (units + 73) / 74;
       // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
       // measured, the narrow tile runs ~1.5x slower per flop
-      double cost = double(rounds) * kps * bnt * (bnt == 128 ? 1.5 : 1.0) + double(rounds) * 1500.0;
+      double cost = double(waves) * kps * bnt * (bnt == 128 ? 1.5 : 1.0) + double(waves) * 1500.0;
       if (s > 1) cost += (double(s + 2) * M * n_out * 4.0 / 5.0e6 + 4.0) * 455.0;
       if (cost < best_cost) { best_cost = cost; best_bnt = bnt; best_s = s; }
     }
