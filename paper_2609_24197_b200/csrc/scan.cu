@@ -338,15 +338,24 @@ __global__ void scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* _
   const size_t row0 = size_t(b) * a.k;
   const int GN = a.G * a.N;
   const int c_col = ch - a.Di - GN;                          // >= 0 for C channels
-  for (int i = 0; i < a.k; ++i) {
-    const float cur = a.zxbcdt[(row0 + i) * a.ld_in + a.Di + ch];
-    const float v = silu_f(bias + w[0] * h0 + w[1] * h1 + w[2] * h2 + w[3] * cur);
-    h0 = h1; h1 = h2; h2 = cur;
-    xact[(row0 + i) * a.d_xBC + ch] = v;
-    if (c_col >= 0) {
-      const __half hi = __float2half_rn(v);
-      c16[((row0 + i) * 2 + 0) * GN + c_col] = hi;
-      c16[((row0 + i) * 2 + 1) * GN + c_col] = __float2half_rn(v - __half2float(hi));
+  // eight rows' loads are issued together: the recurrence over rows is short, the load latency is not
+  for (int i0 = 0; i0 < a.k; i0 += 8) {
+    float in[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) in[j] = (i0 + j < a.k) ? __ldcs(a.zxbcdt + (row0 + i0 + j) * a.ld_in + a.Di + ch) : 0.f;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int i = i0 + j;
+      if (i >= a.k) break;
+      const float cur = in[j];
+      const float v = silu_f(bias + w[0] * h0 + w[1] * h1 + w[2] * h2 + w[3] * cur);
+      h0 = h1; h1 = h2; h2 = cur;
+      xact[(row0 + i) * a.d_xBC + ch] = v;
+      if (c_col >= 0) {
+        const __half hi = __float2half_rn(v);
+        c16[((row0 + i) * 2 + 0) * GN + c_col] = hi;
+        c16[((row0 + i) * 2 + 1) * GN + c_col] = __float2half_rn(v - __half2float(hi));
+      }
     }
   }
 }
