@@ -60,3 +60,32 @@ def test_no_cpu_path(lib):
     cfg = synth.get_config("tiny")
     with pytest.raises(hs.HSpecError, match="no CUDA device"):
         hs.Drafter(cfg, {}, 1, 8, 256)
+
+
+def test_markov_config_and_workspace_without_a_gpu(lib):
+    """markov_rank is validated at init, enlarges the step's workspace (fp32 logits of the block + the per-position
+    scratch), and the stand-alone op reports its scratch size."""
+    import synth
+    plain = synth.get_config("tiny")
+    with_head = synth.get_config("tiny", markov_rank=64)
+    w0 = hs.hspec_workspace_bytes(hs.make_config(plain, 2, 8, 16))
+    w1 = hs.hspec_workspace_bytes(hs.make_config(with_head, 2, 8, 16))
+    assert w1 >= w0 + 2 * 8 * plain["V"] * 4
+    with pytest.raises(hs.HSpecError, match="markov_rank"):
+        hs.hspec_init(hs.make_config(synth.get_config("tiny", markov_rank=12), 2, 8, 16))
+    B, Vd, r = 3, 1000, 64
+    need = hs.hspec_markov_workspace_bytes(B, Vd, r)
+    tiles = (Vd + 127) // 128
+    assert need >= B * r * 2 + 2 * tiles * B * 4
+    assert hs.hspec_markov_workspace_bytes(0, Vd, r) == 0
+
+
+def test_new_entry_points_reject_bad_arguments_without_touching_the_gpu(lib):
+    """Argument checks come first: NULL pointers and bad sizes are refused with HSPEC_ERR_INVALID_ARG (-1 .. small
+    negative codes), never passed to a kernel."""
+    null = ctypes.c_void_p(None)
+    assert lib.hspec_op_accept(null, null, null, null, 4, 4, null) < 0
+    assert lib.hspec_op_token_probs(null, 10, null, null, 1, 10, null) < 0
+    assert lib.hspec_op_markov_head(null, 10, null, null, hs.HSPEC_F16, null, null, null, 1, 1, 10, 64, 0, null, 0, null) < 0
+    msg = lib.hspec_last_error(None)
+    assert msg and b"hspec_op_markov_head" in msg
