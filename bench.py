@@ -211,6 +211,32 @@ def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=
     out = dict(name=name, B=B, k=k, ms_per_step=total_ms / steps, step_ms=step_ms, acct=acct, prof=prof,
                launches_per_step=launches, clocks=clocks, ctx_sum=sum(ctx), ctx_max=max_ctx, cfg=cfg,
                ms_per_step_profiled=sum(step_ms) / steps)
+    # ---- the step captured once in a CUDA graph and replayed (what a serving loop does with a launch-bound step);
+    # reported beside `value`, which stays on plain launches
+    out["graph_replay_ms_per_step"] = None
+    if not lean:
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            with torch.cuda.stream(side):
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    step()
+            torch.cuda.synchronize()
+            for _ in range(3):
+                graph.replay()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            g0.record(stream)
+            for _ in range(steps):
+                graph.replay()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            out["graph_replay_ms_per_step"] = g0.elapsed_time(g1) / steps
+            del graph
+        except Exception as exc:                   # a capture failure must not cost the bench line
+            print(f"[bench] graph capture skipped: {exc}", file=sys.stderr)
+            torch.cuda.synchronize()
     if lean:                                       # launch-list captures: nothing more
         out["e2e"] = dict(ms_per_step=float("nan"), h2d_bytes_per_step=0, d2h_bytes_per_step=0)
         out["_keep"] = (drafter, batch)
@@ -341,6 +367,8 @@ def summarize(res, peaks):
         roofline=roof, rooflines=roofs, drafter_kv_GB_avoided=round(a["drafter_kv_bytes_avoided"] / 1e9, 3),
         launches_per_step=res["launches_per_step"],
         ms_per_step_profiled=round(res["ms_per_step_profiled"], 4),
+        graph_replay_ms_per_step=(round(res["graph_replay_ms_per_step"], 4)
+                                  if res.get("graph_replay_ms_per_step") is not None else None),
     )
 
 
@@ -381,7 +409,8 @@ def main_ours(args):
         "clocks": head["clocks"],
         "roofline": s["roofline"], "rooflines": s["rooflines"],
         "step": {k: s[k] for k in ("hbm_roofline_ms", "hbm_roofline_frac", "tensor_roofline_ms", "max_roofline_frac",
-                                   "weight_GB", "kv_GB", "drafter_kv_GB_avoided", "ms_per_step_profiled")},
+                                   "weight_GB", "kv_GB", "drafter_kv_GB_avoided", "ms_per_step_profiled",
+                                   "graph_replay_ms_per_step")},
         "attention": s["attention"], "gemm": s["gemm"], "kernels": kernel_table(head),
         "peaks": peaks,
     }
@@ -398,13 +427,15 @@ def main_ours(args):
             if name == args.workload:
                 byc[conc] = dict(workload=name, draft_tokens_per_s=s["draft_tokens_per_s"], ms_per_step=s["ms_per_step"],
                                  hbm_roofline_frac=s["hbm_roofline_frac"], max_roofline_frac=s["max_roofline_frac"],
-                                 attention_frac_of_hbm=s["attention"]["frac_of_hbm"])
+                                 attention_frac_of_hbm=s["attention"]["frac_of_hbm"],
+                                 graph_replay_ms_per_step=s["graph_replay_ms_per_step"])
                 continue
             r = run_workload(name, args.steps, args.warmup, rank, want_e2e=False)
             t = summarize(r, peaks)
             byc[conc] = dict(workload=name, draft_tokens_per_s=t["draft_tokens_per_s"], ms_per_step=t["ms_per_step"],
                              hbm_roofline_frac=t["hbm_roofline_frac"], max_roofline_frac=t["max_roofline_frac"],
-                             attention_frac_of_hbm=t["attention"]["frac_of_hbm"], gemm=t["gemm"],
+                             attention_frac_of_hbm=t["attention"]["frac_of_hbm"],
+                             graph_replay_ms_per_step=t["graph_replay_ms_per_step"], gemm=t["gemm"],
                              kernels=kernel_table(r))
             del r
             torch.cuda.empty_cache()

@@ -186,3 +186,34 @@ def test_bounded_wait_gives_up_and_reports_without_killing_the_context():
     torch.cuda.synchronize()
     assert torch.equal(ids0, ids1) and drafter.stats()["device_status"] == 0
     drafter.close()
+
+
+def test_step_is_capturable_in_a_cuda_graph_and_replays_bit_exactly():
+    """hspec_draft_block only enqueues work on the caller's stream (no host synchronisation, no allocation), so a
+    serving loop can capture it once and replay it; the replay reads the CURRENT contents of the input buffers."""
+    cfg = synth.derived(dict(MID, B=3))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[300, 41, 1500])
+    k = 9
+    ids_direct = drafter.draft(batch, k)[0].clone()
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ids_graph = drafter.draft(batch, k)[0]
+    torch.cuda.synchronize()
+    ids_graph.fill_(-1)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(ids_graph, ids_direct)
+    # new inputs in the same buffers: the replay follows them
+    batch["last_token"].copy_((batch["last_token"] + 7) % cfg["V"])
+    batch["last_hidden"].copy_(batch["last_hidden"].flip(0))
+    graph.replay()
+    torch.cuda.synchronize()
+    ids_new = drafter.draft(batch, k)[0]
+    torch.cuda.synchronize()
+    assert torch.equal(ids_graph, ids_new)
+    assert not torch.equal(ids_new, ids_direct)
+    assert drafter.stats()["device_status"] == 0
+    drafter.close()
