@@ -203,12 +203,13 @@ __global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4*
   __shared__ int bucket[64];
   __shared__ int offset[64];
   const int per_chunk = a.Hkv * a.n_row_tiles;
+  const int pairs = a.B * a.max_chunks;            // one thread per (request, chunk slot); slots past n_chunks are skipped
   for (int i = threadIdx.x; i < 64; i += blockDim.x) bucket[i] = 0;
   __syncthreads();
-  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
-    const int ctx = a.ctx_lens[b];
-    const int n_chunks = make_range(ctx, a.window, a.chunk, 0, a.k).n_chunks;
-    for (int c = 0; c < n_chunks; ++c) atomicAdd(&bucket[min(make_range(ctx, a.window, a.chunk, c, a.k).T, 63)], per_chunk);
+  for (int i = threadIdx.x; i < pairs; i += blockDim.x) {
+    const int b = i / a.max_chunks, c = i % a.max_chunks;
+    const Range g = make_range(a.ctx_lens[b], a.window, a.chunk, c, a.k);
+    if (c < g.n_chunks) atomicAdd(&bucket[min(g.T, 63)], per_chunk);
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -217,14 +218,14 @@ __global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4*
     *count = off;
   }
   __syncthreads();
-  for (int b = threadIdx.x; b < a.B; b += blockDim.x) {
+  for (int i = threadIdx.x; i < pairs; i += blockDim.x) {
+    const int b = i / a.max_chunks, c = i % a.max_chunks;
     const int ctx = a.ctx_lens[b];
-    const int n_chunks = make_range(ctx, a.window, a.chunk, 0, a.k).n_chunks;
-    for (int c = 0; c < n_chunks; ++c) {
-      int at = atomicAdd(&offset[min(make_range(ctx, a.window, a.chunk, c, a.k).T, 63)], per_chunk);
-      for (int kvh = 0; kvh < a.Hkv; ++kvh)
-        for (int rt = 0; rt < a.n_row_tiles; ++rt) items[at++] = make_int4(b, kvh | (rt << 16), c, ctx);
-    }
+    const Range g = make_range(ctx, a.window, a.chunk, c, a.k);
+    if (c >= g.n_chunks) continue;
+    int at = atomicAdd(&offset[min(g.T, 63)], per_chunk);
+    for (int kvh = 0; kvh < a.Hkv; ++kvh)
+      for (int rt = 0; rt < a.n_row_tiles; ++rt) items[at++] = make_int4(b, kvh | (rt << 16), c, ctx);
   }
 }
 
