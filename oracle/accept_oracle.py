@@ -23,6 +23,13 @@ with the CUDA library and is never imported by the product path.
                   example, no formula); the arithmetic of the reading itself is
                   pinned as listed below.
 
+  kv_inject_rows  the comparison drafters' KV injection (Sec. 2.2 "KV injection in block
+                  drafting"), kept as a measured counter-example to the bytes H-Spec avoids:
+                  per new position, projected key rows get the per-head RMSNorm (optional)
+                  and rotate-half RoPE at that position, value rows are taken as they are,
+                  and both are written into a drafter-side paged KV cache (scatter_kv).
+                  The projection in front of it is an ordinary bias-free linear map.
+
 What pins each function (tests/test_oracle_accept.py):
   token_probs     rows sum to one over all tokens, uniform logits, shift
                   invariance, two-token closed form (logistic)
@@ -33,6 +40,11 @@ What pins each function (tests/test_oracle_accept.py):
   markov_head     dense bigram table + Python loops on tiny sizes, W_out = 0 is the
                   plain arg-max, a constructed chain (table forces t -> t + 1), and
                   locality (a change at position j cannot alter positions < j)
+  kv_inject_rows / scatter_kv
+                  scatter then gather (hspec_oracle.gather_kv) returns the rows, rows not
+                  addressed keep their bits, position 0 leaves keys unrotated, the norm of
+                  a key row is preserved by the rotation, relative-position law
+                  <RoPE(a, p), RoPE(b, p + d)> independent of p
 """
 import numpy as np
 
@@ -105,3 +117,38 @@ def markov_head(logits, W_in, W_out, last_token, id_map=None, dtype=np.float64):
                 margin[b, i] = np.inf
             prev = t if id_map is None else int(id_map[t])
     return ids, adj, margin
+
+
+def kv_inject_rows(kv, k_norm_w, pos, theta, eps=1e-6, k_norm=True, dtype=np.float64):
+    """Key / value rows of T new positions as a KV-injecting drafter would cache them.
+
+    kv [T, 2, Hkv, dh] (projected keys | values); k_norm_w [dh]; pos [T] absolute positions.
+    Keys: optional per-head RMSNorm over dh, then rotate-half RoPE at pos (pairs (j, j + dh/2),
+    inv_freq = theta^(-2j/dh) rounded to float32, angle = ONE float32 product float(pos) * inv_freq);
+    values unchanged.  Returns (K [T, Hkv, dh], V [T, Hkv, dh]) in `dtype`.
+    """
+    kv = np.asarray(kv).astype(dtype)
+    T, _, Hkv, dh = kv.shape
+    half = dh // 2
+    K = kv[:, 0].copy()
+    V = kv[:, 1].copy()
+    if k_norm:
+        K = K / np.sqrt(np.mean(K * K, axis=-1, keepdims=True) + eps) * np.asarray(k_norm_w).astype(dtype)
+    inv_freq = (np.float64(theta) ** (-2.0 * np.arange(half, dtype=np.float64) / dh)).astype(np.float32)
+    out = np.empty_like(K)
+    for t in range(T):
+        ang = (np.float32(pos[t]) * inv_freq).astype(np.float32).astype(np.float64)
+        cs, sn = np.cos(ang), np.sin(ang)
+        a, b = K[t, :, :half], K[t, :, half:]
+        out[t, :, :half] = a * cs - b * sn
+        out[t, :, half:] = b * cs + a * sn
+    return out, V
+
+
+def scatter_kv(pool, page_row, pos, rows):
+    """Inverse of a paged gather: pool[page_row[p // page], p % page] = rows[i] for p = pos[i].
+    pool [num_pages, page, Hkv, dh] is modified in place; pure data movement."""
+    page = pool.shape[1]
+    for i, p in enumerate(pos):
+        pool[int(page_row[int(p) // page]), int(p) % page] = rows[i]
+    return pool

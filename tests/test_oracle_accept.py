@@ -174,3 +174,62 @@ def test_markov_locality():
     z2[:, 5] += rng.normal(size=(B, V)) * 10
     ids1, _, _ = ao.markov_head(z2, W_in, W_out, last)
     np.testing.assert_array_equal(ids0[:, :5], ids1[:, :5])
+
+
+# --------------------------------------------------------------------------- kv_inject_rows / scatter_kv
+
+def test_scatter_then_gather_round_trip_and_untouched_rows():
+    from oracle import hspec_oracle as O
+    rng = np.random.default_rng(11)
+    pool = rng.normal(size=(9, 16, 2, 8)).astype(np.float32)
+    before = pool.copy()
+    page_row = np.array([5, 2, 7, 0])
+    pos = np.array([3, 17, 18, 40])
+    rows = rng.normal(size=(4, 2, 8)).astype(np.float32)
+    ao.scatter_kv(pool, page_row, pos, rows)
+    got = O.gather_kv(pool, page_row, 41)
+    np.testing.assert_array_equal(got[pos], rows)
+    mask = np.ones(41, dtype=bool); mask[pos] = False
+    np.testing.assert_array_equal(got[mask], O.gather_kv(before, page_row, 41)[mask])
+    untouched = [p for p in range(9) if p not in page_row]
+    np.testing.assert_array_equal(pool[untouched], before[untouched])
+
+
+def test_kv_inject_rows_rotation_properties():
+    rng = np.random.default_rng(12)
+    T, Hkv, dh = 5, 2, 16
+    kv = rng.normal(size=(T, 2, Hkv, dh))
+    ones = np.ones(dh)
+    K0, V0 = ao.kv_inject_rows(kv, ones, np.zeros(T, dtype=int), 1.0e4, k_norm=False)
+    np.testing.assert_array_equal(K0, kv[:, 0])                      # position 0: no rotation
+    np.testing.assert_array_equal(V0, kv[:, 1])                      # values are never touched
+    pos = np.array([1, 7, 100, 4095, 31999])
+    K, _ = ao.kv_inject_rows(kv, ones, pos, 1.0e4, k_norm=False)
+    np.testing.assert_allclose(np.linalg.norm(K, axis=-1), np.linalg.norm(kv[:, 0], axis=-1), rtol=1e-12)
+    # with the norm on, every key head has unit RMS times the gain
+    Kn, _ = ao.kv_inject_rows(kv, 2.0 * ones, pos, 1.0e4, eps=0.0, k_norm=True)
+    np.testing.assert_allclose(np.sqrt(np.mean(Kn * Kn, axis=-1)), 2.0, rtol=1e-12)
+
+
+def test_kv_inject_rows_relative_position_law():
+    """<RoPE(a, p), RoPE(b, p + d)> depends on d only (up to the float32 rounding of the angles)."""
+    rng = np.random.default_rng(13)
+    a = rng.normal(size=(1, 2, 1, 32)); b = rng.normal(size=(1, 2, 1, 32))
+    ones = np.ones(32)
+    dots = []
+    for p in (0, 5, 64, 1000):
+        Ka, _ = ao.kv_inject_rows(a, ones, [p], 1.0e6, k_norm=False)
+        Kb, _ = ao.kv_inject_rows(b, ones, [p + 9], 1.0e6, k_norm=False)
+        dots.append(float(np.sum(Ka * Kb)))
+    np.testing.assert_allclose(dots, dots[0], rtol=0, atol=2e-3)
+
+
+def test_kv_inject_keys_match_the_step_oracles_rope():
+    """The injected key of position p equals what the draft step's own RoPE gives a block key at that position."""
+    from oracle import hspec_oracle as O
+    rng = np.random.default_rng(14)
+    kv = rng.normal(size=(3, 2, 2, 16))
+    pos = np.array([2, 50, 777])
+    K, _ = ao.kv_inject_rows(kv, np.ones(16), pos, 1.0e6, k_norm=False)
+    for t in range(3):
+        np.testing.assert_allclose(K[t], O.rope(kv[t, 0], int(pos[t]), 1.0e6), rtol=1e-12, atol=1e-12)
