@@ -276,6 +276,55 @@ def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=
     return out
 
 
+def kv_injection_counterexample(cfg, reps=10):
+    """What a KV-injecting block drafter of the same shape adds to every step (Sec. 2.2 of the paper) and this
+    drafter does not do: for the positions verified since the last step, fuse the target's hidden states, project
+    them to keys and values for each attention layer and write them into a drafter-side paged cache.  Measured with
+    the library's own GEMM and cache-write kernels on k new positions per request (the case where a whole block was
+    accepted), beside the number of bytes the cache grows by per step."""
+    import paper_2609_24197_b200 as hs
+    dev = torch.device("cuda", torch.cuda.current_device())
+    B, k, D, r = cfg["B"], cfg["k"], cfg["D"], cfg["r"]
+    Hkv, dh, ps = cfg["Hkv"], cfg["dh"], cfg["page_size"]
+    layers = int(sum(cfg["has_attn"]))
+    T = B * k
+    g = torch.Generator(device=dev).manual_seed(synth.BASE_SEED + 77)
+    h = torch.randn((T, cfg["n_fuse"] * D), generator=g, device=dev).to(torch.float16)
+    w_fuse = (torch.randn((r, cfg["n_fuse"] * D), generator=g, device=dev) * 0.02).to(torch.float16)
+    w_kv = [(torch.randn((2 * Hkv * dh, r), generator=g, device=dev) * 0.02).to(torch.float16) for _ in range(layers)]
+    kw = torch.ones(dh, device=dev)
+    pages_per_req = (k + ps - 1) // ps
+    page_table = torch.arange(B * pages_per_req, dtype=torch.int32, device=dev).reshape(B, pages_per_req).contiguous()
+    pools = [(torch.zeros((B * pages_per_req, ps, Hkv, dh), dtype=torch.bfloat16, device=dev),
+              torch.zeros((B * pages_per_req, ps, Hkv, dh), dtype=torch.bfloat16, device=dev)) for _ in range(layers)]
+    req = torch.arange(B, dtype=torch.int32, device=dev).repeat_interleave(k).contiguous()
+    pos = torch.arange(k, dtype=torch.int32, device=dev).repeat(B).contiguous()
+    f = torch.empty((T, r), dtype=torch.float16, device=dev)
+    kv = torch.empty((T, 2 * Hkv * dh), dtype=torch.float32, device=dev)
+    ws = torch.empty(max(hs.hspec_gemm_workspace_bytes(T, r, cfg["n_fuse"] * D),
+                         hs.hspec_gemm_workspace_bytes(T, 2 * Hkv * dh, r)), dtype=torch.uint8, device=dev)
+
+    def once():
+        hs.hspec_op_gemm(h, w_fuse, f, workspace=ws)
+        for l in range(layers):
+            hs.hspec_op_gemm(f, w_kv[l], kv, workspace=ws)
+            hs.hspec_op_kv_inject_write(kv.view(T, 2, Hkv, dh), kw, req, pos, page_table, pools[l][0], pools[l][1],
+                                        cfg["rope_theta"], cfg["rms_eps"], True)
+    for _ in range(3):
+        once()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        once()
+    e1.record()
+    torch.cuda.synchronize()
+    return dict(positions_per_step=T, layers=layers, ms_per_step=round(e0.elapsed_time(e1) / reps, 4),
+                cache_bytes_added_per_step=T * layers * 2 * Hkv * dh * 2,
+                note="fusion GEMM + per-layer K/V GEMM + paged bf16 cache write for k new positions per request; "
+                     "the draft step measured above does none of this and keeps no drafter-side cache")
+
+
 def cpu_baseline(cfg_name, k_rows=None, rank=0):
     """Times the oracle as it stands on one request (median context) of the workload, on the host cores."""
     from oracle import hspec_oracle as O
@@ -416,6 +465,12 @@ def main_ours(args):
     }
     del head["_keep"]
     torch.cuda.empty_cache()
+    if world == 1 and not args.lean:
+        try:
+            line["kv_injection_counterexample"] = kv_injection_counterexample(head["cfg"])
+        except Exception as exc:                   # a side measurement must not cost the bench line
+            print(f"[bench] KV-injection counter-example skipped: {exc}", file=sys.stderr)
+        torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cb, _ = cpu_baseline(args.workload)
         cb.pop("ids")

@@ -246,6 +246,18 @@ int hspec_op_markov_head(float* logits, int64_t ld, const void* W_in, const void
                          const int32_t* id_map, int32_t* ids, int32_t B, int32_t k, int32_t Vd, int32_t r, int32_t write_logits,
                          void* workspace, size_t workspace_bytes, void* stream);
 size_t hspec_markov_workspace_bytes(int32_t B, int32_t Vd, int32_t r);
+/* The cache write of the KV-injecting block drafters the paper compares with (Sec. 2.2 "KV injection in block
+ * drafting"), kept as a measured counter-example to the drafter-side KV bytes the draft step avoids; the draft step
+ * itself never calls it.  For T new positions: key rows get the per-head RMSNorm (if k_norm) and rotate-half RoPE at
+ * their position, value rows are converted as they are, and both are stored as bf16 in a drafter-side paged cache.
+ *   kv fp32 device [T, 2, Hkv, dh] (projected keys | values, e.g. from hspec_op_gemm); k_norm_w fp32 [dh] or NULL
+ *   req, pos int32 device [T]: request (page-table row) and absolute position of each row
+ *   page_table int32 device [*, page_table_stride]; k_pool, v_pool bf16 device [num_pages, page_size, Hkv, dh], written
+ *   in place at (page_table[req, pos / page_size], pos % page_size); all other entries keep their bits.
+ * Two rows with the same (req, pos) race. */
+int hspec_op_kv_inject_write(const float* kv, const float* k_norm_w, const int32_t* req, const int32_t* pos,
+                             const int32_t* page_table, int32_t page_table_stride, void* k_pool, void* v_pool, int32_t T,
+                             int32_t Hkv, int32_t dh, int32_t page_size, float theta, float eps, int32_t k_norm, void* stream);
 /* RMSNorm over the last axis: y fp16 [M, n] = x fp32 [M, n] / sqrt(mean(x^2) + eps) * w. */
 int hspec_op_rmsnorm(const float* x, const float* w, void* y_f16, int32_t M, int32_t n, float eps, void* stream);
 /* Mamba-2 mixer core for B requests x k rows (Sec. 3.3.1): causal depthwise conv + SiLU on xBC (zero left

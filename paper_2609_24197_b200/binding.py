@@ -23,6 +23,7 @@ EXPORTS = [
     "hspec_op_lm_head_argmax", "hspec_op_lm_head_argmax_noalloc", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
     "hspec_op_accept", "hspec_op_token_probs", "hspec_op_markov_head", "hspec_markov_workspace_bytes",
+    "hspec_op_kv_inject_write",
 ]
 
 
@@ -107,6 +108,7 @@ def load_library(path=None):
     lib.hspec_op_markov_head.argtypes = [vp, i64, vp, vp, i32, vp, vp, vp, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.hspec_markov_workspace_bytes.argtypes = [i32, i32, i32]
     lib.hspec_markov_workspace_bytes.restype = sz
+    lib.hspec_op_kv_inject_write.argtypes = [vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, i32, i32, f32, f32, i32, vp]
     lib.hspec_op_mamba_scan.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, sz, vp]
     lib.hspec_scan_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     lib.hspec_scan_workspace_bytes.restype = sz
@@ -307,6 +309,15 @@ def hspec_op_markov_head(logits, W_in, W_out, last_token, id_map, ids, B, k, wri
         _ptr(logits, torch.float32), logits.shape[1], _ptr(W_in), _ptr(W_out, W_in.dtype), _DT[W_in.dtype],
         _ptr(last_token, torch.int32), _ptr(id_map, torch.int32), _ptr(ids, torch.int32), B, k, Vd, r, int(write_logits),
         _ptr(workspace), workspace.numel() * workspace.element_size(), _stream()), None, "hspec_op_markov_head")
+
+
+def hspec_op_kv_inject_write(kv, k_norm_w, req, pos, page_table, k_pool, v_pool, theta, eps, k_norm=True):
+    """The comparison drafters' cache write: fp32 rows [T, 2, Hkv, dh] -> bf16 paged pools, in place (Sec. 2.2)."""
+    T, _, Hkv, dh = kv.shape
+    _check(load_library().hspec_op_kv_inject_write(
+        _ptr(kv, torch.float32), _ptr(k_norm_w, torch.float32), _ptr(req, torch.int32), _ptr(pos, torch.int32),
+        _ptr(page_table, torch.int32), page_table.shape[1], _ptr(k_pool, torch.bfloat16), _ptr(v_pool, torch.bfloat16), T, Hkv,
+        dh, k_pool.shape[1], float(theta), float(eps), int(bool(k_norm)), _stream()), None, "hspec_op_kv_inject_write")
 
 
 def hspec_op_rmsnorm(x, w, y, eps):

@@ -117,6 +117,48 @@ __global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* 
   }
 }
 
+// The comparison drafters' cache write (Sec. 2.2 "KV injection in block drafting"): one warp per (new position, head).
+// Key heads: optional RMSNorm over dh, rotate-half RoPE at the position, bf16, into the paged key pool; value heads:
+// bf16 into the paged value pool.  Row t belongs to request req[t] and sits at absolute position pos[t].
+__global__ void kv_inject_write_kernel(const float* __restrict__ kv, const float* __restrict__ kw,
+                                       const float* __restrict__ inv_freq, const int32_t* __restrict__ req,
+                                       const int32_t* __restrict__ pos, const int32_t* __restrict__ page_table,
+                                       int page_table_stride, __nv_bfloat16* __restrict__ k_pool,
+                                       __nv_bfloat16* __restrict__ v_pool, int Hkv, int dh, int page_size, float eps,
+                                       int k_norm, int n_pairs) {
+  const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (pair >= n_pairs) return;
+  const int t = pair / (2 * Hkv), hh = pair % (2 * Hkv);
+  const int lane = threadIdx.x & 31;
+  const float* src = kv + (size_t(t) * 2 * Hkv + hh) * dh;
+  const int p = pos[t];
+  const int page = page_table[size_t(req[t]) * page_table_stride + p / page_size];
+  const size_t slot = (size_t(page) * page_size + p % page_size) * Hkv;
+  if (hh >= Hkv) {                                    // values: plain conversion
+    __nv_bfloat16* dst = v_pool + (slot + (hh - Hkv)) * dh;
+    for (int d = lane; d < dh; d += 32) dst[d] = __float2bfloat16_rn(src[d]);
+    return;
+  }
+  const int half = dh / 2;
+  float inv = 1.f;
+  if (k_norm) {
+    float ss = 0.f;
+    for (int d = lane; d < dh; d += 32) { const float v = src[d]; ss += v * v; }
+    for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    inv = rsqrtf(ss / float(dh) + eps);
+  }
+  const float fp = float(p);
+  __nv_bfloat16* dst = k_pool + (slot + hh) * dh;
+  for (int j = lane; j < half; j += 32) {
+    float v1 = src[j] * inv, v2 = src[j + half] * inv;
+    if (k_norm) { v1 *= kw[j]; v2 *= kw[j + half]; }
+    float sn, cs;
+    sincosf(fp * inv_freq[j], &sn, &cs);
+    dst[j] = __float2bfloat16_rn(v1 * cs - v2 * sn);
+    dst[j + half] = __float2bfloat16_rn(v2 * cs + v1 * sn);
+  }
+}
+
 __global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F) {
   const long long total = (long long)M * F;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
@@ -181,6 +223,19 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
   qk_norm_rope_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(qkv, qw, kw, tab, ctx_lens, (__nv_bfloat16*)q,
                                                              (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps,
                                                              qk_norm, n_pairs);
+  return cudaGetLastError();
+}
+
+cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32_t* req, const int32_t* pos,
+                                   const int32_t* page_table, int page_table_stride, void* k_pool, void* v_pool, int T,
+                                   int Hkv, int dh, int page_size, float theta, float eps, int k_norm, cudaStream_t stream) {
+  if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
+  const float* tab = rope_table(theta, dh, stream);
+  if (!tab) return cudaErrorMemoryAllocation;
+  const int n_pairs = T * 2 * Hkv;
+  kv_inject_write_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(kv, kw, tab, req, pos, page_table, page_table_stride,
+                                                                (__nv_bfloat16*)k_pool, (__nv_bfloat16*)v_pool, Hkv, dh,
+                                                                page_size, eps, k_norm, n_pairs);
   return cudaGetLastError();
 }
 

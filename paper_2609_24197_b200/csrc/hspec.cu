@@ -696,6 +696,18 @@ int hspec_op_token_probs(const float* logits, int64_t ld, const int32_t* ids, fl
   return HSPEC_OK;
 }
 
+int hspec_op_kv_inject_write(const float* kv, const float* k_norm_w, const int32_t* req, const int32_t* pos,
+                             const int32_t* page_table, int32_t page_table_stride, void* k_pool, void* v_pool, int32_t T,
+                             int32_t Hkv, int32_t dh, int32_t page_size, float theta, float eps, int32_t k_norm, void* stream) {
+  if (!kv || !req || !pos || !page_table || !k_pool || !v_pool || (k_norm && !k_norm_w) || T < 1 || Hkv < 1 || dh < 2 ||
+      page_size < 1 || page_table_stride < 1)
+    return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_kv_inject_write: bad argument");
+  std::string errtxt;
+  OP_TRY(kv_inject_write_launch(kv, k_norm_w, req, pos, page_table, page_table_stride, k_pool, v_pool, T, Hkv, dh, page_size,
+                                theta, eps, k_norm, reinterpret_cast<cudaStream_t>(stream)));
+  return HSPEC_OK;
+}
+
 size_t hspec_markov_workspace_bytes(int32_t B, int32_t Vd, int32_t r) {
   if (B < 1 || Vd < 1 || r < 1) return 0;
   return markov_workspace_bytes(B, Vd, r);

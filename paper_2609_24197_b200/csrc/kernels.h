@@ -112,6 +112,9 @@ struct MarkovCall {
   void* ws;                         // markov_workspace_bytes(B, Vd, r)
   uint32_t* status;
 };
+cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32_t* req, const int32_t* pos,
+                                   const int32_t* page_table, int page_table_stride, void* k_pool, void* v_pool, int T,
+                                   int Hkv, int dh, int page_size, float theta, float eps, int k_norm, cudaStream_t stream);
 cudaError_t accept_launch(const float* pt, const float* pd, const float* alpha, int* n_accept, int B, int k, cudaStream_t stream);
 cudaError_t token_probs_launch(const float* logits, long long ld, const int* ids, float* p, int M, int V, cudaStream_t stream);
 size_t markov_workspace_bytes(int B, int Vd, int r);

@@ -134,3 +134,54 @@ def test_markov_strong_table_changes_the_draft(hs):
 def test_markov_full_vocab_rank_256(hs):
     """Serving shape: 152 064-token vocabulary, rank 256, 16 positions; sampled requests against the oracle."""
     _markov_case(hs, B=4, k=16, V=152064, Vd=152064, r=256, seed=6)
+
+
+# --------------------------------------------------------------------------- KV-injection cache write (counter-example)
+
+@pytest.mark.parametrize("Hkv,dh,k_norm", [(2, 64, True), (8, 128, True), (1, 128, False)])
+def test_kv_inject_write(hs, Hkv, dh, k_norm):
+    """Projected key / value rows of new positions -> a drafter-side paged bf16 cache: values bit-exact, keys within
+    bf16 rounding of the oracle's norm + RoPE, every slot that is not addressed keeps its bits."""
+    import synth
+    from harness import assert_bf16_close, bf16_round
+    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
+    ctx = [40, 0, 333, 17]
+    batch = synth.make_request_batch(cfg, ctx_lens=ctx, device="cuda", extra_pages=3)
+    k_pool, v_pool = batch["k_pools"][0].clone(), batch["v_pools"][0].clone()
+    before_k, before_v = to_np(k_pool).copy(), to_np(v_pool).copy()
+    # each request appends a few positions after its context (position = ctx_len + i), as a verification step would
+    new = [3, 5, 1, 16]
+    req = torch.tensor([b for b, n in enumerate(new) for _ in range(n)], dtype=torch.int32)
+    pos = torch.tensor([ctx[b] + i for b, n in enumerate(new) for i in range(n)], dtype=torch.int32)
+    T = int(req.numel())
+    g = _gen(Hkv * 1000 + dh)
+    kv = torch.randn((T, 2, Hkv, dh), generator=g)
+    kw = 1.0 + 0.1 * torch.randn(dh, generator=g)
+    # the page table must cover the appended positions: give every request enough pages from the spare ones
+    pt = batch["page_table"].clone()
+    need = max((ctx[b] + new[b] + 15) // 16 for b in range(4))
+    if pt.shape[1] < need:
+        pt = torch.nn.functional.pad(pt, (0, need - pt.shape[1]))
+    used = set(int(x) for b in range(4) for x in pt[b, :(ctx[b] + 15) // 16].tolist())
+    spare = [p for p in range(k_pool.shape[0]) if p not in used]
+    for b in range(4):
+        for j in range((ctx[b] + 15) // 16, (ctx[b] + new[b] + 15) // 16):
+            pt[b, j] = spare.pop()
+    pt = pt.contiguous()
+    hs.hspec_op_kv_inject_write(kv.cuda(), kw.cuda() if k_norm else None, req.cuda(), pos.cuda(), pt, k_pool, v_pool,
+                                1.0e6, 1e-6, k_norm)
+    torch.cuda.synchronize()
+    K_ref, V_ref = ao.kv_inject_rows(kv.numpy(), kw.numpy(), pos.numpy(), 1.0e6, eps=1e-6, k_norm=k_norm)
+    ok, ov = before_k.copy().view(np.uint16), before_v.copy().view(np.uint16)      # bf16 bit patterns
+    got_k, got_v = to_np(k_pool), to_np(v_pool)
+    ptab = pt.cpu().numpy()
+    touched = np.zeros(got_k.shape[:2], dtype=bool)
+    from conftest import to_np as _to_np  # noqa: F401
+    widen = lambda a: (a.astype(np.uint32) << 16).view(np.float32)
+    for t in range(T):
+        page, slot = int(ptab[int(req[t]), int(pos[t]) // 16]), int(pos[t]) % 16
+        touched[page, slot] = True
+        np.testing.assert_array_equal(widen(got_v[page, slot]), bf16_round(V_ref[t]))
+        assert_bf16_close(widen(got_k[page, slot]), K_ref[t], f"injected key row {t}")
+    np.testing.assert_array_equal(got_k[~touched], before_k[~touched])
+    np.testing.assert_array_equal(got_v[~touched], before_v[~touched])
