@@ -61,3 +61,23 @@ def test_two_rank_replicas_take_the_max_time():
     mp.spawn(_worker, args=(2, port, out), nprocs=2, join=True)
     assert out[0][0] == 15.0 and out[1][0] == 15.0               # every rank sees the slowest rank's time
     assert out[0][1] == pytest.approx(2 * 128 * 16 / 15e-3)
+
+
+def test_reference_arm_prints_one_contract_line_on_cpu():
+    """`bench.py --impl reference` times the oracle on the host cores and prints one JSON line with the contract's keys
+    (run here on the tiny workload; no GPU involved)."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--impl", "reference", "--workload", "tiny",
+                          "--steps", "1", "--warmup", "0"], capture_output=True, text=True, timeout=600, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["value"] > 0 and line["higher_is_better"] is True
+    for key in ("metric", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "scaling", "vs_baseline", "dtype", "data",
+                "config", "cpu_baseline", "e2e"):
+        assert key in line, key
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] >= 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert line["config"]["workload"] == "tiny"
