@@ -243,6 +243,16 @@ def test_attention_shapes_and_long_contexts(hs, k, Hq, Hkv, dh):
     _attn_case(hs, 4, k, Hq, Hkv, dh, [300, 1000, 4099, 2047], 2048, 0, seed=3)
 
 
+def test_attention_many_short_requests_fill_the_work_list(hs):
+    """Persistent tcgen05 kernel: far more work items than SMs (each CTA walks several, most of them one ragged tile
+    long, a few multi-chunk), and a windowed variant whose chunk grid starts at a page-aligned offset."""
+    g = torch.Generator().manual_seed(11)
+    ctxs = torch.randint(0, 200, (300,), generator=g).tolist()
+    ctxs[7], ctxs[123], ctxs[299] = 0, 3000, 1537
+    _attn_case(hs, 300, 4, 8, 4, 128, ctxs, 0, 256, seed=4, poison=False)
+    _attn_case(hs, 300, 4, 8, 4, 128, ctxs, 100, 128, seed=5, poison=False)
+
+
 def test_attention_page_permutation_is_bit_exact(hs):
     B, k, Hq, Hkv, dh = 2, 4, 8, 2, 128
     cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
