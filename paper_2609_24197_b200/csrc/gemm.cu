@@ -125,6 +125,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                         // TMEM lane quarter this warp may read
+    if (g.addend != nullptr) {
+      // the addend rows of this tile do not depend on the accumulator: pull this warp's 128-byte piece of every
+      // row into L2 while the main loop runs (one line per lane and pass)
+      const int n_w = tile_n * TILE_W + q * 32;
+      if (n_w < g.N_out)
+        for (int c = lane; c < g.BN; c += 32) {
+          const int m = tile_m * g.BN + c;
+          if (m < g.M) asm volatile("prefetch.global.L2 [%0];" ::"l"(g.addend + size_t(m) * g.ld_add + n_w));
+        }
+    }
     bool ok = mbar_wait(smem_u32(&tail->tmem_full), 0);
     if (!ok) atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
     tc_fence_after();
