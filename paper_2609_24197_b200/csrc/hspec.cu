@@ -322,7 +322,17 @@ int hspec_init(const hspec_config* cfg, hspec_handle** out) {
 
 size_t hspec_workspace_bytes(const hspec_config* cfg) {
   if (!cfg || check_config(*cfg)) return 0;
-  return make_plan(*cfg, cfg->max_batch, cfg->max_k, cfg->max_pages_per_req * cfg->page_size).total;
+  // The layout of a step depends on its own (B, k): how the contexts are cut into chunks and how many K-slices a GEMM
+  // uses change at thresholds, so a smaller step can need MORE of some scratch buffer than the largest one.  The
+  // size handed out covers every (B, k) the handle accepts.
+  const int max_ctx = cfg->max_pages_per_req * cfg->page_size;
+  size_t total = 0;
+  for (int B = 1; B <= cfg->max_batch; ++B)
+    for (int k = 1; k <= cfg->max_k; ++k) {
+      const size_t t = make_plan(*cfg, B, k, max_ctx).total;
+      if (t > total) total = t;
+    }
+  return total;
 }
 
 int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {

@@ -217,3 +217,15 @@ def test_step_is_capturable_in_a_cuda_graph_and_replays_bit_exactly():
     assert not torch.equal(ids_new, ids_direct)
     assert drafter.stats()["device_status"] == 0
     drafter.close()
+
+
+def test_smaller_batch_than_planned_fits_the_workspace():
+    """The scratch layout depends on the step's own (B, k) (context chunking and K-slices change at thresholds), so the
+    size reported for (max_batch, max_k) must cover every smaller step too: 73 requests on a handle made for 128,
+    with contexts long enough that the two batch sizes cut them into different chunk lengths."""
+    cfg = synth.derived(dict(MID, Hq=8, Hkv=8, B=73))
+    ctx = [4200 + 13 * b for b in range(73)]
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=ctx, max_batch=128, max_k=16, poison_tail=False, extra_pages=0)
+    r = check_step(cfg, drafter, w, batch, 16, requests=[0, 72], what="B=73 of 128")
+    assert r["ids_compared"] > 0
+    drafter.close()
