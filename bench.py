@@ -445,7 +445,9 @@ def main_ours(args):
         "metric": METRIC, "value": round(units / (head["ms_per_step"] * 1e-3), 1), "unit": "draft tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": s["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16 tensor-core operands (bf16 weights widened at load), f32 accumulate; bf16 target KV",
+        "dtype": "f16",
+        "dtype_note": "f16 tensor-core operands (bf16 weights widened exactly at load), f32 accumulate, f32 residual / scan / "
+                      "softmax; the target KV is read as bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "B": head["B"], "k": head["k"], "ctx_sum": head["ctx_sum"],
                    "ctx_max": head["ctx_max"], "window": head["cfg"]["window"],
@@ -532,7 +534,7 @@ def main_reference(args):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": "draft tokens/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(sec * 1e3, 2), "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f32 (numpy oracle on host cores)", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "dtype_note": "numpy oracle on the host cores", "data": "synthetic",
         "config": {"workload": args.workload, "sample": sample},
         "cpu_baseline": {"value": round(value, 3), "unit": "draft tokens/s", "cores": cores, "kind": "oracle",
                          "sample": sample},
