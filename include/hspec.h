@@ -171,7 +171,11 @@ size_t hspec_workspace_bytes(const hspec_config* cfg);
 /* Copies n named device tensors into library-owned device memory (may be called several times; synchronises the
  * device).  Shapes are checked against the config. */
 int hspec_load_weights(hspec_handle* h, const hspec_tensor* tensors, int32_t n);
-/* Enqueues one block-parallel draft step (Sec. 3.3) on in->stream.  Needs every tensor loaded. */
+/* Enqueues one block-parallel draft step (Sec. 3.3) on in->stream.  Needs every tensor loaded.  The first call on a
+ * device builds a small RoPE table (one allocation, one copy) and sets kernel attributes; every later call only
+ * launches kernels on the stream, so a warmed-up step may be captured in a CUDA graph and replayed: the replay reads
+ * the current contents of the same input buffers.  The workspace must hold hspec_workspace_bytes(cfg) bytes, which
+ * covers every (B, k) up to (max_batch, max_k). */
 int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* out);
 /* Frees the handle and its weight copies.  Pools and the workspace stay the caller's. */
 int hspec_destroy(hspec_handle* h);
