@@ -437,7 +437,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   for (int t = 0; t < k; ++t) {
     const float ct = __shfl_sync(0xffffffffu, cum, t);
     float w = 0.f;
-    if (lane <= t) w = expf(ct - cum) * dt * CB[t * ROWS + lane];
+    if (lane <= t) w = __expf(ct - cum) * dt * CB[t * ROWS + lane];
     if (lane < ROWS) Wh[t * (ROWS + 1) + lane] = w;
   }
   __syncwarp();
@@ -483,7 +483,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int t = mt * 16 + gq + half * 8;
-      const float dec = expf(__shfl_sync(0xffffffffu, cum, t & 31));
+      const float dec = __expf(__shfl_sync(0xffffffffu, cum, t & 31));
       if (t >= k) continue;
       const size_t row = row0 + t;
       float2 z[NT];
