@@ -29,7 +29,11 @@ struct Gemm2Args {
   int BNT;                 // activation rows per cluster tile (128 or 256); each CTA stages BNT/2
   int k_tiles, stages;
   int n_tiles_w, n_tiles_m;
-  int splits, k_tiles_per_split;   // K-slices per tile (work unit = tile x slice); > 1: fp32 partials to `out`
+  // Work units: the first n_full_tiles tiles run whole (full waves of the SM pairs); each of the remaining "tail" tiles
+  // is cut into tail_splits K-slices so that the last, partly filled wave keeps every pair busy.  A slice stores an
+  // fp32 partial tile to `part` ([tail tile][slice][activation row][256 weight rows]); a second kernel sums them.
+  int n_full_tiles, tail_splits, k_tiles_per_split;
+  float* part;
   int f16, mode;
   void* out;
   long long ldo;
@@ -117,7 +121,17 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();
   const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
-  const int total_units = g.n_tiles_w * g.n_tiles_m * g.splits;   // unit u = tile u / splits, K-slice u % splits
+  const int total_tiles = g.n_tiles_w * g.n_tiles_m;
+  const int total_units = g.n_full_tiles + (total_tiles - g.n_full_tiles) * g.tail_splits;
+  // unit u < n_full_tiles: tile u, all of K; else tail tile n_full_tiles + v / tail_splits, K-slice v % tail_splits
+  auto decode = [&](int u, int& tile, int& sp, int& kt_begin, int& kt_end) {
+    if (u < g.n_full_tiles) { tile = u; sp = -1; kt_begin = 0; kt_end = g.k_tiles; return; }
+    const int v = u - g.n_full_tiles;
+    tile = g.n_full_tiles + v / g.tail_splits;
+    sp = g.tail_splits > 1 ? v % g.tail_splits : -1;          // -1: the unit is a whole tile with the real epilogue
+    kt_begin = (v % g.tail_splits) * g.k_tiles_per_split;
+    kt_end = min(g.k_tiles, kt_begin + g.k_tiles_per_split);
+  };
   const uint32_t tmem_cols = 2u * uint32_t(g.BNT);           // two accumulators (256 or 512 columns)
 
   if (threadIdx.x == 0) {
@@ -154,10 +168,10 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       uint32_t it = 0;
       bool ok = true;
       for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters) {
-        const int tile = unit / g.splits, sp = unit % g.splits;
+        int tile, sp, kt_begin, kt_end;
+        decode(unit, tile, sp, kt_begin, kt_end);
         const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
-        const int kt_end = min(g.k_tiles, (sp + 1) * g.k_tiles_per_split);
-        for (int kt = sp * g.k_tiles_per_split; kt < kt_end; ++kt, ++it) {
+        for (int kt = kt_begin; kt < kt_end; ++kt, ++it) {
           const int s = it % g.stages;
           const uint32_t lap = it / g.stages;
           if (lap > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (lap - 1) & 1)) {
@@ -180,8 +194,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       uint32_t it = 0, tile_count = 0;
       bool ok = true;
       for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters, ++tile_count) {
-        const int sp = unit % g.splits;
-        const int kt_begin = sp * g.k_tiles_per_split, kt_end = min(g.k_tiles, (sp + 1) * g.k_tiles_per_split);
+        int tile, sp, kt_begin, kt_end;
+        decode(unit, tile, sp, kt_begin, kt_end);
         const uint32_t acc = tile_count & 1, use = tile_count >> 1;
         if (use > 0 && !mbar_wait(smem_u32(&tail->tmem_empty[acc]), (use - 1) & 1)) { ok = false; break; }
         tc_fence_after();
@@ -210,8 +224,10 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t empty_leader0 = mapa_rank(smem_u32(&tail->tmem_empty[0]), 0);
     const uint32_t empty_leader1 = mapa_rank(smem_u32(&tail->tmem_empty[1]), 0);
     for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters, ++tile_count) {
-      const int tile = unit / g.splits, sp = unit % g.splits;
+      int tile, sp, kt_begin, kt_end;
+      decode(unit, tile, sp, kt_begin, kt_end);
       const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
+      const int mode = sp >= 0 ? EPI_PARTIAL_F32 : g.mode;
       const uint32_t acc = tile_count & 1, use = tile_count >> 1;
       if (!mbar_wait(smem_u32(&tail->tmem_full[acc]), use & 1)) {
         atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
@@ -225,18 +241,24 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       const int m0 = tm * g.BNT;
       const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT) + (uint32_t(q * 32) << 16);
       for (int c0 = 0; c0 < g.BNT; c0 += 16) {
-        if (m0 + c0 >= g.M && g.mode != EPI_ARGMAX) break;    // rows past M: nothing to store (warp-uniform)
+        if (m0 + c0 >= g.M && mode != EPI_ARGMAX) break;    // rows past M: nothing to store (warp-uniform)
         uint32_t r[16];
         tmem_ld16(tmem_acc + uint32_t(c0), r);
         tmem_ld_wait();
-        if (g.mode == EPI_STORE_F32 || g.mode == EPI_PARTIAL_F32) {
-          float* out = reinterpret_cast<float*>(g.out) + (g.mode == EPI_PARTIAL_F32 ? size_t(sp) * g.M * g.ldo : 0);
+        if (mode == EPI_PARTIAL_F32) {
+          // slice of a tail tile: [tail tile][slice][activation row of the tile][256 weight rows of the pair]
+          float* out = g.part + (size_t(tile - g.n_full_tiles) * g.tail_splits + sp) * size_t(g.BNT) * 256 +
+                       int(rank) * 128 + q * 32 + lane;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) out[size_t(c0 + j) * 256] = __uint_as_float(r[j]);
+        } else if (mode == EPI_STORE_F32) {
+          float* out = reinterpret_cast<float*>(g.out);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __uint_as_float(r[j]);
           }
-        } else if (g.mode == EPI_ACCUM_F32) {
+        } else if (mode == EPI_ACCUM_F32) {
           // read-modify-write of the residual stream: issue the 16 loads together, then add and store
           float* out = reinterpret_cast<float*>(g.out);
           float old[16];
@@ -250,17 +272,17 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int m = m0 + c0 + j;
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = old[j] + __uint_as_float(r[j]);
           }
-        } else if (g.mode == EPI_SWIGLU_F16) {
+        } else if (mode == EPI_SWIGLU_F16) {
           const int f = tile_n128 * 64 + q * 16 + (lane & 15);
           swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane);
-        } else if (g.mode == EPI_STORE_F16) {
+        } else if (mode == EPI_STORE_F16) {
           __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2half_rn(__uint_as_float(r[j]));
           }
-        } else if (g.mode == EPI_STORE_BF16) {
+        } else if (mode == EPI_STORE_BF16) {
           __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(g.out);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
@@ -285,7 +307,7 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       // accumulator drained: hand it back to the MMA issuer in the leader CTA
       tc_fence_before();
       mbar_arrive_cluster(acc ? empty_leader1 : empty_leader0);
-      if (g.mode == EPI_ARGMAX) {
+      if (mode == EPI_ARGMAX) {
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const int t = threadIdx.x - 64;
         for (int c = t; c < g.BNT; c += 128) {
@@ -314,6 +336,41 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   }
 }
 
+// Sums the K-slices of the tail tiles in slice order (deterministic) and applies the real epilogue.
+// Block = (tail tile, group of 4 activation rows); thread = one of the pair's 256 weight rows; all slices' loads are
+// issued before the first add.
+constexpr int TAIL_MAX_SPLITS = 8, TAIL_ROWS = 4;
+__global__ void __launch_bounds__(256)
+gemm2_tail_reduce_kernel(Gemm2Args g) {
+  const int tail = blockIdx.x, tile = g.n_full_tiles + tail;
+  const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
+  const int n = tn * 256 + threadIdx.x;
+  const int m_base = tm * g.BNT + blockIdx.y * TAIL_ROWS;
+  if (m_base >= g.M) return;
+  const float* src = g.part + size_t(tail) * g.tail_splits * g.BNT * 256 + size_t(blockIdx.y) * TAIL_ROWS * 256 + threadIdx.x;
+  float v[TAIL_MAX_SPLITS][TAIL_ROWS];
+#pragma unroll
+  for (int sp = 0; sp < TAIL_MAX_SPLITS; ++sp)
+#pragma unroll
+    for (int j = 0; j < TAIL_ROWS; ++j)
+      v[sp][j] = (sp < g.tail_splits && m_base + j < g.M) ? __ldcs(src + (size_t(sp) * g.BNT + j) * 256) : 0.f;
+  if (n >= g.N_out) return;
+#pragma unroll
+  for (int j = 0; j < TAIL_ROWS; ++j) {
+    const int m = m_base + j;
+    if (m >= g.M) break;
+    float acc = 0.f;
+#pragma unroll
+    for (int sp = 0; sp < TAIL_MAX_SPLITS; ++sp)
+      if (sp < g.tail_splits) acc += v[sp][j];
+    const size_t o = size_t(m) * g.ldo + n;
+    if (g.mode == EPI_STORE_F32) reinterpret_cast<float*>(g.out)[o] = acc;
+    else if (g.mode == EPI_ACCUM_F32) reinterpret_cast<float*>(g.out)[o] += acc;
+    else if (g.mode == EPI_STORE_F16) reinterpret_cast<__half*>(g.out)[o] = __float2half_rn(acc);
+    else reinterpret_cast<__nv_bfloat16*>(g.out)[o] = __float2bfloat16_rn(acc);
+  }
+}
+
 int g_smem_optin2 = -1;
 
 }  // namespace
@@ -326,10 +383,10 @@ bool gemm2_preferred(int M, int n_out) {
   return !off && M >= 256;
 }
 
-// Tile width (activation rows per cluster tile) and number of K-slices per tile that finish soonest by a simple
-// model: waves of the 74 SM pairs x k-steps per wave x cost of a k-step, plus a fixed cost per wave (pipeline fill,
-// the last epilogue) and, with slices, the pass that sums the fp32 partials.  One cost unit ~ 2.2 ns (a k-step of a
-// 256-wide pair tile = 256 units ~ 0.56 us).
+// Tile width (activation rows per pair tile) and the number of K-slices for the tiles of the last, partly filled wave,
+// by a simple model: full waves of the 74 SM pairs x k-steps x cost of a k-step, plus the tail wave (k-steps / slices),
+// a fixed cost per wave (pipeline fill, the last epilogue) and, with slices, the pass that sums the partial tiles.
+// One cost unit ~ 2.2 ns (a k-step of a 256-wide pair tile = 256 units ~ 0.56 us).
 void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out) {
   const int tw = (n_out + 255) / 256;
   const int k_tiles = (K + TILE_K - 1) / TILE_K;
@@ -337,22 +394,27 @@ void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out
   double best_cost = 1e30;
   int best_bnt = 256, best_s = 1;
   for (int bnt : {256, 128}) {
-    for (int s : {1, 2, 3, 4, 6, 8}) {
-      if (s > 1 && (!may_split || k_tiles / s < 8)) continue;
+    const int tiles = tw * ((M + bnt - 1) / bnt);
+    const int full_waves = tiles / 74, tail = tiles % 74;
+    // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
+    // measured, the narrow tile runs ~1.5x slower per flop
+    const double kstep = bnt * (bnt == 128 ? 1.5 : 1.0);
+    for (int s = 1; s <= 8; ++s) {
+      if (s > 1 && (!may_split || tail == 0 || tail * s > 74 || k_tiles / s < 8)) continue;
       const int kps = (k_tiles + s - 1) / s;
       if (s > 1 && kps * (s - 1) >= k_tiles) continue;         // an empty last slice
-      const long long units = (long long)tw * ((M + bnt - 1) / bnt) * s;
-      const long long waves = (units + 73) / 74;
-      // a 128-wide tile needs 96 B/clk of shared-memory fill per SM at full MMA rate, a 256-wide one 64 B/clk:
-      // measured, the narrow tile runs ~1.5x slower per flop
-      double cost = double(waves) * kps * bnt * (bnt == 128 ? 1.5 : 1.0) + double(waves) * 1500.0;
-      if (s > 1) cost += (double(s + 2) * M * n_out * 4.0 / 5.0e6 + 4.0) * 455.0;
+      double cost = double(full_waves) * (k_tiles * kstep + 1500.0);
+      if (tail > 0) cost += kps * kstep + 1500.0;
+      if (s > 1) cost += (double(s + 2) * tail * bnt * 256 * 4.0 / 4.0e6 + 4.0) * 455.0;
       if (cost < best_cost) { best_cost = cost; best_bnt = bnt; best_s = s; }
     }
   }
   *bnt_out = best_bnt;
   *splits_out = best_s;
 }
+
+// Scratch for the tail tiles' partials: at most one wave of pair tiles, each up to 256 x 256 fp32, times the slices.
+size_t gemm2_tail_bytes() { return size_t(74) * 256 * 256 * 4; }
 
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (g_smem_optin2 < 0) {
@@ -366,25 +428,23 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.M = c.M; g.N_out = c.n_out; g.K = c.K;
   int splits = 1;
   gemm2_pick(c.M, c.n_out, c.K, c.mode, &g.BNT, &splits);
-  if (c.splits > 0) {                                     // the caller fixed the number of K-slices
-    splits = c.splits;
-    if (splits > 1 && (c.mode == EPI_ARGMAX || c.mode == EPI_SWIGLU_F16)) { if (err) *err = "this epilogue cannot be K-sliced"; return cudaErrorInvalidValue; }
-  }
   g.k_tiles = (c.K + TILE_K - 1) / TILE_K;
-  if (splits > g.k_tiles) splits = g.k_tiles;
-  g.k_tiles_per_split = (g.k_tiles + splits - 1) / splits;
-  splits = (g.k_tiles + g.k_tiles_per_split - 1) / g.k_tiles_per_split;   // no empty slice
-  g.splits = splits;
   g.n_tiles_w = (c.n_out + 255) / 256;
   g.n_tiles_m = (c.M + g.BNT - 1) / g.BNT;
+  const int tiles = g.n_tiles_w * g.n_tiles_m;
+  const int tail = tiles % 74;
+  if (c.splits > 0) splits = c.splits;                    // the caller fixed the number of K-slices (of the tail tiles)
+  if (c.mode == EPI_ARGMAX || c.mode == EPI_SWIGLU_F16 || tail == 0) splits = 1;
+  if (splits > g.k_tiles) splits = g.k_tiles;
+  if (splits > TAIL_MAX_SPLITS) splits = TAIL_MAX_SPLITS;
+  while (splits > 1 && size_t(tail) * splits * g.BNT * 256 * 4 > c.splitk_ws_bytes) --splits;   // never more than the scratch holds
+  if (c.splitk_ws == nullptr) splits = 1;
+  g.k_tiles_per_split = (g.k_tiles + splits - 1) / splits;
+  splits = (g.k_tiles + g.k_tiles_per_split - 1) / g.k_tiles_per_split;   // no empty slice
+  g.tail_splits = splits;
+  g.n_full_tiles = splits > 1 ? tiles - tail : tiles;
+  g.part = reinterpret_cast<float*>(c.splitk_ws);
   g.f16 = c.f16 ? 1 : 0; g.mode = c.mode; g.out = c.out; g.ldo = c.ldo;
-  if (splits > 1) {
-    if (c.splitk_ws == nullptr || c.splitk_ws_bytes < gemm_splitk_bytes(c.M, c.n_out, splits)) {
-      if (err) *err = "K-slice workspace too small";
-      return cudaErrorInvalidValue;
-    }
-    g.mode = EPI_PARTIAL_F32; g.out = c.splitk_ws; g.ldo = c.n_out;
-  }
   if (c.addend != nullptr) { if (err) *err = "the 2-SM kernel has no addend epilogue"; return cudaErrorInvalidValue; }
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
   const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
@@ -395,7 +455,7 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.stages = stages;
   CUtensorMap tmB;
   if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BNT / 2, c.f16, err)) return cudaErrorInvalidValue;
-  const int total = g.n_tiles_w * g.n_tiles_m * splits;
+  const int total = g.n_full_tiles + (tiles - g.n_full_tiles) * splits;
   const int clusters = total < 74 ? total : 74;
   const size_t smem = size_t(stages) * stage_bytes + fixed;
   // profile name "gemm2:<what>" tells this kernel's launches from the one-CTA kernel's "gemm:<what>"
@@ -405,8 +465,12 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   gemm_2sm_kernel<<<2 * clusters, 192, smem, stream>>>(*c.tmW, tmB, g);
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
-  if (e == cudaSuccess && splits > 1)
-    e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk);
+  if (e == cudaSuccess && splits > 1) {
+    trk_begin(trk, "gemm2_tail_reduce", 0, double(splits + 1) * tail * g.BNT * 256 * 4);
+    gemm2_tail_reduce_kernel<<<dim3(tail, g.BNT / TAIL_ROWS), 256, 0, stream>>>(g);
+    trk_end(trk);
+    e = cudaGetLastError();
+  }
   return e;
 }
 

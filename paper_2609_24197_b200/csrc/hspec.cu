@@ -58,6 +58,7 @@ struct Plan {
 };
 
 size_t splitk_need(int M, int n_out, int K) {
+  if (gemm2_preferred(M, n_out)) return gemm2_tail_bytes();
   return gemm_splitk_bytes(M, n_out, gemm_pick_splits(M, n_out, K, kNumSMs));
 }
 
@@ -644,7 +645,7 @@ int hspec_get_profile(hspec_handle* h, hspec_prof_entry* out, int32_t max_entrie
   } while (0)
 
 size_t hspec_gemm_workspace_bytes(int32_t M, int32_t n_out, int32_t K) {
-  return gemm_splitk_bytes(M, n_out, 16) + size_t((n_out + 127) / 128) * M * 8 + 2048;
+  return gemm_splitk_bytes(M, n_out, 16) + gemm2_tail_bytes() + size_t((n_out + 127) / 128) * M * 8 + 2048;
 }
 
 int hspec_op_gemm(const void* x, const void* Wt, int32_t in_dtype, void* y, int32_t M, int32_t n_out, int32_t K, int64_t ldy,

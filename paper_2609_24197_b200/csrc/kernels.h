@@ -91,6 +91,7 @@ int gemm_pick_splits(int M, int n_out, int K, int num_sms, int mode = EPI_STORE_
 size_t gemm_splitk_bytes(int M, int n_out, int splits);
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 bool gemm2_preferred(int M, int n_out);        // many rows and at least one full round of cluster tiles
+size_t gemm2_tail_bytes();                     // scratch the 2-SM kernel's K-sliced tail wave may use
 void gemm2_pick(int M, int n_out, int K, int mode, int* bnt, int* splits);   // tile width and K-slices of the 2-SM kernel
 cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, void* out, long long ldo, int mode,
                                  cudaStream_t stream, Tracker* trk);
