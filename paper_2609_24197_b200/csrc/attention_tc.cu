@@ -59,8 +59,8 @@ struct __align__(8) AttnTcBars {
   uint64_t s_ready[2], p_ready[2];
   uint32_t tmem_base;
   uint32_t abort_flag;
-  __half xmax[2][2][128];  // [tile parity][column half][row]: half-row maxima exchanged between the two threads of a row
-                           // (1 KiB; one parity's 512 bytes are reused as a float per row for the final row-sum exchange)
+  float xmax[2][2][128];   // [tile parity][column half][row]: half-row maxima exchanged between the two threads of a row
+                           // (2 KiB; one parity's first 512 bytes are reused as a float per row for the final row-sum exchange)
 };
 
 // byte offset of (row, 16-byte chunk 0..15) inside a [128 x 128] bf16 operand tile stored as two K-major halves
@@ -548,16 +548,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           mx4[0] = fmaxf(mx4[0], s[j]); mx4[1] = fmaxf(mx4[1], s[j + 1]);
           mx4[2] = fmaxf(mx4[2], s[j + 2]); mx4[3] = fmaxf(mx4[3], s[j + 3]);
         }
-        // exchanged as fp16 (rounded UP, so the reference never undershoots): both threads of the row then hold the
-        // same two values and take the same decision; the reference maximum need not be the exact maximum
-        const __half mx_own = __float2half_ru(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])));
+        // both threads of the row then hold the same two values and take the same decision below
+        const float mx_own = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         TCLK(2)
         bars->xmax[gt & 1][hf][r_local] = mx_own;
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->x_ready[gt & 1]));       // bounded exchange between the eight softmax warps
         if (!mbar_wait(smem_u32(&bars->x_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
         // (past this barrier both threads of the row hold their scores in registers: P may overwrite the S columns)
-        const float mx = fmaxf(__half2float(mx_own), __half2float(bars->xmax[gt & 1][hf ^ 1][r_local])) * a.scale_log2;
+        const float mx = fmaxf(mx_own, bars->xmax[gt & 1][hf ^ 1][r_local]) * a.scale_log2;
         TCLK(3)
         // ---- reference maximum moves only when the row maximum outgrows it by 2^LAZY (same decision in both halves)
         float factor = 1.f;
@@ -605,7 +604,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       // ---- partial (m, l, O) of this chunk: the row sum is the sum of the two halves.
       // The exchange buffer of parity gt & 1 was last used two tiles ago and is not written again before every
       // softmax warp has signalled q_ready for the next item, i.e. after this read: 512 bytes = one float per row.
-      float* xl = reinterpret_cast<float*>(&bars->xmax[gt & 1][0][0]);
+      float* xl = &bars->xmax[gt & 1][0][0];
       float l_row = l_sum;
       if (hf == 1) {
         xl[r_local] = l_sum;
