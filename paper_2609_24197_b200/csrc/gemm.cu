@@ -77,7 +77,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (warp == 0) {
     if (lane == 0) {
-      const uint64_t pol_w = policy_evict_first();   // weights are streamed once per step
+      // weights are streamed once per step, unless the caller runs the same matrix again right away
+      const uint64_t pol_w = g.keep_w ? policy_evict_last() : policy_evict_first();
       const uint64_t pol_x = policy_evict_last();    // activations are re-read by every weight tile
       for (int i = 0; i < n_kt; ++i) {
         const int s = i % g.stages;
@@ -424,6 +425,7 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   g.status = c.status;
   g.f16 = c.f16 ? 1 : 0;
   g.logits = c.logits; g.addend = c.addend; g.ld_add = c.ld_add; g.part_val = c.part_val; g.part_idx = c.part_idx;
+  g.keep_w = c.keep_weights_in_l2 ? 1 : 0;
   g.ldo = c.ldo;
   if (splits > 1) {
     if (c.mode == EPI_ARGMAX) { if (err) *err = "LM-head epilogue cannot be K-sliced"; return cudaErrorInvalidValue; }

@@ -58,6 +58,7 @@ struct GemmArgs {       // kernel argument block
   float* logits;
   const float* addend;  // EPI_ARGMAX only (one-CTA kernel): value = acc + addend[m * ld_add + n] (may be null)
   long long ld_add;
+  int keep_w;           // weights loaded evict-last instead of evict-first
   float* part_val;
   int* part_idx;
   uint32_t* status;
@@ -78,6 +79,7 @@ struct GemmCall {       // host-side description of one y = x W^T
   float* logits;            // EPI_ARGMAX only (may be null)
   const float* addend;      // EPI_ARGMAX, one-CTA kernel only: fp32 [M, ld_add] added before the arg-max (may be null)
   long long ld_add;
+  bool keep_weights_in_l2;  // one-CTA kernel: the same W is used again by the next launch (keep it in L2 if it fits)
   float* part_val;
   int* part_idx;
   uint32_t* status;

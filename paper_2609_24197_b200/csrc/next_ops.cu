@@ -173,6 +173,7 @@ cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk
     g.logits = c.write_logits ? c.logits + size_t(i) * c.ld : nullptr;
     g.ldo = (long long)c.k * c.ld;
     g.part_val = part_val; g.part_idx = part_idx; g.status = c.status;
+    g.keep_weights_in_l2 = true;                            // W_out (78 MB at V = 152 064, r = 256) serves every position
     g.label = "markov";
     e = gemm_launch(g, stream, trk, err);
     if (e != cudaSuccess) return e;
