@@ -354,15 +354,24 @@ gemm2_tail_reduce_kernel(Gemm2Args g) {
 #pragma unroll
     for (int j = 0; j < TAIL_ROWS; ++j)
       v[sp][j] = (sp < g.tail_splits && m_base + j < g.M) ? __ldcs(src + (size_t(sp) * g.BNT + j) * 256) : 0.f;
-  if (n >= g.N_out) return;
+  const int lane = threadIdx.x & 31;
+  // SwiGLU epilogue: weight rows are interleaved in blocks of 16 (gate | up), so lanes l and l ^ 16 of a warp hold the
+  // gate and the up projection of feature f
+  const int f = (tn * 2 + (threadIdx.x >> 7)) * 64 + ((threadIdx.x >> 5) & 3) * 16 + (lane & 15);
 #pragma unroll
   for (int j = 0; j < TAIL_ROWS; ++j) {
     const int m = m_base + j;
-    if (m >= g.M) break;
+    if (m >= g.M) break;                                    // uniform over the block
     float acc = 0.f;
 #pragma unroll
     for (int sp = 0; sp < TAIL_MAX_SPLITS; ++sp)
       if (sp < g.tail_splits) acc += v[sp][j];
+    if (g.mode == EPI_SWIGLU_F16) {
+      const float up = __shfl_xor_sync(0xffffffffu, acc, 16);
+      if (lane < 16 && 2 * f < g.N_out) reinterpret_cast<__half*>(g.out)[size_t(m) * g.ldo + f] = __float2half_rn(silu_f(acc) * up);
+      continue;
+    }
+    if (n >= g.N_out) continue;
     const size_t o = size_t(m) * g.ldo + n;
     if (g.mode == EPI_STORE_F32) reinterpret_cast<float*>(g.out)[o] = acc;
     else if (g.mode == EPI_ACCUM_F32) reinterpret_cast<float*>(g.out)[o] += acc;
@@ -390,7 +399,7 @@ bool gemm2_preferred(int M, int n_out) {
 void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out) {
   const int tw = (n_out + 255) / 256;
   const int k_tiles = (K + TILE_K - 1) / TILE_K;
-  const bool may_split = mode == EPI_STORE_F32 || mode == EPI_ACCUM_F32 || mode == EPI_STORE_F16 || mode == EPI_STORE_BF16;
+  const bool may_split = mode != EPI_ARGMAX;            // every other epilogue can be applied after the slices are summed
   double best_cost = 1e30;
   int best_bnt = 256, best_s = 1;
   for (int bnt : {256, 128}) {
@@ -434,7 +443,7 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   const int tiles = g.n_tiles_w * g.n_tiles_m;
   const int tail = tiles % 74;
   if (c.splits > 0) splits = c.splits;                    // the caller fixed the number of K-slices (of the tail tiles)
-  if (c.mode == EPI_ARGMAX || c.mode == EPI_SWIGLU_F16 || tail == 0) splits = 1;
+  if (c.mode == EPI_ARGMAX || tail == 0) splits = 1;
   if (splits > g.k_tiles) splits = g.k_tiles;
   if (splits > TAIL_MAX_SPLITS) splits = TAIL_MAX_SPLITS;
   while (splits > 1 && size_t(tail) * splits * g.BNT * 256 * 4 > c.splitk_ws_bytes) --splits;   // never more than the scratch holds
