@@ -45,6 +45,7 @@ struct AttnTcArgs {
   const int32_t* ctx_lens;
   float* ws_o;
   float* ws_ml;
+  __half* o_final;       // [B*k, Hq, dh] fp16: requests whose context is one chunk are finished here, without partials
   uint32_t* status;
   int page_table_stride;
   int B, k, Hq, Hkv, rep, R, n_row_tiles;
@@ -328,7 +329,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     tma_prefetch_desc(&tmV);
     mbar_init(smem_u32(&bars->q_ready), 8);            // one arrival per softmax warp
     mbar_init(smem_u32(&bars->o_free), 8);
-    mbar_init(smem_u32(&bars->l_ready), 4);            // the four warps that own the upper column half
+    mbar_init(smem_u32(&bars->l_ready), 8);
     mbar_init(smem_u32(&bars->o_done), 1);
     for (int s = 0; s < NSK; ++s) {
       mbar_init(smem_u32(&bars->k_full[s]), 1);
@@ -601,19 +602,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         TCLK(5)
       }
       if (!ok) break;
-      // ---- partial (m, l, O) of this chunk: the row sum is the sum of the two halves.
-      // The exchange buffer of parity gt & 1 was last used two tiles ago and is not written again before every
-      // softmax warp has signalled q_ready for the next item, i.e. after this read: 512 bytes = one float per row.
-      float* xl = &bars->xmax[gt & 1][0][0];
-      float l_row = l_sum;
-      if (hf == 1) {
-        xl[r_local] = l_sum;
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&bars->l_ready));
-      } else {
-        if (!mbar_wait(smem_u32(&bars->l_ready), n & 1)) { ok = false; break; }
-        l_row += xl[r_local];
-      }
+      // ---- the row sum is the sum of the two halves: the threads of a row swap theirs.
+      // The exchange buffer of parity gt & 1 was last used two tiles ago, and a thread's slot is not written again
+      // before every softmax warp has signalled q_ready for the next item, i.e. after the partner's read.
+      bars->xmax[gt & 1][hf][r_local] = l_sum;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->l_ready));
+      if (!mbar_wait(smem_u32(&bars->l_ready), n & 1)) { ok = false; break; }
+      const float l_row = l_sum + bars->xmax[gt & 1][hf ^ 1][r_local];
       {
         // every MMA of the item has finished (so has every read of Q): the next item's Q goes in at once and the
         // tensor core starts on its scores during the read-out
@@ -625,23 +621,48 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         if (has_next) store_q(qv);
       }
       const size_t slab = (size_t(b) * a.Hkv + kvh) * a.max_chunks + c;
-      float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH + hf * 64;
+      const bool whole = g.n_chunks == 1;            // the request's only chunk: normalise and finish here
+      if (whole) {
+        // (the last chunk always holds the row's own block key, so the row sum is positive)
+        const float inv = 1.f / l_row;
+        __half* dsth = a.o_final + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH + hf * 64;
 #pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        uint32_t o[32];
-        tmem_ld32(tmem_o + lane_base + hf * 64 + j * 32, o);
-        tmem_wait_ld32(o);
-        if (row_ok) {
+        for (int j = 0; j < 2; ++j) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_base + hf * 64 + j * 32, o);
+          tmem_wait_ld32(o);
+          if (row_ok) {
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<uint4*>(dst + j * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+            for (int e = 0; e < 32; e += 8) {
+              uint32_t h[4];
+#pragma unroll
+              for (int q2 = 0; q2 < 4; ++q2) {
+                const __half2 v = __floats2half2_rn(__uint_as_float(o[e + 2 * q2]) * inv, __uint_as_float(o[e + 2 * q2 + 1]) * inv);
+                h[q2] = *reinterpret_cast<const uint32_t*>(&v);
+              }
+              *reinterpret_cast<uint4*>(dsth + j * 32 + e) = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+          }
+        }
+      } else {
+        float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH + hf * 64;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+          uint32_t o[32];
+          tmem_ld32(tmem_o + lane_base + hf * 64 + j * 32, o);
+          tmem_wait_ld32(o);
+          if (row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; e += 4)
+              *reinterpret_cast<uint4*>(dst + j * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+          }
         }
       }
       // O has been read out: the next item's first P V product may overwrite it
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->o_free));
-      if (row_ok && hf == 0) {
+      if (row_ok && hf == 0 && !whole) {
         float* ml = a.ws_ml + (slab * a.R + rg) * 2;
         ml[0] = (m_ref == NEG) ? -INFINITY : m_ref;
         ml[1] = l_row;
@@ -674,6 +695,7 @@ __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n
   const int b = m / a.k, i = m % a.k;
   const int kvh = hq / a.rep, r = i * a.rep + hq % a.rep;
   const Range g = make_range(a.ctx_lens[b], a.window, a.chunk, 0, a.k);
+  if (g.n_chunks == 1) return;                     // finished by the attention kernel itself
   const size_t slab0 = (size_t(b) * a.Hkv + kvh) * a.max_chunks;
   float m_tot = -INFINITY;
   for (int c = 0; c < g.n_chunks; ++c) m_tot = fmaxf(m_tot, a.ws_ml[((slab0 + c) * a.R + r) * 2]);
@@ -743,6 +765,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   a.scale_log2 = 1.4426950408889634f / sqrtf(float(c.dh));
   const size_t slabs = size_t(c.B) * c.Hkv * max_chunks;
   a.ws_o = reinterpret_cast<float*>(c.ws);
+  a.o_final = reinterpret_cast<__half*>(c.o);
   a.ws_ml = a.ws_o + slabs * a.R * c.dh;
   CUtensorMap tmK, tmV;
   if (!make_pool_tmap(&tmK, c.k_pool, c.num_pages, c.Hkv, err) || !make_pool_tmap(&tmV, c.v_pool, c.num_pages, c.Hkv, err))
