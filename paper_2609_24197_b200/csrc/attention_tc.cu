@@ -18,7 +18,8 @@
 //               reference maximum that only moves when the row maximum outgrows it by 2^8 (then, rarely, rescales
 //               its O row in TMEM), and writes P (bf16, two keys per 32-bit column) over the first half of the S
 //               buffer it came from.  At the end of an item they put the next item's Q tile into shared memory
-//               first (the tensor core starts on its scores), then read O out.
+//               first (the tensor core starts on its scores), then read O out: as a finished fp16 row when the
+//               request has a single chunk, else as an fp32 partial for the merge kernel.
 //
 // The MMA warp issues S_{t+1} before it waits for P_t, so the tensor core works on the next tile's scores while
 // the softmax warps are busy.  Every wait is bounded; a timed-out role sets a status word and the CTA unwinds.
