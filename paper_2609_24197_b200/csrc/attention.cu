@@ -48,6 +48,8 @@ __device__ __forceinline__ uint32_t swz(int row, int col) {   // byte offset of 
 template <int DH>
 __global__ void __launch_bounds__(256)
 attn_partial_kernel(AttnArgs a) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ __align__(128) uint8_t smem[];
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, kvh = blockIdx.y;
@@ -237,6 +239,8 @@ attn_partial_kernel(AttnArgs a) {
 // One block per (row of the block, query head): merge the chunk partials in chunk order.
 template <int DH>
 __global__ void attn_merge_kernel(AttnArgs a) {
+  pdl_wait();
+  pdl_trigger();
   const int m = blockIdx.x;             // b * k + i
   const int hq = blockIdx.y;
   const int b = m / a.k, i = m % a.k;

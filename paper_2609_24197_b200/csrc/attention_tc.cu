@@ -202,6 +202,8 @@ __device__ __forceinline__ Item unpack_item(const int4 w) {
 // bytes of the same pages.  The order inside a bucket depends on atomics; every item is computed independently, so
 // results do not.
 __global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4* __restrict__ items) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ int bucket[64];
   __shared__ int offset[64];
   const int per_chunk = a.Hkv * a.n_row_tiles;
@@ -312,6 +314,8 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
 __global__ void __launch_bounds__(352, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a,
                const int* __restrict__ count, const int4* __restrict__ items) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ __align__(1024) uint8_t smem[];
   uint8_t* sQ = smem;                               // Q tile, 32 KiB
   uint8_t* sKV = smem + KV_BYTES;                   // K ring (NSK x 32 KiB), then V ring (NSV x 32 KiB)
@@ -689,6 +693,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 
 // One block per (row of the block, query head): merge the chunk partials in chunk order (page-aligned chunk geometry).
 __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n_pairs) {
+  pdl_wait();
+  pdl_trigger();
   // one warp per (row, head): each lane merges four adjacent head-dim columns with 16-byte loads
   const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (pair >= n_pairs) return;
@@ -782,7 +788,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   int* count = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(a.ws_ml + slabs * a.R * 2) + 15) & ~uintptr_t(15));
   int4* items = reinterpret_cast<int4*>(count + 4);
   trk_begin(trk, "attn_plan");
-  attn_tc_plan_kernel<<<1, 256, 0, stream>>>(a, count, items);
+  launch_pdl(attn_tc_plan_kernel, dim3(1), dim3(256), 0, stream, a, count, items);
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -793,13 +799,13 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
       n_sms = 148;
   }
   trk_begin(trk, "attn_partial");
-  attn_tc_kernel<<<n_sms, 352, smem, stream>>>(tmK, tmV, a, count, items);
+  launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(352), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
   trk_end(trk);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   const int n_pairs = c.B * c.k * c.Hq;
   trk_begin(trk, "attn_merge");
-  attn_tc_merge_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(a, reinterpret_cast<__half*>(c.o), n_pairs);
+  launch_pdl(attn_tc_merge_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, a, reinterpret_cast<__half*>(c.o), n_pairs);
   trk_end(trk);
   return cudaGetLastError();
 }

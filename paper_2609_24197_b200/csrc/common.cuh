@@ -33,6 +33,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // (fast exponential and fast division: ~2 ulp each, far inside every tolerance that follows an fp16 or bf16 rounding)
 __device__ __forceinline__ float silu_f(float v) { return __fdividef(v, 1.0f + __expf(-v)); }
 
+// ------------------------------------------------------------------ programmatic dependent launch
+// A kernel launched with launch_pdl() may start while the kernel before it on the stream is still running: its CTAs
+// run their set-up and then block in pdl_wait() until that kernel has finished and its writes are visible.  Nothing
+// produced by an earlier kernel may be read, and nothing may be written to global memory, before pdl_wait().
+// pdl_trigger() lets the NEXT kernel on the stream start launching once every CTA of this one has called it.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------------ mbarrier
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));

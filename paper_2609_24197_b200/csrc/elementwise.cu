@@ -11,6 +11,8 @@ namespace {
 // embedding; no positional embedding is added (paper Sec. 3.3.1).
 __global__ void embed_rows_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ last_token,
                                   int mask_id, float* __restrict__ X, int k, int D) {
+  pdl_wait();
+  pdl_trigger();
   const int m = blockIdx.x;
   const int b = m / k, i = m % k;
   const int tok = (i == 0) ? last_token[b] : mask_id;
@@ -38,6 +40,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 out.
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __half* __restrict__ y,
                                int n, float eps) {
+  pdl_wait();
+  pdl_trigger();
   __shared__ float red[32];
   const float* xr = x + size_t(blockIdx.x) * n;
   __half* yr = y + size_t(blockIdx.x) * n;
@@ -84,6 +88,8 @@ __global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* 
                                     const int32_t* __restrict__ ctx_lens, __nv_bfloat16* __restrict__ q,
                                     __nv_bfloat16* __restrict__ kb, __nv_bfloat16* __restrict__ vb, int k, int Hq,
                                     int Hkv, int dh, float eps, int qk_norm, int n_pairs) {
+  pdl_wait();
+  pdl_trigger();
   const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (pair >= n_pairs) return;
   const int heads = Hq + 2 * Hkv;
@@ -126,6 +132,8 @@ __global__ void kv_inject_write_kernel(const float* __restrict__ kv, const float
                                        int page_table_stride, __nv_bfloat16* __restrict__ k_pool,
                                        __nv_bfloat16* __restrict__ v_pool, int Hkv, int dh, int page_size, float eps,
                                        int k_norm, int n_pairs) {
+  pdl_wait();
+  pdl_trigger();
   const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (pair >= n_pairs) return;
   const int t = pair / (2 * Hkv), hh = pair % (2 * Hkv);
@@ -160,6 +168,8 @@ __global__ void kv_inject_write_kernel(const float* __restrict__ kv, const float
 }
 
 __global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F) {
+  pdl_wait();
+  pdl_trigger();
   const long long total = (long long)M * F;
   for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
        idx += (long long)gridDim.x * blockDim.x) {
@@ -170,6 +180,8 @@ __global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__
 }
 
 __global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, size_t n) {
+  pdl_wait();
+  pdl_trigger();
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x)
     dst[i] = src[i];
 }
@@ -203,14 +215,14 @@ int grid_for(long long total, int threads) {
 
 cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
                               int D, cudaStream_t stream) {
-  embed_rows_kernel<<<B * k, 256, 0, stream>>>((const __nv_bfloat16*)embed_bf16, last_token, mask_id, X, k, D);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(embed_rows_kernel, dim3(B * k), dim3(256), 0, stream, (const __nv_bfloat16*)embed_bf16, last_token, mask_id, X, k, D);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream) {
   const int threads = n >= 2048 ? 512 : 256;
-  rmsnorm_kernel<<<M, threads, 0, stream>>>(x, w, (__half*)y_f16, n, eps);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, (__half*)y_f16, n, eps);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
@@ -220,10 +232,9 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
   const float* tab = rope_table(theta, dh, stream);
   if (!tab) return cudaErrorMemoryAllocation;
   const int n_pairs = B * k * (Hq + 2 * Hkv);
-  qk_norm_rope_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(qkv, qw, kw, tab, ctx_lens, (__nv_bfloat16*)q,
-                                                             (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps,
-                                                             qk_norm, n_pairs);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(qk_norm_rope_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, qkv, qw, kw, tab, ctx_lens,
+                             (__nv_bfloat16*)q, (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps, qk_norm, n_pairs);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32_t* req, const int32_t* pos,
@@ -240,13 +251,13 @@ cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32
 }
 
 cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream) {
-  swiglu_kernel<<<grid_for((long long)M * F, 256), 256, 0, stream>>>(gu, (__half*)h_f16, M, F);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(swiglu_kernel, dim3(grid_for((long long)M * F, 256)), dim3(256), 0, stream, gu, (__half*)h_f16, M, F);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream) {
-  copy_f32_kernel<<<grid_for((long long)n, 256), 256, 0, stream>>>(src, dst, n);
-  return cudaGetLastError();
+  cudaError_t e = launch_pdl(copy_f32_kernel, dim3(grid_for((long long)n, 256)), dim3(256), 0, stream, src, dst, n);
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
 }  // namespace hspec

@@ -74,6 +74,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_acc = tail->tmem_base;
+  pdl_wait();                                   // set-up done: now the previous kernel's results may be read
+  pdl_trigger();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -242,6 +244,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 // Sum the K-slice partials in slice order (deterministic) and apply the final store.
 __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, int M, int N, void* out,
                                      long long ldo, int mode) {
+  pdl_wait();
+  pdl_trigger();
   const long long total = (long long)M * N;
   for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
        i += (long long)gridDim.x * blockDim.x) {
@@ -269,6 +273,8 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
 template <int SPLITS>
 __global__ void splitk_reduce_f32x4_kernel(const float* __restrict__ part, int M, int N, float* __restrict__ out,
                                            long long ldo, int accumulate) {
+  pdl_wait();
+  pdl_trigger();
   const int m = blockIdx.y;
   const size_t slice = size_t(M) * N;
   for (int n4 = blockIdx.x * blockDim.x + threadIdx.x; n4 < (N >> 2); n4 += gridDim.x * blockDim.x) {
@@ -288,6 +294,8 @@ __global__ void splitk_reduce_f32x4_kernel(const float* __restrict__ part, int M
 // ids[m] = lowest index among the per-tile maxima (tiles are in ascending vocabulary order).
 __global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
                                      int* __restrict__ ids, const int* __restrict__ id_map) {
+  pdl_wait();
+  pdl_trigger();
   const int m = blockIdx.x;
   float v = -INFINITY;
   int idx = 0x7fffffff;
@@ -442,9 +450,9 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   dim3 grid((c.M + g.BN - 1) / g.BN, (c.n_out + TILE_W - 1) / TILE_W, splits);
   const size_t smem = size_t(stages) * stage_bytes + fixed;
   trk_begin(trk, c.label ? c.label : "gemm", 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
-  gemm_tcgen05_kernel<<<grid, 192, smem, stream>>>(*c.tmW, tmB, g);
+  cudaError_t e = launch_pdl(gemm_tcgen05_kernel, grid, dim3(192), smem, stream, *c.tmW, tmB, g);
   trk_end(trk);
-  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (splits > 1)
     e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk);
@@ -461,13 +469,13 @@ cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, vo
     dim3 grid((N / 4 + 255) / 256, M);
     float* o = reinterpret_cast<float*>(out);
     const int acc = mode == EPI_ACCUM_F32;
-    if (splits == 2) splitk_reduce_f32x4_kernel<2><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
-    else if (splits == 3) splitk_reduce_f32x4_kernel<3><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
-    else splitk_reduce_f32x4_kernel<4><<<grid, 256, 0, stream>>>(part, M, N, o, ldo, acc);
+    if (splits == 2) launch_pdl(splitk_reduce_f32x4_kernel<2>, grid, dim3(256), 0, stream, part, M, N, o, ldo, acc);
+    else if (splits == 3) launch_pdl(splitk_reduce_f32x4_kernel<3>, grid, dim3(256), 0, stream, part, M, N, o, ldo, acc);
+    else launch_pdl(splitk_reduce_f32x4_kernel<4>, grid, dim3(256), 0, stream, part, M, N, o, ldo, acc);
   } else {
     int blocks = int((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(part, splits, M, N, out, ldo, mode);
+    launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, part, splits, M, N, out, ldo, mode);
   }
   trk_end(trk);
   return cudaGetLastError();
@@ -476,7 +484,7 @@ cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, vo
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk, const int* id_map) {
   trk_begin(trk, "argmax_reduce", 0, double(n_tiles) * M * 8);
-  argmax_reduce_kernel<<<M, 256, 0, stream>>>(pv, pi, n_tiles, M, ids, id_map);
+  launch_pdl(argmax_reduce_kernel, dim3(M), dim3(256), 0, stream, pv, pi, n_tiles, M, ids, id_map);
   trk_end(trk);
   return cudaGetLastError();
 }

@@ -157,6 +157,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = tail->tmem_base;
   volatile uint32_t* abort_flag = &tail->abort_flag;
+  pdl_wait();                                   // set-up done: now the previous kernel's results may be read
+  pdl_trigger();
 
   if (warp == 0) {
     if (lane == 0) {
@@ -342,6 +344,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 constexpr int TAIL_MAX_SPLITS = 8, TAIL_ROWS = 4;
 __global__ void __launch_bounds__(256)
 gemm2_tail_reduce_kernel(Gemm2Args g) {
+  pdl_wait();
+  pdl_trigger();
   const int tail = blockIdx.x, tile = g.n_full_tiles + tail;
   const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
   const int n = tn * 256 + threadIdx.x;
@@ -471,12 +475,12 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   std::string label = "gemm2:";
   if (c.label) { const char* colon = strchr(c.label, ':'); label += colon ? colon + 1 : c.label; }
   trk_begin(trk, label.c_str(), 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
-  gemm_2sm_kernel<<<2 * clusters, 192, smem, stream>>>(*c.tmW, tmB, g);
+  cudaError_t e = launch_pdl(gemm_2sm_kernel, dim3(2 * clusters), dim3(192), smem, stream, *c.tmW, tmB, g);
   trk_end(trk);
-  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e == cudaSuccess && splits > 1) {
     trk_begin(trk, "gemm2_tail_reduce", 0, double(splits + 1) * tail * g.BNT * 256 * 4);
-    gemm2_tail_reduce_kernel<<<dim3(tail, g.BNT / TAIL_ROWS), 256, 0, stream>>>(g);
+    launch_pdl(gemm2_tail_reduce_kernel, dim3(tail, g.BNT / TAIL_ROWS), dim3(256), 0, stream, g);
     trk_end(trk);
     e = cudaGetLastError();
   }

@@ -267,6 +267,8 @@ std::vector<std::string> required_names(const hspec_config& c) {
 }
 
 __global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n) {
+  pdl_wait();
+  pdl_trigger();
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x)
     dst[i] = __float2half_rn(__bfloat162float(src[i]));
 }
@@ -296,6 +298,8 @@ __global__ void wait_selftest_kernel(uint32_t* status, unsigned long long limit_
 
 __global__ void cvt_cols_f16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
                                     __half* __restrict__ dst) {
+  pdl_wait();
+  pdl_trigger();
   const int total = M * ncols;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x)
     dst[i] = __float2half_rn(src[size_t(i / ncols) * ld + col0 + i % ncols]);

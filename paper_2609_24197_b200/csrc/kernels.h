@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cstdlib>
 #include <string>
 #include <vector>
 
@@ -34,6 +35,19 @@ struct Tracker {
 };
 inline void trk_begin(Tracker* t, const char* name, double flops = 0, double bytes = 0) { if (t) t->begin(name, flops, bytes); }
 inline void trk_end(Tracker* t) { if (t) t->end(); }
+
+// Launch with programmatic stream serialisation: the kernel MUST call pdl_wait() before it touches global data.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+  static const bool off = [] { const char* e = getenv("HSPEC_NO_PDL"); return e && e[0] == '1'; }();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = off ? 0 : 1;
+  cfg.attrs = at; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 enum GemmEpilogue : int {
   EPI_STORE_F32 = 0,    // y fp32 = acc

@@ -85,6 +85,8 @@ __global__ void token_probs_kernel(const float* __restrict__ logits, long long l
 // position's rank-r product with W_out.
 __global__ void markov_gather_kernel(const uint16_t* __restrict__ W_in, const int* __restrict__ prev, long long prev_stride,
                                      uint16_t* __restrict__ x, int r) {
+  pdl_wait();
+  pdl_trigger();
   const int b = blockIdx.x;
   const uint16_t* src = W_in + size_t(prev[size_t(b) * prev_stride]) * r;
   for (int i = threadIdx.x; i < (r >> 3); i += blockDim.x)
@@ -96,6 +98,8 @@ __global__ void markov_gather_kernel(const uint16_t* __restrict__ W_in, const in
 __global__ void markov_reduce_gather_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int B,
                                             int* __restrict__ ids, int k, int i, const int* __restrict__ id_map,
                                             const uint16_t* __restrict__ W_in, uint16_t* __restrict__ x, int r, int gather) {
+  pdl_wait();
+  pdl_trigger();
   const int b = blockIdx.x;
   float v = -INFINITY;
   int idx = 0x7fffffff;
@@ -178,8 +182,8 @@ cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk
     e = gemm_launch(g, stream, trk, err);
     if (e != cudaSuccess) return e;
     trk_begin(trk, "markov_reduce");
-    markov_reduce_gather_kernel<<<c.B, 128, 0, stream>>>(part_val, part_idx, int(vt), c.B, c.ids, c.k, i, c.id_map,
-                                                         reinterpret_cast<const uint16_t*>(c.W_in), x, c.r, i + 1 < c.k);
+    launch_pdl(markov_reduce_gather_kernel, dim3(c.B), dim3(128), 0, stream, (const float*)part_val, (const int*)part_idx,
+               int(vt), c.B, c.ids, c.k, i, c.id_map, reinterpret_cast<const uint16_t*>(c.W_in), x, c.r, int(i + 1 < c.k));
     trk_end(trk);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

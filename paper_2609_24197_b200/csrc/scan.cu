@@ -31,6 +31,8 @@ __device__ __forceinline__ float softplus_f(float v) { return v > 20.f ? v : log
 
 __global__ void __launch_bounds__(SCAN_THREADS)
 mamba_scan_kernel(ScanArgs a) {
+  pdl_wait();
+  pdl_trigger();
   extern __shared__ __align__(16) float sm[];
   const int tid = threadIdx.x;
   const int h = blockIdx.x, b = blockIdx.y;
@@ -157,6 +159,8 @@ mamba_scan_kernel(ScanArgs a) {
 template <int P, int N, int MT>
 __global__ void __launch_bounds__(128)
 mamba_scan_mma_kernel(ScanArgs a) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int HPC = 4;                 // heads (= warps) per CTA
   constexpr int NT = P / 8;              // n-tiles of the MMA (head channels)
   constexpr int KP = N / 32;             // k-step pairs
@@ -328,6 +332,8 @@ mamba_scan_mma_kernel(ScanArgs a) {
 //   mamba_scan_stream_kernel  one warp per head: everything it needs is fetched up front (cp.async for the
 //                      shared operands, 16-byte loads of S_init straight into the MMA fragments)
 __global__ void scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* __restrict__ c16) {
+  pdl_wait();
+  pdl_trigger();
   const int ch = blockIdx.x * blockDim.x + threadIdx.x;
   const int b = blockIdx.y;
   if (ch >= a.d_xBC) return;
@@ -361,6 +367,8 @@ __global__ void scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* _
 }
 
 __global__ void scan_cb_kernel(ScanArgs a, const float* __restrict__ xact, float* __restrict__ cb) {
+  pdl_wait();
+  pdl_trigger();
   const int g = blockIdx.x, b = blockIdx.y;
   const int k = a.k, N = a.N;
   const size_t row0 = size_t(b) * k;
@@ -381,6 +389,8 @@ template <int P, int N, int MT>
 __global__ void __launch_bounds__(128)
 mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __half* __restrict__ c16,
                          const float* __restrict__ cb) {
+  pdl_wait();
+  pdl_trigger();
   constexpr int HPC = 4, NT = P / 8, KP = N / 32, ROWS = MT * 16;
   extern __shared__ __align__(16) float sm[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -552,10 +562,10 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
     float* cbw = xact + M * a.d_xBC;
     __half* c16 = reinterpret_cast<__half*>(cbw + size_t(c.B) * c.G * KMAX * KMAX);
     trk_begin(trk, "scan_conv", 0, double(M) * a.d_xBC * 8);
-    scan_conv_kernel<<<dim3((a.d_xBC + 255) / 256, c.B), 256, 0, stream>>>(a, xact, c16);
+    launch_pdl(scan_conv_kernel, dim3((a.d_xBC + 255) / 256, c.B), dim3(256), 0, stream, a, xact, c16);
     trk_end(trk);
     trk_begin(trk, "scan_cb", 0, 0);
-    scan_cb_kernel<<<dim3(c.G, c.B), 256, 0, stream>>>(a, xact, cbw);
+    launch_pdl(scan_cb_kernel, dim3(c.G, c.B), dim3(256), 0, stream, a, xact, (float*)cbw);
     trk_end(trk);
     const size_t smem_s = two ? scan_stream_smem<2>() : scan_stream_smem<1>();
     static bool sset1 = false, sset2 = false;
@@ -568,8 +578,8 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
     }
     dim3 grid_s(a.H / 4, c.B);
     trk_begin(trk, "mamba_scan", 2.0 * c.B * c.k * a.H * c.P * c.N, double(c.B) * a.H * c.P * c.N * 2);
-    if (two) mamba_scan_stream_kernel<64, 128, 2><<<grid_s, 128, smem_s, stream>>>(a, xact, c16, cbw);
-    else mamba_scan_stream_kernel<64, 128, 1><<<grid_s, 128, smem_s, stream>>>(a, xact, c16, cbw);
+    if (two) launch_pdl(mamba_scan_stream_kernel<64, 128, 2>, grid_s, dim3(128), smem_s, stream, a, (const float*)xact, (const __half*)c16, (const float*)cbw);
+    else launch_pdl(mamba_scan_stream_kernel<64, 128, 1>, grid_s, dim3(128), smem_s, stream, a, (const float*)xact, (const __half*)c16, (const float*)cbw);
     trk_end(trk);
     return cudaGetLastError();
   }
