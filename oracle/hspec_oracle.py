@@ -24,12 +24,21 @@ What pins each function (tests/test_oracle_*.py):
                         invariance, window, NaN-poisoned slots
   argmax_margin         full sort, constructed ties
   kv_bytes_per_token    Table 1 of the paper (tests/golden/table1_kv_bytes.txt)
-  draft_block           request independence, page-permutation invariance,
+  mlp_block, attention_block, mamba_mixer
+                        scalar index loops over nested lists that spell out the
+                        documented layouts (gate | up; q | k | v, norm before the
+                        rotation, row i at position ctx_len + i; z | xBC | dt,
+                        x | B | C, gate then norm over all Di), each with planted
+                        mistakes that must disagree
+  draft_block           the same scalar loops composed into the whole step;
+                        request independence, page-permutation invariance,
                         causal k-prefix property, ablation special cases.
-                        The COMPOSITION itself (which sub-blocks, pre-norm
-                        placement, Mamba-2 mixer internals) is a reading of a
-                        paper that prints no worked forward pass:
-                        **parity unpinned** for the composition.
+                        The scalar loops pin the code to the layouts and the
+                        order stated here.  That order itself (which sub-blocks,
+                        pre-norm placement, Mamba-2 mixer internals) is a reading
+                        of a paper that prints no worked forward pass:
+                        **parity unpinned** with respect to the paper for the
+                        composition.
 """
 import numpy as np
 
