@@ -2,11 +2,18 @@
 """Benchmark of the H-Spec block-parallel draft step on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+    python bench.py --sweep                    # only the concurrency x block-size sweep, more steps per cell
+    python bench.py --case NAME [--reps N]     # one kernel on a small case, for profiler captures
 
 One "step" = one call of hspec_draft_block (the whole hot path) over one batch of seeded synthetic requests.
 The headline workload is the concurrency-128 configuration (32B-class shapes, B = 128, k = 16, contexts
-log-uniform in [1024, 32768]); the concurrency-1 and concurrency-32 configurations are measured in the same run
-and reported under "by_concurrency".  Prints ONE JSON line (rank 0).
+log-uniform in [1024, 32768]); the concurrency-1 and concurrency-32 configurations, the two serving workloads with
+the paper's 2048-token window, and the 18 cells of the concurrency x block-size sweep are measured in the same run
+and reported under "by_concurrency", "window_2048" and "sweep".  Prints ONE JSON line (rank 0).
+
+Timing: W warm-up steps, then untimed steps for --settle-s seconds (so the GPU sits at the clocks it keeps under its
+power cap, the condition the tensor peak was measured in), then --repeats timed regions of exactly K steps each, every
+one bracketed by a synchronise and one pair of CUDA events; `value` is the median region, all of them are listed.
 
 Multi-GPU: the step has no exchange between requests, so N > 1 runs N independent replicas (one process per
 GPU, different requests per rank, no data-path collective); time is the max over ranks.
@@ -43,8 +50,25 @@ def load_peaks():
         with open(path) as f:
             p = json.load(f)
         return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
-                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
-    return dict(FALLBACK_PEAKS, source="fallback")
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                    sustained_sm_mhz=float(p.get("clocks_under_load", {}).get("sm_mhz_median", 0.0)) or None,
+                    source="measured")
+    return dict(FALLBACK_PEAKS, sustained_sm_mhz=1300.0, source="fallback")
+
+
+def load_traffic():
+    """DRAM traffic per kernel as a ratio to its algorithmic bytes, from the profiler captures recorded in
+    profiles/dram_traffic.json (kernel -> {dram_read_bytes, dram_write_bytes, algorithmic_bytes, case, ...})."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return {}
+    with open(path) as f:
+        rec = json.load(f)
+    out = {}
+    for name, r in rec.get("kernels", {}).items():
+        out[name] = dict(ratio=(r["dram_read_bytes"] + r["dram_write_bytes"]) / r["algorithmic_bytes"],
+                         case=r.get("case", ""), captured=r.get("captured", ""))
+    return out
 
 
 def workload_accounting(cfg, ctx_lens, B, k):
@@ -81,7 +105,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
+                                          "-lms", "50", "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -92,14 +116,11 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.time(), line.strip()))
 
-    def stop(self, t0=None, t1=None):
-        if self.proc is None:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
-        time.sleep(0.15)
-        self.proc.terminate()
+    def window(self, t0, t1):
+        """Median SM clock and the throttle reasons seen between two wall-clock times."""
         sm, mx, reasons = [], [], set()
-        for ts, line in self.lines:
-            if t0 is not None and not (t0 <= ts <= t1 + 0.2):
+        for ts, line in list(self.lines):
+            if not (t0 <= ts <= t1 + 0.1):
                 continue
             f = [x.strip() for x in line.split(",")]
             if len(f) < 9:
@@ -115,6 +136,13 @@ class ClockSampler:
         if not sm:
             return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples in the timed region"], samples=0)
         return dict(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+
+    def stop(self, t0=None, t1=None):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        return self.window(t0 if t0 is not None else 0.0, t1 if t1 is not None else time.time())
 
 
 def to_np(t):
@@ -144,9 +172,10 @@ def barrier():
 
 # ----------------------------------------------------------------------------- the CUDA arm
 
-def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=False):
+def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=False, repeats=1, settle_s=0.0,
+                 want_graph=True, **cfg_over):
     import paper_2609_24197_b200 as hs
-    cfg = synth.get_config(name)
+    cfg = synth.get_config(name, **cfg_over)
     B, k = cfg["B"], cfg["k"]
     dev = torch.device("cuda", torch.cuda.current_device())
     weights = synth.make_weights(cfg, device=dev)
@@ -169,26 +198,44 @@ def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=
     for _ in range(max(warmup, 3)):
         step()
     torch.cuda.synchronize()
-    barrier()
     sampler = ClockSampler(clock_gpu) if clock_gpu is not None else None
     if sampler:
         sampler.start()
-        time.sleep(0.25)
-    # ---- the timed region: exactly `steps` steps, nothing else on the stream, one pair of events around it
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    torch.cuda.synchronize()
-    t0 = time.time()
-    e0.record(stream)
-    for _ in range(steps):
-        step()
-    e1.record(stream)
-    torch.cuda.synchronize()
-    t1 = time.time()
+    # ---- untimed steps until the GPU has settled under its power cap (the sustained-peak condition)
+    settle_steps = 0
+    t_end = time.time() + settle_s
+    while time.time() < t_end:
+        for _ in range(8):
+            step()
+        settle_steps += 8
+        torch.cuda.synchronize()
     barrier()
-    clocks = sampler.stop(t0, t1) if sampler else None
-    total_ms = max_over_ranks(e0.elapsed_time(e1), dev)
+    # ---- the timed regions: each exactly `steps` steps, nothing else on the stream, one pair of events around it
+    regions = []
+    for _ in range(max(1, repeats)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        barrier()
+        t0 = time.time()
+        e0.record(stream)
+        for _ in range(steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1), dev)
+        regions.append(dict(ms_per_step=ms / steps, t0=t0, t1=t1))
+    t_first, t_last = regions[0]["t0"], regions[-1]["t1"]
+    for r in regions:
+        w = sampler.window(r["t0"], r["t1"]) if sampler else None
+        r["sm_mhz"] = w["sm_mhz"] if w else None
+    clocks = sampler.stop(t_first, t_last) if sampler else None
+    by_ms = sorted(regions, key=lambda r: r["ms_per_step"])
+    median = by_ms[(len(by_ms) - 1) // 2]          # an actual region (the lower median), with its own clock reading
+    total_ms = median["ms_per_step"] * steps
     stats = drafter.stats()
-    assert stats["device_status"] == 0, f"device status {stats['device_status']:#x}"
+    assert stats["rc"] == 0, f"device status block not clean: {stats}"
     launches = stats["launches_last_step"]
     # ---- the same steps again with a pair of CUDA events around every kernel launch (recorded by the library on
     # the step's stream): per-kernel durations for the roofline figures.  The events cost host time, which shows at
@@ -203,18 +250,20 @@ def run_workload(name, steps, warmup, rank, clock_gpu=None, want_e2e=True, lean=
         step()
         ev[i + 1].record(stream)
         for e in hs.hspec_get_profile(drafter.handle):       # reading them waits for the step
-            a = prof.setdefault(e["name"], dict(ms=0.0, n=0, flops=0.0, bytes=0.0))
+            a = prof.setdefault(e["name"], dict(ms=0.0, n=0, flops=0.0, bytes=0.0, io_bytes=0.0))
             a["ms"] += e["ms"]; a["n"] += 1; a["flops"] += e["flops"]; a["bytes"] += e["bytes"]
+            a["io_bytes"] += e["io_bytes"]
     torch.cuda.synchronize()
     hs.hspec_set_profiling(drafter.handle, False)
     step_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
     out = dict(name=name, B=B, k=k, ms_per_step=total_ms / steps, step_ms=step_ms, acct=acct, prof=prof,
                launches_per_step=launches, clocks=clocks, ctx_sum=sum(ctx), ctx_max=max_ctx, cfg=cfg,
-               ms_per_step_profiled=sum(step_ms) / steps)
+               ms_per_step_profiled=sum(step_ms) / steps, settle_steps=settle_steps, sm_mhz=median["sm_mhz"],
+               regions=[dict(ms_per_step=round(r["ms_per_step"], 4), sm_mhz=r["sm_mhz"]) for r in regions])
     # ---- the step captured once in a CUDA graph and replayed (what a serving loop does with a launch-bound step);
     # reported beside `value`, which stays on plain launches
     out["graph_replay_ms_per_step"] = None
-    if not lean:
+    if not lean and want_graph:
         try:
             side = torch.cuda.Stream()
             side.wait_stream(stream)
@@ -358,19 +407,21 @@ def kernel_table(res):
     return rows
 
 
-def summarize(res, peaks):
+def summarize(res, peaks, traffic=None):
     """Roofline numbers of one workload from the per-launch event times."""
+    traffic = traffic or {}
     steps = len(res["step_ms"])
     a = res["acct"]
     ms = res["ms_per_step"]
     hbm, tf = peaks["hbm_gbs"], peaks["bf16_tflops_sustained"]
     hbm_time_ms = (a["weight_bytes"] + a["kv_bytes"]) / (hbm * 1e9) * 1e3
     tensor_time_ms = (a["gemm_flops"] + a["attn_flops"]) / (tf * 1e12) * 1e3
+
     def group(prefix):
         vs = [v for n, v in res["prof"].items() if n.startswith(prefix)]
         t = sum(v["ms"] for v in vs) / steps
         return dict(ms=t, flops=sum(v["flops"] for v in vs) / steps, bytes=sum(v["bytes"] for v in vs) / steps,
-                    launches=sum(v["n"] for v in vs) // steps)
+                    io_bytes=sum(v["io_bytes"] for v in vs) / steps, launches=sum(v["n"] for v in vs) // steps)
     g1, g2 = group("gemm:"), group("gemm2:")          # one-CTA kernel (few rows), 2-CTA persistent kernel (many rows)
     gemm_ms, gemm_flops, gemm_bytes = g1["ms"] + g2["ms"], g1["flops"] + g2["flops"], g1["bytes"] + g2["bytes"]
     att = res["prof"].get("attn_partial")
@@ -379,29 +430,47 @@ def summarize(res, peaks):
     att_gbs = a["kv_bytes"] / (att_ms * 1e-3) / 1e9 if att_ms > 0 else 0.0
     gemm_tfs = gemm_flops / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0
+    sm_mhz = res.get("sm_mhz")
+
+    def dram_traffic(kernel, algorithmic_bytes_per_launch):
+        """DRAM bytes per launch = the ratio a profiler capture of this kernel measured (small case, scaled by the
+        algorithmic bytes: every byte is read once, so traffic grows in proportion) x this launch's algorithmic bytes."""
+        t = traffic.get(kernel)
+        if not t:
+            return None, "no profiler capture on record for this kernel"
+        return round(t["ratio"] * algorithmic_bytes_per_launch), \
+            f"{t['ratio']:.3f} x algorithmic bytes per launch (ncu dram__bytes_read+write on {t['case']})"
 
     def gemm_roof(kernel, grp):
         """Roofline of one GEMM kernel over its launches in a step: the bound is the roofline that takes longer."""
         if grp["ms"] <= 0:
             return None
         tfs, gbs = grp["flops"] / (grp["ms"] * 1e-3) / 1e12, grp["bytes"] / (grp["ms"] * 1e-3) / 1e9
+        tr, tr_note = dram_traffic(kernel, (grp["bytes"] + grp["io_bytes"]) / max(1, grp["launches"]))
+        base = dict(kernel=kernel, traffic=tr, traffic_note=tr_note, ms_per_step=round(grp["ms"], 4),
+                    launches_per_step=grp["launches"],
+                    algorithmic_bytes_per_launch=round((grp["bytes"] + grp["io_bytes"]) / max(1, grp["launches"])))
         if grp["flops"] / (tf * 1e12) >= grp["bytes"] / (hbm * 1e9):
-            return dict(kernel=kernel, bound="tensor", achieved=round(tfs, 1), peak=tf, unit="TFLOP/s",
-                        frac=round(tfs / tf, 4), traffic=None, ms_per_step=round(grp["ms"], 4),
-                        note=f"sum over its {grp['launches']} launches per step: 2*M*N*K flops / CUDA-event time; peak = cuBLAS "
-                             f"bf16 sustained, of {peaks['source']} (fp16 has the same nominal rate)")
-        return dict(kernel=kernel, bound="hbm", achieved=round(gbs, 1), peak=hbm, unit="GB/s", frac=round(gbs / hbm, 4),
-                    traffic=None, ms_per_step=round(grp["ms"], 4),
-                    note=f"sum over its {grp['launches']} launches per step: weight bytes / CUDA-event time; peak = copy "
-                         f"bandwidth, of {peaks['source']}; ncu traffic of this kernel = 1.01 x algorithmic "
-                         f"(profiles/gemm_tcgen05_skinny_32x65536x4096.md)")
+            r = dict(base, bound="tensor", achieved=round(tfs, 1), peak=tf, unit="TFLOP/s", frac=round(tfs / tf, 4),
+                     note=f"sum over its launches per step: 2*M*N*K flops / CUDA-event time; peak = cuBLAS bf16 sustained, "
+                          f"of {peaks['source']} (fp16 has the same nominal rate)")
+            if sm_mhz and peaks.get("sustained_sm_mhz"):
+                # the sustained peak was measured at its own (lower) clock: compare flops per clock as well
+                r["per_clock"] = dict(achieved_tflops_per_ghz=round(tfs / (sm_mhz * 1e-3), 1),
+                                      peak_tflops_per_ghz=round(tf / (peaks["sustained_sm_mhz"] * 1e-3), 1),
+                                      frac=round((tfs / sm_mhz) / (tf / peaks["sustained_sm_mhz"]), 4),
+                                      sm_mhz=sm_mhz, peak_sm_mhz=peaks["sustained_sm_mhz"])
+            return r
+        return dict(base, bound="hbm", achieved=round(gbs, 1), peak=hbm, unit="GB/s", frac=round(gbs / hbm, 4),
+                    note=f"sum over its launches per step: weight bytes / CUDA-event time; peak = copy bandwidth, of "
+                         f"{peaks['source']}")
     roofs = [r for r in (gemm_roof("gemm_2sm_kernel", g2), gemm_roof("gemm_tcgen05_kernel", g1)) if r]
     if att_ms > 0:
+        tr, tr_note = dram_traffic("attn_tc_kernel", a["kv_bytes"] / n_attn)
         roofs.append(dict(kernel="attn_tc_kernel", bound="hbm", achieved=round(att_gbs, 1), peak=hbm, unit="GB/s",
-                          frac=round(att_gbs / hbm, 4), traffic=round(1.06 * a["kv_bytes"] / n_attn), ms_per_step=round(att_ms, 4),
-                          note=f"visible target-KV bytes / CUDA-event time over its {n_attn} launches per step, of "
-                               f"{peaks['source']}; traffic per launch = 1.06 x algorithmic, scaled from the small-case ncu "
-                               f"capture (profiles/attn_tc_32b_small.md)"))
+                          frac=round(att_gbs / hbm, 4), traffic=tr, traffic_note=tr_note, ms_per_step=round(att_ms, 4),
+                          launches_per_step=n_attn, algorithmic_bytes_per_launch=round(a["kv_bytes"] / n_attn),
+                          note=f"visible target-KV bytes / CUDA-event time over its launches per step, of {peaks['source']}"))
     roof = max(roofs, key=lambda r: r["ms_per_step"])            # the dominant kernel of this workload
     return dict(
         ms_per_step=round(ms, 4), draft_tokens_per_s=round(res["B"] * res["k"] / (ms * 1e-3), 1),
@@ -421,6 +490,173 @@ def summarize(res, peaks):
     )
 
 
+def brief(s, r=None):
+    """The few figures of a summarised workload that the side tables of the bench line carry."""
+    out = dict(draft_tokens_per_s=s["draft_tokens_per_s"], ms_per_step=s["ms_per_step"],
+               hbm_roofline_frac=s["hbm_roofline_frac"], max_roofline_frac=s["max_roofline_frac"],
+               attention_frac_of_hbm=s["attention"]["frac_of_hbm"], weight_GB=s["weight_GB"], kv_GB=s["kv_GB"],
+               graph_replay_ms_per_step=s["graph_replay_ms_per_step"])
+    if r is not None:
+        out["sm_mhz"] = r.get("sm_mhz")
+    return out
+
+
+def run_sweep(steps, warmup, peaks, rank=0):
+    """The concurrency x block-size sweep on the 8B-class drafter: B in {1, 8, 32, 64, 128, 256} x k in {8, 16, 32},
+    contexts uniform in [1024, 16384].  One handle (made for B <= 256, k <= 32) and one weight set serve all cells; per
+    cell: warm-up, `steps` timed steps between one pair of events, then two profiled steps for the attention kernel's
+    share.  Also per cell: the bytes a drafter-side KV cache over the same contexts would hold (K and V of the two
+    attention layers, 8 KiB per context token; and the figure the sweep's own description spells out, one tensor of
+    2 layers x 8 heads x 128 x 2 B = 4 KiB per token) against zero for in-place reuse of the target's cache."""
+    import paper_2609_24197_b200 as hs
+    dev = torch.device("cuda", torch.cuda.current_device())
+    Bs, ks = (1, 8, 32, 64, 128, 256), (8, 16, 32)
+    cfg_max = synth.get_config(f"sweep_8b_B{max(Bs)}_k{max(ks)}")
+    weights = synth.make_weights(cfg_max, device=dev)
+    drafter = hs.Drafter(cfg_max, weights, max(Bs), max(ks), cfg_max["ctx"][2])
+    del weights
+    torch.cuda.empty_cache()
+    stream = torch.cuda.current_stream()
+    cells = []
+    for B in Bs:
+        cfg = synth.get_config(f"sweep_8b_B{B}_k8")
+        batch = synth.make_request_batch(cfg, device=dev, seed_offset=1000 * rank)
+        ctx = batch["ctx_lens_host"]
+        max_ctx = max(ctx)
+        for k in ks:
+            ids = torch.empty((B, k), dtype=torch.int32, device=dev)
+
+            def step():
+                hs.hspec_draft_block(drafter.handle, batch["page_table"], batch["ctx_lens"], batch["last_hidden"],
+                                     batch["last_token"], k, batch["k_pools"], batch["v_pools"], drafter.workspace, ids,
+                                     max_ctx=max_ctx)
+            for _ in range(max(warmup, 3)):
+                step()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(steps):
+                step()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / steps
+            hs.hspec_set_profiling(drafter.handle, True)
+            att_ms, n_prof = 0.0, 2
+            for _ in range(n_prof):
+                step()
+                att_ms += sum(e["ms"] for e in hs.hspec_get_profile(drafter.handle) if e["name"] == "attn_partial")
+            hs.hspec_set_profiling(drafter.handle, False)
+            att_ms /= n_prof
+            a = workload_accounting(dict(cfg, k=k), ctx, B, k)
+            hbm_ms = (a["weight_bytes"] + a["kv_bytes"]) / (peaks["hbm_gbs"] * 1e9) * 1e3
+            tensor_ms = (a["gemm_flops"] + a["attn_flops"]) / (peaks["bf16_tflops_sustained"] * 1e12) * 1e3
+            cells.append(dict(
+                B=B, k=k, ms_per_step=round(ms, 4), draft_tokens_per_s=round(B * k / (ms * 1e-3), 1),
+                hbm_roofline_frac=round(hbm_ms / ms, 4), max_roofline_frac=round(max(hbm_ms, tensor_ms) / ms, 4),
+                attention_frac_of_hbm=round(a["kv_bytes"] / (att_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4) if att_ms > 0 else None,
+                kv_GB_read=round(a["kv_bytes"] / 1e9, 3),
+                drafter_kv_GB_avoided=round(a["drafter_kv_bytes_avoided"] / 1e9, 3),
+                drafter_kv_GB_avoided_single_tensor=round(a["drafter_kv_bytes_avoided"] / 2e9, 3)))
+        stats = drafter.stats()
+        assert stats["rc"] == 0, f"device status block not clean: {stats}"
+        del batch
+        torch.cuda.empty_cache()
+    drafter.close()
+    torch.cuda.empty_cache()
+    return dict(workload="sweep_8b_B<B>_k<k>: 8B-class drafter, contexts uniform in [1024, 16384], full context",
+                steps_per_cell=steps, weight_GB=round(a["weight_bytes"] / 1e9, 3),
+                drafter_kv_note="bytes a drafter-side KV cache over the same contexts would hold (K and V, 2 layers: 8 KiB per "
+                                "token; single_tensor = 2 layers x 8 heads x 128 x 2 B = 4 KiB per token) vs 0 for in-place reuse",
+                cells=cells)
+
+
+# ----------------------------------------------------------------------------- single-kernel cases (profiler captures)
+
+def _randn(shape, seed, std, dtype):
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std).to(dtype)
+
+
+def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16):
+    """One attention layer of the serving shapes: dh = 128, contexts uniform in [lo, hi]."""
+    import paper_2609_24197_b200 as hs
+    dh = 128
+    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16, B=B, ctx=("uniform", lo, hi))
+    ctx = synth.make_ctx_lens(cfg)
+    batch = synth.make_request_batch(cfg, ctx_lens=ctx, device="cuda")
+    M = B * k
+    q, kb, vb = (_randn((M, h, dh), s, 1.0, torch.bfloat16) for h, s in ((Hq, 1), (Hkv, 2), (Hkv, 3)))
+    o = torch.empty((M, Hq * dh), dtype=torch.float16, device="cuda")
+    mc = max(ctx)
+    ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, mc, 0, 0), dtype=torch.uint8, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for i in range(reps):
+        hs.hspec_op_attention(q, kb, vb, batch["k_pools"][0], batch["v_pools"][0], batch["page_table"],
+                              batch["ctx_lens"], mc, o, B, k, Hq, Hkv, dh, 16, 0, 0, ws)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    kv_bytes = sum(ctx) * Hkv * dh * 2 * 2
+    us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(reps)]
+    print(f"attention: B={B} k={k} Hq={Hq} Hkv={Hkv} sum ctx={sum(ctx)} target-KV bytes per launch={kv_bytes} "
+          f"us per call={[round(u, 1) for u in us]} -> {kv_bytes / (min(us) * 1e-6) / 1e12:.2f} TB/s")
+
+
+def case_gemm(reps, M=2048, n_out=25600, K=5120):
+    import paper_2609_24197_b200 as hs
+    x, W = _randn((M, K), 4, 1.0, torch.float16), _randn((n_out, K), 5, 0.02, torch.float16)
+    y = torch.empty((M, n_out), dtype=torch.float32, device="cuda")
+    ws = torch.empty(hs.hspec_gemm_workspace_bytes(M, n_out, K), dtype=torch.uint8, device="cuda")
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for i in range(reps):
+        hs.hspec_op_gemm(x, W, y, workspace=ws)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(reps)]
+    print(f"gemm: M={M} n_out={n_out} K={K} flops per launch={2 * M * n_out * K} weight bytes={2 * n_out * K} "
+          f"x bytes={2 * M * K} y bytes={4 * M * n_out} us per call={[round(u, 1) for u in us]} -> "
+          f"{2 * n_out * K / (min(us) * 1e-6) / 1e12:.2f} TB/s of weights, {2 * M * n_out * K / (min(us) * 1e-6) / 1e12:.0f} TFLOP/s")
+
+
+def case_scan(reps):
+    import paper_2609_24197_b200 as hs
+    B, k, Di, P, N, G = 32, 16, 8192, 64, 128, 4
+    H = Di // P
+    ld = 2 * Di + 2 * G * N + H
+    zx = _randn((B * k, ld), 6, 1.0, torch.float32)
+    s0 = _randn((B, H, P, N), 7, 1.0, torch.float16)
+    cw, cb = _randn((Di + 2 * G * N, 4), 8, 0.3, torch.float32), _randn((Di + 2 * G * N,), 9, 0.02, torch.float32)
+    dtb, Al, Ds = _randn((H,), 10, 1.0, torch.float32) - 4, torch.rand(H, device="cuda") * 2, torch.ones(H, device="cuda")
+    y = torch.empty((B * k, Di), dtype=torch.float32, device="cuda")
+    ws = torch.empty(hs.hspec_scan_workspace_bytes(B, k, Di, N, G), dtype=torch.uint8, device="cuda")
+    for _ in range(reps):
+        hs.hspec_op_mamba_scan(zx, None, s0, cw, cb, dtb, Al, Ds, y, B, k, Di, P, N, G, 4, ws)
+    torch.cuda.synchronize()
+    print(f"scan: B={B} H={H} S_init bytes per launch={B * H * P * N * 2}")
+
+
+CASES = {
+    # name: (function, keyword arguments) - each runs ONE kernel family a few times on inputs larger than L2
+    "attention": (case_attention, {}),                                             # 8B-class, 64 query rows per KV head
+    "attention32b": (case_attention, dict(Hq=64, Hkv=8, B=16, lo=2048, hi=16384)),  # 32B-class, 128 rows per KV head
+    "gemm": (case_gemm, {}),                                                       # the 2-SM kernel, M = 2048
+    "gemm_skinny": (case_gemm, dict(M=32, n_out=65536, K=4096)),                   # weight streaming, Proj_dS class
+    "gemm_skinny64": (case_gemm, dict(M=64, n_out=262144, K=5120)),                # Proj_dS at concurrency 64 (a fifth of it)
+    "gemm_skinny128": (case_gemm, dict(M=128, n_out=262144, K=5120)),              # Proj_dS at concurrency 128 (a fifth of it)
+    "scan": (case_scan, {}),
+}
+
+
+def main_case(args):
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --case needs a CUDA device")
+    from paper_2609_24197_b200 import build
+    build.build()
+    fn, kw = CASES[args.case]
+    fn(args.reps, **kw)
+
+
 # ----------------------------------------------------------------------------- entry points
 
 def main_ours(args):
@@ -436,11 +672,24 @@ def main_ours(args):
         build.build()
     barrier()
     peaks = load_peaks()
+    traffic = load_traffic()
+    if args.sweep:                                 # only the sweep, as a line of its own
+        sw = run_sweep(args.steps, args.warmup, peaks, rank)
+        if rank == 0:
+            head = next(c for c in sw["cells"] if c["B"] == 128 and c["k"] == 16)
+            print(json.dumps({"metric": METRIC, "value": head["draft_tokens_per_s"], "unit": "draft tokens/s", "n_gpus": world,
+                              "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"],
+                              "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+                              "data": "synthetic", "config": {"workload": "sweep_8b_B128_k16", "note": "value = the B = 128, "
+                                                              "k = 16 cell; every cell under `sweep`"},
+                              "sweep": sw, "peaks": peaks}))
+        return
     head = run_workload(args.workload, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device(),
-                        lean=args.lean)
-    s = summarize(head, peaks)
+                        lean=args.lean, repeats=args.repeats, settle_s=args.settle_s)
+    s = summarize(head, peaks, traffic)
     e2e_ms = head["e2e"]["ms_per_step"]
     units = head["B"] * head["k"] * world
+    reg = sorted(r["ms_per_step"] for r in head["regions"])
     line = {
         "metric": METRIC, "value": round(units / (head["ms_per_step"] * 1e-3), 1), "unit": "draft tokens/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": s["ms_per_step"],
@@ -453,6 +702,10 @@ def main_ours(args):
                    "ctx_max": head["ctx_max"], "window": head["cfg"]["window"],
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "l2": f"inputs larger than L2: {s['weight_GB'] + s['kv_GB']:.1f} GB touched per step, no flush"},
+        "timing": {"regions": head["regions"], "region_steps": args.steps, "ms_per_step_min": round(reg[0], 4),
+                   "ms_per_step_median": s["ms_per_step"], "ms_per_step_max": round(reg[-1], 4),
+                   "settle_steps_untimed": head["settle_steps"],
+                   "note": "value = the median region; every region is exactly `steps` steps between one pair of CUDA events"},
         "e2e": {"value": round(units / (e2e_ms * 1e-3), 1), "unit": "draft tokens/s",
                 "h2d_bytes_per_step": head["e2e"]["h2d_bytes_per_step"],
                 "d2h_bytes_per_step": head["e2e"]["d2h_bytes_per_step"], "ms_per_step": round(e2e_ms, 4)},
@@ -482,21 +735,34 @@ def main_ours(args):
         byc = {}
         for conc, name in BY_CONCURRENCY.items():
             if name == args.workload:
-                byc[conc] = dict(workload=name, draft_tokens_per_s=s["draft_tokens_per_s"], ms_per_step=s["ms_per_step"],
-                                 hbm_roofline_frac=s["hbm_roofline_frac"], max_roofline_frac=s["max_roofline_frac"],
-                                 attention_frac_of_hbm=s["attention"]["frac_of_hbm"],
-                                 graph_replay_ms_per_step=s["graph_replay_ms_per_step"])
+                byc[conc] = dict(brief(s, head), workload=name)
                 continue
-            r = run_workload(name, args.steps, args.warmup, rank, want_e2e=False)
-            t = summarize(r, peaks)
-            byc[conc] = dict(workload=name, draft_tokens_per_s=t["draft_tokens_per_s"], ms_per_step=t["ms_per_step"],
-                             hbm_roofline_frac=t["hbm_roofline_frac"], max_roofline_frac=t["max_roofline_frac"],
-                             attention_frac_of_hbm=t["attention"]["frac_of_hbm"],
-                             graph_replay_ms_per_step=t["graph_replay_ms_per_step"], gemm=t["gemm"],
-                             kernels=kernel_table(r))
+            r = run_workload(name, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device(), want_e2e=False,
+                             settle_s=min(args.settle_s, 1.0))
+            t = summarize(r, peaks, traffic)
+            byc[conc] = dict(brief(t, r), workload=name, gemm=t["gemm"], rooflines=t["rooflines"], kernels=kernel_table(r))
             del r
             torch.cuda.empty_cache()
         line["by_concurrency"] = byc
+        # the paper's 2048-token sliding window (App. B.1) on the two serving workloads, beside the full-context rows
+        win = {}
+        for name in ("serving_8b", "conc128_32b"):
+            try:
+                r = run_workload(name, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device(), want_e2e=False,
+                                 settle_s=min(args.settle_s, 1.0), want_graph=False, window=2048)
+                t = summarize(r, peaks, traffic)
+                win[name] = dict(brief(t, r), window=2048, attention=t["attention"])
+                del r
+            except Exception as exc:
+                print(f"[bench] window row of {name} skipped: {exc}", file=sys.stderr)
+            torch.cuda.empty_cache()
+        line["window_2048"] = win
+        if not args.no_sweep:
+            try:
+                line["sweep"] = run_sweep(args.sweep_steps, args.warmup, peaks, rank)
+            except Exception as exc:
+                print(f"[bench] sweep skipped: {exc}", file=sys.stderr)
+            torch.cuda.empty_cache()
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -547,14 +813,27 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--repeats", type=int, default=5, help="timed regions of --steps steps each; value = the median one")
+    ap.add_argument("--settle-s", type=float, default=2.0,
+                    help="seconds of untimed steps after the warm-up, so the clocks have settled under the power cap")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE,
                     help="one of %s, or a sweep cell sweep_8b_B<B>_k<k>" % ", ".join(sorted(synth.CONFIGS)))
-    ap.add_argument("--headline-only", action="store_true", help="skip the concurrency-1 and -32 workloads")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the concurrency-1 / -32 workloads, the window rows and the sweep")
+    ap.add_argument("--no-sweep", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run only the concurrency x block-size sweep (--steps per cell)")
+    ap.add_argument("--sweep-steps", type=int, default=10, help="timed steps per sweep cell inside the default run")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lean", action="store_true", help="only warm-up + timed steps (for profiler launch lists)")
+    ap.add_argument("--case", choices=sorted(CASES), help="run one kernel on a small case (for profiler captures) and exit")
+    ap.add_argument("--reps", type=int, default=3, help="launches of --case")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.lean:
+        args.repeats, args.settle_s = 1, 0.0
+    if args.case:
+        main_case(args)
+    elif args.impl == "reference":
         main_reference(args)
     else:
         main_ours(args)

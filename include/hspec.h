@@ -23,7 +23,11 @@
  *   bf16 activations (8 bits) put the step's rounding noise at ~3e-2 of the output RMS over a full logits
  *   tensor, above the 2e-2 parity bound.  Accumulation is fp32; the residual stream, scan and softmax are
  *   fp32.  The target's KV pools are read in place as bf16, so q, the block's k/v and the softmax weights
- *   enter the attention MMAs as bf16.  fp16 saturates at 65504: hidden states beyond that are out of range.
+ *   enter the attention MMAs as bf16.
+ *   Range: fp16 ends at 65504.  |last_hidden| and every GEMM input the library forms must stay below that; a finite
+ *   value beyond it is CLAMPED to +-65504 at the store (never turned into inf) and counted, and hspec_get_stats then
+ *   returns HSPEC_ERR_F16_RANGE with the count in f16_range_events.  A target whose hidden states carry outlier channels
+ *   above 65504 needs them scaled by the caller (Proj_r is linear: scale last_hidden by s and proj_r by 1/s).
  *
  * Conventions
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers are
@@ -56,9 +60,12 @@ typedef enum {
   HSPEC_ERR_BAD_SHAPE = -2,          /* config or tensor shape the kernels cannot take */
   HSPEC_ERR_NOT_LOADED = -3,         /* a required weight tensor was never loaded */
   HSPEC_ERR_WORKSPACE_TOO_SMALL = -4,
-  HSPEC_ERR_PAGE_OUT_OF_RANGE = -5,  /* host-side validation of a page table found a bad id */
+  HSPEC_ERR_PAGE_OUT_OF_RANGE = -5,  /* a page id outside [0, num_pages) or a context length outside [0, max_ctx]: found by the
+                                        host-side validation (HSPEC_DEBUG=1, before anything is enqueued) or met by a kernel,
+                                        which clamps the length, reads the page as zeros and counts the event */
   HSPEC_ERR_CUDA = -6,               /* a CUDA runtime / driver call failed (message has the text) */
-  HSPEC_ERR_TIMEOUT = -7             /* a bounded in-kernel wait gave up (status word) */
+  HSPEC_ERR_TIMEOUT = -7,            /* a bounded in-kernel wait gave up (status word) */
+  HSPEC_ERR_F16_RANGE = -8           /* finite values beyond +-65504 reached an fp16 store and were clamped (counted) */
 } hspec_status;
 
 typedef enum { HSPEC_BF16 = 0, HSPEC_F32 = 1, HSPEC_I32 = 2, HSPEC_F16 = 3 } hspec_dtype;
@@ -153,6 +160,10 @@ typedef struct {
   uint32_t device_status;     /* 0, or a code written by a bounded in-kernel wait that gave up
                                  (reading it synchronises the handle's last stream) */
   uint32_t launches_last_step;
+  uint32_t attn_rescales;     /* informational: (warp, key tile) events in which the attention kernel moved a row's reference
+                                 maximum and rescaled its accumulator (peaked score rows; never an error) */
+  uint32_t f16_range_events;  /* finite values that left the fp16 range in a store and were clamped to +-65504 */
+  uint32_t bad_inputs;        /* out-of-range context lengths / page ids met by a kernel (clamped / read as zeros) */
 } hspec_stats;
 
 /* One kernel launch of the last step, as recorded when profiling is on. */
@@ -162,6 +173,7 @@ typedef struct {
   double flops;      /* algorithmic flops of the launch (GEMMs: 2*M*N*K), 0 if not a contraction */
   double bytes;      /* algorithmic bytes where the library knows them without the context lengths (GEMMs: the
                         weight matrix; scan: S_init), else 0 */
+  double io_bytes;   /* GEMMs: activation bytes read and result bytes written besides the weights, else 0 */
 } hspec_prof_entry;
 
 /* Validates the config, creates the handle (host memory only; no weights yet).  Sec. 3.3 / App. B.1. */
@@ -181,6 +193,9 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
 int hspec_destroy(hspec_handle* h);
 /* Message of the last failure on this handle (or of the last failed hspec_init if h is NULL). */
 const char* hspec_last_error(const hspec_handle* h);
+/* Reads the handle's counters and device status block (synchronises the handle's last stream).  Returns HSPEC_OK, or
+ * the most severe condition recorded since the last hspec_clear_status: HSPEC_ERR_TIMEOUT (device_status != 0),
+ * HSPEC_ERR_PAGE_OUT_OF_RANGE (bad_inputs != 0), HSPEC_ERR_F16_RANGE (f16_range_events != 0); `out` is filled either way. */
 int hspec_get_stats(hspec_handle* h, hspec_stats* out);
 /* Failure-path self-test: enqueues a one-thread kernel that waits, for at most limit_ms (1..2000), on a barrier nothing
  * completes; it then gives up, writes a code to the handle's device status word and returns normally (no trap: the
@@ -225,6 +240,13 @@ int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t in_dtype, int3
  * Inputs and outputs are the caller's, as in hspec_op_lm_head_argmax; results are identical to it. */
 int hspec_op_lm_head_argmax_noalloc(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M,
                                     int32_t V, int32_t K, void* stream);
+/* Status of the hspec_op_* entry points, which take no handle: synchronises the current device, then reads the status
+ * block those calls share on this device and the one inside the allocation-free entry point's built-in array.
+ * words4 (host, may be NULL) receives {give-up code of a bounded wait or 0, attention rescale events, fp16 range events,
+ * out-of-range inputs}; clear != 0 zeroes the blocks afterwards.  Returns like hspec_get_stats.  A handle-less call
+ * whose bounded wait gave up has already returned HSPEC_OK when it was enqueued: this is the only place where that
+ * shows (arg-max ids of such a call are 0x7fffffff). */
+int hspec_op_device_status(uint32_t* words4, int32_t clear);
 /* Acceptance rule of speculative decoding (App. A): draft i of request b is accepted if every earlier draft of b
  * was and min(1, P_T / P_D) >= alpha.  p_target, p_draft, alpha: device fp32 [B, k] (probabilities of the drafted
  * tokens under the target and under the drafter, and the caller's uniform draws); n_accept: device int32 [B], the

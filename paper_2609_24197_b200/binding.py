@@ -23,7 +23,7 @@ EXPORTS = [
     "hspec_op_lm_head_argmax", "hspec_op_lm_head_argmax_noalloc", "hspec_op_rmsnorm", "hspec_op_mamba_scan", "hspec_scan_workspace_bytes", "hspec_op_qk_norm_rope",
     "hspec_op_attention", "hspec_attention_workspace_bytes", "hspec_debug_gather_kv", "hspec_op_swiglu",
     "hspec_op_accept", "hspec_op_token_probs", "hspec_op_markov_head", "hspec_markov_workspace_bytes",
-    "hspec_op_kv_inject_write",
+    "hspec_op_kv_inject_write", "hspec_op_device_status",
 ]
 
 
@@ -63,11 +63,13 @@ class hspec_out(C.Structure):
 
 
 class hspec_stats(C.Structure):
-    _fields_ = [("kernel_launches", C.c_uint64), ("device_status", C.c_uint32), ("launches_last_step", C.c_uint32)]
+    _fields_ = [("kernel_launches", C.c_uint64), ("device_status", C.c_uint32), ("launches_last_step", C.c_uint32),
+                ("attn_rescales", C.c_uint32), ("f16_range_events", C.c_uint32), ("bad_inputs", C.c_uint32)]
 
 
 class hspec_prof_entry(C.Structure):
-    _fields_ = [("name", C.c_char * 40), ("ms", C.c_float), ("flops", C.c_double), ("bytes", C.c_double)]
+    _fields_ = [("name", C.c_char * 40), ("ms", C.c_float), ("flops", C.c_double), ("bytes", C.c_double),
+                ("io_bytes", C.c_double)]
 
 
 _lib = None
@@ -119,6 +121,7 @@ def load_library(path=None):
     lib.hspec_attention_workspace_bytes.restype = sz
     lib.hspec_debug_gather_kv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp]
     lib.hspec_op_swiglu.argtypes = [vp, vp, i32, i32, vp]
+    lib.hspec_op_device_status.argtypes = [C.POINTER(C.c_uint32), i32]
     if path == LIB_PATH:
         _lib = lib
     return lib
@@ -226,7 +229,15 @@ def hspec_get_stats(handle):
     s = hspec_stats()
     rc = load_library().hspec_get_stats(handle, C.byref(s))
     return dict(kernel_launches=int(s.kernel_launches), device_status=int(s.device_status),
-                launches_last_step=int(s.launches_last_step), rc=rc)
+                launches_last_step=int(s.launches_last_step), attn_rescales=int(s.attn_rescales),
+                f16_range_events=int(s.f16_range_events), bad_inputs=int(s.bad_inputs), rc=rc)
+
+
+def hspec_op_device_status(clear=False):
+    """Status block of the handle-less hspec_op_* calls on the current device (synchronises it)."""
+    w = (C.c_uint32 * 4)()
+    rc = load_library().hspec_op_device_status(w, int(bool(clear)))
+    return dict(device_status=int(w[0]), attn_rescales=int(w[1]), f16_range_events=int(w[2]), bad_inputs=int(w[3]), rc=rc)
 
 
 def hspec_debug_wait_selftest(handle, limit_ms=100):
@@ -247,8 +258,8 @@ def hspec_get_profile(handle, max_entries=512):
     n = load_library().hspec_get_profile(handle, arr, max_entries)
     if n < 0:
         _check(n, handle, "hspec_get_profile")
-    return [dict(name=arr[i].name.decode(), ms=float(arr[i].ms), flops=float(arr[i].flops), bytes=float(arr[i].bytes))
-            for i in range(n)]
+    return [dict(name=arr[i].name.decode(), ms=float(arr[i].ms), flops=float(arr[i].flops), bytes=float(arr[i].bytes),
+                 io_bytes=float(arr[i].io_bytes)) for i in range(n)]
 
 
 # ----------------------------------------------------------------------------- single operations

@@ -26,11 +26,17 @@ struct AttnArgs {
   float* ws_o;       // [B, Hkv, max_chunks, R, DH]
   float* ws_ml;      // [B, Hkv, max_chunks, R, 2]
   __half* o;         // [B*k, Hq*DH]
+  uint32_t* status;
   int page_table_stride;
   int B, k, Hq, Hkv, rep, R, RT, n_row_tiles;
   int chunk, max_chunks, page_size, window;
+  int max_ctx;       // host bound on the context lengths: a length outside [0, max_ctx] is clamped and counted
+  int num_pages;     // a page id outside [0, num_pages) is read as zeros and counted
   float scale_log2;
 };
+
+// A request's context length as both kernels use it: clamped to the bound the host sized the grid and the partials for.
+__device__ __forceinline__ int clamped_ctx(const AttnArgs& a, int b) { return min(max(a.ctx_lens[b], 0), a.max_ctx); }
 
 // Visible prefix range of a request: [lo0, ctx).  With a window W row i sees positions
 // > ctx + i - W, so the union over rows starts at ctx - W + 1 (row 0).
@@ -54,7 +60,8 @@ attn_partial_kernel(AttnArgs a) {
   const int tid = threadIdx.x, nthr = blockDim.x, warp = tid >> 5, lane = tid & 31;
   const int b = blockIdx.z, kvh = blockIdx.y;
   const int c = blockIdx.x / a.n_row_tiles, rt = blockIdx.x % a.n_row_tiles;
-  const int ctx = a.ctx_lens[b];
+  const int ctx = clamped_ctx(a, b);
+  if (tid == 0 && blockIdx.x == 0 && kvh == 0 && ctx != a.ctx_lens[b]) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
   int lo0, n_chunks;
   visible_range(ctx, a.window, a.chunk, lo0, n_chunks);
   if (c >= n_chunks) return;
@@ -90,11 +97,16 @@ attn_partial_kernel(AttnArgs a) {
       for (int idx = tid; idx < KT * CPR; idx += nthr) {
         const int r = idx / CPR, ch = idx % CPR;
         const int p = base + r;
-        const bool ok = p < p_end;
+        bool ok = p < p_end;
         size_t off = 0;
         if (ok) {
           const int page = ptab[p / a.page_size];
-          off = ((size_t(page) * a.page_size + (p % a.page_size)) * a.Hkv + kvh) * DH + ch * 8;
+          if (unsigned(page) >= unsigned(a.num_pages)) {     // never form an address from a bad id: zero row, counted once
+            ok = false;
+            if (ch == 0 && p % a.page_size == 0) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
+          } else {
+            off = ((size_t(page) * a.page_size + (p % a.page_size)) * a.Hkv + kvh) * DH + ch * 8;
+          }
         }
         cp_async16(dK + swz<DH>(r, ch * 8), a.k_pool + off, ok);
         cp_async16(dV + swz<DH>(r, ch * 8), a.v_pool + off, ok);
@@ -245,7 +257,7 @@ __global__ void attn_merge_kernel(AttnArgs a) {
   const int hq = blockIdx.y;
   const int b = m / a.k, i = m % a.k;
   const int kvh = hq / a.rep, r = i * a.rep + hq % a.rep;
-  const int ctx = a.ctx_lens[b];
+  const int ctx = clamped_ctx(a, b);
   int lo0, n_chunks;
   visible_range(ctx, a.window, a.chunk, lo0, n_chunks);
   const size_t slab0 = (size_t(b) * a.Hkv + kvh) * a.max_chunks;
@@ -260,7 +272,7 @@ __global__ void attn_merge_kernel(AttnArgs a) {
       L += ml[1] * w;
       acc += a.ws_o[((slab0 + c) * a.R + r) * DH + d] * w;
     }
-    a.o[(size_t(m) * a.Hq + hq) * DH + d] = __float2half_rn(acc / L);
+    a.o[(size_t(m) * a.Hq + hq) * DH + d] = f16_sat(acc / L, a.status);
   }
 }
 
@@ -322,6 +334,9 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* tr
   a.R = c.k * a.rep; a.RT = rows_per_cta(a.R); a.n_row_tiles = (a.R + a.RT - 1) / a.RT;
   a.chunk = c.chunk_tokens; a.max_chunks = max_chunks_of(c.max_ctx, c.window, c.chunk_tokens);
   a.page_size = c.page_size; a.window = c.window;
+  a.status = c.status;
+  a.max_ctx = c.max_ctx < c.page_table_stride * c.page_size ? c.max_ctx : c.page_table_stride * c.page_size;
+  a.num_pages = int(c.num_pages < 0x7fffffff ? c.num_pages : 0x7fffffff);
   a.scale_log2 = 1.4426950408889634f / sqrtf(float(c.dh));
   if (c.k > KT) { if (err) *err = "block longer than one key tile"; return cudaErrorInvalidValue; }
   const size_t need = attn_workspace_bytes(c.B, c.k, c.Hq, c.Hkv, c.dh, c.max_ctx, c.window, c.chunk_tokens);
@@ -336,17 +351,16 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* tr
   const size_t smem = size_t(a.RT) * c.dh * 2 + size_t(2) * NSTAGE * KT * c.dh * 2;
   dim3 grid(a.max_chunks * a.n_row_tiles, c.Hkv, c.B);
   const int threads = a.RT * 2;
-  cudaError_t e;
+  static bool attr_done[MAX_DEVICES] = {};
+  cudaError_t e = once_per_device(attr_done, [](int) {
+    cudaError_t e2 = cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e2 != cudaSuccess) return e2;
+    return cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  });
+  if (e != cudaSuccess) return e;
   trk_begin(trk, "attn_partial");
-  if (c.dh == 128) {
-    static bool set128 = false;
-    if (!set128) { e = cudaFuncSetAttribute(attn_partial_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); if (e != cudaSuccess) return e; set128 = true; }
-    attn_partial_kernel<128><<<grid, threads, smem, stream>>>(a);
-  } else {
-    static bool set64 = false;
-    if (!set64) { e = cudaFuncSetAttribute(attn_partial_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); if (e != cudaSuccess) return e; set64 = true; }
-    attn_partial_kernel<64><<<grid, threads, smem, stream>>>(a);
-  }
+  if (c.dh == 128) attn_partial_kernel<128><<<grid, threads, smem, stream>>>(a);
+  else attn_partial_kernel<64><<<grid, threads, smem, stream>>>(a);
   trk_end(trk);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -51,8 +51,14 @@ struct AttnTcArgs {
   int page_table_stride;
   int B, k, Hq, Hkv, rep, R, n_row_tiles;
   int chunk, max_chunks, window;
+  int max_ctx;           // host bound on the context lengths: a length outside [0, max_ctx] is clamped and counted
+  int num_pages;         // pages in each pool: a page id outside [0, num_pages) is read as zeros and counted
   float scale_log2;
 };
+
+// A request's context length as every kernel of the attention uses it: the device array's value clamped to the bound
+// the host sized the work list, the partials and the page-table row for.
+__device__ __forceinline__ int clamped_ctx(const AttnTcArgs& a, int b) { return min(max(a.ctx_lens[b], 0), a.max_ctx); }
 
 struct __align__(8) AttnTcBars {
   uint64_t q_ready, o_done, o_free, l_ready;
@@ -197,6 +203,14 @@ __device__ __forceinline__ Item unpack_item(const int4 w) {
   return it;
 }
 
+// The n-th item of this CTA.  The list is sorted longest first; handing round n out in ascending CTA order for even n and
+// in descending order for odd n evens out the CTAs' shares (plain round-robin gives CTA 0 the longest item of every
+// round).  Once an index falls past the end of the list, every later one does too.
+__device__ __forceinline__ int item_at(int n) {
+  const int G = int(gridDim.x), c = int(blockIdx.x);
+  return n * G + ((n & 1) ? G - 1 - c : c);
+}
+
 // Work list: one item per (request, KV head, context chunk, 128-row tile), longest first (bucketed by tile count),
 // heads of one request and chunk next to each other so the CTAs that run them at the same time read neighbouring
 // bytes of the same pages.  The order inside a bucket depends on atomics; every item is computed independently, so
@@ -212,7 +226,8 @@ __global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4*
   __syncthreads();
   for (int i = threadIdx.x; i < pairs; i += blockDim.x) {
     const int b = i / a.max_chunks, c = i % a.max_chunks;
-    const Range g = make_range(a.ctx_lens[b], a.window, a.chunk, c, a.k);
+    if (c == 0 && a.ctx_lens[b] != clamped_ctx(a, b)) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
+    const Range g = make_range(clamped_ctx(a, b), a.window, a.chunk, c, a.k);
     if (c < g.n_chunks) atomicAdd(&bucket[min(g.T, 63)], per_chunk);
   }
   __syncthreads();
@@ -224,7 +239,7 @@ __global__ void attn_tc_plan_kernel(AttnTcArgs a, int* __restrict__ count, int4*
   __syncthreads();
   for (int i = threadIdx.x; i < pairs; i += blockDim.x) {
     const int b = i / a.max_chunks, c = i % a.max_chunks;
-    const int ctx = a.ctx_lens[b];
+    const int ctx = clamped_ctx(a, b);
     const Range g = make_range(ctx, a.window, a.chunk, c, a.k);
     if (c >= g.n_chunks) continue;
     int at = atomicAdd(&offset[min(g.T, 63)], per_chunk);
@@ -245,10 +260,10 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
                                                 volatile uint32_t* abort_flag, const int4* __restrict__ items, int n_items,
                                                 int lane, int ns) {
   uint32_t gt = 0;                                 // tiles issued so far, across items
-  int4 w_next = items[blockIdx.x];
-  for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
+  int4 w_next = items[item_at(0)];
+  for (int n = 0; item_at(n) < n_items; ++n) {
     const Item wi = unpack_item(w_next);
-    if (it + int(gridDim.x) < n_items) w_next = items[it + gridDim.x];     // consumed one item later
+    if (item_at(n + 1) < n_items) w_next = items[item_at(n + 1)];         // consumed one item later
     const int b = wi.b, kvh = wi.kvh;
     const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
     const int32_t* ptab = a.page_table + size_t(b) * a.page_table_stride;
@@ -269,6 +284,8 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
         if (lane == 0) mbar_expect_tx(bar, KV_BYTES);
         __syncwarp();
         if (lane < KT / 16) {
+          // (a page id outside the pool is outside the tensor map: the copy delivers zeros and touches no memory)
+          if (unsigned(page_cur) >= unsigned(a.num_pages)) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
           tma_load_4d(smem_u32(dst) + lane * 2048, tm, 0, kvh, 0, page_cur, bar);
           tma_load_4d(smem_u32(dst) + KV_HALF + lane * 2048, tm, 64, kvh, 0, page_cur, bar);
         }
@@ -281,18 +298,24 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
         __syncwarp();
         if (lane < full_pages) {
           const int page = ptab[(prefix_start >> 4) + lane];
+          if (unsigned(page) >= unsigned(a.num_pages)) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
           tma_load_4d(smem_u32(dst) + lane * 2048, tm, 0, kvh, 0, page, bar);
           tma_load_4d(smem_u32(dst) + KV_HALF + lane * 2048, tm, 64, kvh, 0, page, bar);
         }
         for (int idx = lane; idx < (KT - tma_rows) * 16; idx += 32) {
           const int r = tma_rows + (idx >> 4), chunk16 = idx & 15;
-          const bool valid = r < n_prefix + n_block;
+          bool valid = r < n_prefix + n_block;
           size_t off = 0;
           const __nv_bfloat16* src = pool;
           if (r < n_prefix) {
             const int p = prefix_start + r;
             const int page = ptab[p >> 4];
-            off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
+            if (unsigned(page) >= unsigned(a.num_pages)) {       // never form an address from a bad id: zero row, counted once
+              valid = false;
+              if (chunk16 == 0 && (p & 15) == 0) atomicAdd(a.status + STATUS_WORD_BAD_INPUT, 1u);
+            } else {
+              off = ((size_t(page) * 16 + (p & 15)) * a.Hkv + kvh) * DH + chunk16 * 8;
+            }
           } else if (valid) {
             src = blk;
             off = ((size_t(b) * a.k + (r - n_prefix)) * a.Hkv + kvh) * DH + chunk16 * 8;
@@ -309,7 +332,7 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
   }
 }
 
-// Persistent: one CTA per SM walks the work list (item = blockIdx.x, + gridDim.x, ...).  All ring and buffer indices
+// Persistent: one CTA per SM walks the work list (items item_at(0), item_at(1), ...).  All ring and buffer indices
 // count tiles across items (gt): K slot = gt % NSK, V slot = gt % NSV, S / P buffer = gt & 1.
 __global__ void __launch_bounds__(352, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a,
@@ -323,7 +346,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int n_items = *count;
-  if (int(blockIdx.x) >= n_items) return;           // uniform for the whole CTA
+  if (item_at(0) >= n_items) return;                // uniform for the whole CTA
   if (smem_u32(smem) & 1023) {                      // the swizzled operand tiles need a 1 KiB-aligned base
     if (tid == 0) atomicExch(a.status, STATUS_BAD_SMEM_BASE);
     return;
@@ -404,10 +427,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         umma_commit(smem_u32(&bars->s_ready[g_t & 1]));
         return true;
       };
-      int4 w_next = items[blockIdx.x];
-      for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n) {
+      int4 w_next = items[item_at(0)];
+      for (; item_at(int(n)) < n_items && ok; ++n) {
         const Item wi = unpack_item(w_next);
-        if (it + int(gridDim.x) < n_items) w_next = items[it + gridDim.x];
+        if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
         const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
         MCLK(0)
         if (!mbar_wait(smem_u32(&bars->q_ready), n & 1)) { ok = false; break; }      // this item's Q tile is in place
@@ -495,29 +518,41 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->q_ready));
     };
-    int4 w_cur = items[blockIdx.x];
-    int4 w_next = (int(blockIdx.x + gridDim.x) < n_items) ? items[blockIdx.x + gridDim.x] : w_cur;
+    int4 w_cur = items[item_at(0)];
+    int4 w_next = (item_at(1) < n_items) ? items[item_at(1)] : w_cur;
     {
       uint4 qv[8];
       load_q(unpack_item(w_cur), qv);
       store_q(qv);
     }
-    for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n) {
+    for (; item_at(int(n)) < n_items && ok; ++n) {
       const Item wi = unpack_item(w_cur);
       const int b = wi.b, kvh = wi.kvh, c = wi.c, ctx = wi.ctx;
       const Range g = make_range(ctx, a.window, a.chunk, c, a.k);
       const int rg = wi.rt * 128 + r_local;          // row among the k * rep rows of this KV head
       const bool row_ok = rg < a.R;
       const int i_blk = rg / a.rep;                  // block position of the row
-      const bool has_next = it + int(gridDim.x) < n_items;
+      const bool has_next = item_at(int(n) + 1) < n_items;
       int4 w_next2 = w_next;                         // the descriptor is fetched two items ahead
-      if (it + 2 * int(gridDim.x) < n_items) w_next2 = items[it + 2 * gridDim.x];
+      if (item_at(int(n) + 2) < n_items) w_next2 = items[item_at(int(n) + 2)];
       if (has_next) prefetch_q(unpack_item(w_next));
       float m_ref = NEG, l_sum = 0.f;
+      // a warp all of whose 32 rows are padding (fewer than 128 query rows share the KV head) only keeps the
+      // barriers' arrival counts: its rows of S, P and O are never read, and a row of P feeds no other row of O
+      const bool warp_live = wi.rt * 128 + (warp & 3) * 32 < a.R;
       TCLK(0)
       for (int t = 0; t < g.T && ok; ++t, ++gt) {
         const uint32_t t_s = tmem_s0 + (gt & 1) * 128 + lane_base;
         if (!mbar_wait(smem_u32(&bars->s_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
+        if (!warp_live) {
+          // (waiting for the tile's scores keeps this warp in step: the same barrier's next phase cannot begin before
+          // every warp has arrived on this one)
+          if (lane == 0) {
+            mbar_arrive(smem_u32(&bars->x_ready[gt & 1]));
+            mbar_arrive(smem_u32(&bars->p_ready[gt & 1]));
+          }
+          continue;
+        }
         tc_fence_after();
         TCLK(1)
         float s[64];
@@ -573,6 +608,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           // tile's V slot is committed behind its P V product); each thread rescales its 64 columns
           if (!mbar_wait(smem_u32(&bars->v_empty[(gt - 1) % NSV]), ((gt - 1) / NSV) & 1)) { ok = false; break; }
           tc_fence_after();
+          if (lane == 0 && hf == 0) atomicAdd(a.status + STATUS_WORD_RESCALES, 1u);   // rare; lets a test see the branch run
 #pragma unroll
           for (int j = 0; j < 2; ++j) {
             uint32_t o[32];
@@ -627,7 +663,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       }
       const size_t slab = (size_t(b) * a.Hkv + kvh) * a.max_chunks + c;
       const bool whole = g.n_chunks == 1;            // the request's only chunk: normalise and finish here
-      if (whole) {
+      if (!warp_live) {
+        // nothing to read out
+      } else if (whole) {
         // (the last chunk always holds the row's own block key, so the row sum is positive)
         const float inv = 1.f / l_row;
         __half* dsth = a.o_final + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH + hf * 64;
@@ -642,7 +680,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
               uint32_t h[4];
 #pragma unroll
               for (int q2 = 0; q2 < 4; ++q2) {
-                const __half2 v = __floats2half2_rn(__uint_as_float(o[e + 2 * q2]) * inv, __uint_as_float(o[e + 2 * q2 + 1]) * inv);
+                const __half2 v = __halves2half2(f16_sat(__uint_as_float(o[e + 2 * q2]) * inv, a.status),
+                                                 f16_sat(__uint_as_float(o[e + 2 * q2 + 1]) * inv, a.status));
                 h[q2] = *reinterpret_cast<const uint32_t*>(&v);
               }
               *reinterpret_cast<uint4*>(dsth + j * 32 + e) = make_uint4(h[0], h[1], h[2], h[3]);
@@ -701,7 +740,7 @@ __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n
   const int m = pair / a.Hq, hq = pair % a.Hq;
   const int b = m / a.k, i = m % a.k;
   const int kvh = hq / a.rep, r = i * a.rep + hq % a.rep;
-  const Range g = make_range(a.ctx_lens[b], a.window, a.chunk, 0, a.k);
+  const Range g = make_range(clamped_ctx(a, b), a.window, a.chunk, 0, a.k);
   if (g.n_chunks == 1) return;                     // finished by the attention kernel itself
   const size_t slab0 = (size_t(b) * a.Hkv + kvh) * a.max_chunks;
   float m_tot = -INFINITY;
@@ -718,10 +757,11 @@ __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n
     acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
   }
   const float inv = 1.f / L;
-  __half2 lo = __floats2half2_rn(acc.x * inv, acc.y * inv), hi = __floats2half2_rn(acc.z * inv, acc.w * inv);
+  const __half2 lo = __halves2half2(f16_sat(acc.x * inv, a.status), f16_sat(acc.y * inv, a.status));
+  const __half2 hi = __halves2half2(f16_sat(acc.z * inv, a.status), f16_sat(acc.w * inv, a.status));
   uint2 out;
-  out.x = *reinterpret_cast<uint32_t*>(&lo);
-  out.y = *reinterpret_cast<uint32_t*>(&hi);
+  out.x = *reinterpret_cast<const uint32_t*>(&lo);
+  out.y = *reinterpret_cast<const uint32_t*>(&hi);
   reinterpret_cast<uint2*>(o + (size_t(m) * a.Hq + hq) * DH)[d4] = out;
 }
 
@@ -769,6 +809,8 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   a.B = c.B; a.k = c.k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.rep = c.Hq / c.Hkv; a.R = c.k * a.rep;
   a.n_row_tiles = (a.R + 127) / 128;
   a.chunk = c.chunk_tokens; a.max_chunks = max_chunks; a.window = c.window;
+  a.max_ctx = c.max_ctx < c.page_table_stride * 16 ? c.max_ctx : c.page_table_stride * 16;
+  a.num_pages = int(c.num_pages < 0x7fffffff ? c.num_pages : 0x7fffffff);
   a.scale_log2 = 1.4426950408889634f / sqrtf(float(c.dh));
   const size_t slabs = size_t(c.B) * c.Hkv * max_chunks;
   a.ws_o = reinterpret_cast<float*>(c.ws);
@@ -778,12 +820,17 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   if (!make_pool_tmap(&tmK, c.k_pool, c.num_pages, c.Hkv, err) || !make_pool_tmap(&tmV, c.v_pool, c.num_pages, c.Hkv, err))
     return cudaErrorInvalidValue;
   const size_t smem = size_t(KV_BYTES) * (1 + NSK + NSV) + sizeof(AttnTcBars);
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) return e;
-    attr_set = true;
+  static bool attr_done[MAX_DEVICES] = {};
+  static int sm_count[MAX_DEVICES] = {};
+  {
+    const cudaError_t e0 = once_per_device(attr_done, [smem](int dev) {
+      if (cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count[dev] < 1)
+        sm_count[dev] = 148;
+      return cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+    });
+    if (e0 != cudaSuccess) return e0;
   }
+  const int n_sms = sm_count[current_device()];
   // work list (count + items) behind the partials in the workspace
   int* count = reinterpret_cast<int*>((reinterpret_cast<uintptr_t>(a.ws_ml + slabs * a.R * 2) + 15) & ~uintptr_t(15));
   int4* items = reinterpret_cast<int4*>(count + 4);
@@ -792,12 +839,6 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  static int n_sms = 0;
-  if (n_sms == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sms < 1)
-      n_sms = 148;
-  }
   trk_begin(trk, "attn_partial");
   launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(352), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
   trk_end(trk);

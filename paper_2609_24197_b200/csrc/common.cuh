@@ -7,7 +7,8 @@
 
 namespace hspec {
 
-// Codes a kernel writes to the device status word when a bounded wait gives up.
+// The device status block is 64 words.  Word 0 holds the code of a bounded wait that gave up (codes below); the
+// other words are event counters that kernels bump with atomicAdd and the host reads back with the block.
 enum : uint32_t {
   STATUS_OK = 0,
   STATUS_TIMEOUT_PRODUCER = 0x101,
@@ -16,6 +17,25 @@ enum : uint32_t {
   STATUS_BAD_SMEM_BASE = 0x104,
   STATUS_TIMEOUT_SELFTEST = 0x1ff,
 };
+enum : int {
+  STATUS_WORD_CODE = 0,        // first give-up code (0 = none)
+  STATUS_WORD_RESCALES = 1,    // attention: (warp, tile) events in which a row's reference maximum moved and its
+                               // accumulator row was rescaled in tensor memory
+  STATUS_WORD_F16_RANGE = 2,   // finite fp32 values that left the fp16 range in a store and were clamped to +-65504
+  STATUS_WORD_BAD_INPUT = 3,   // context lengths outside [0, max_ctx] and page ids outside [0, num_pages) that a kernel
+                               // met: the length was clamped, the page's rows were read as zeros
+  STATUS_WORDS = 64,
+};
+
+// fp32 -> fp16 with saturation: a finite value beyond +-65504 is clamped (instead of becoming inf and, one GEMM later,
+// NaN) and counted in the status block; NaN and inf pass through unchanged.
+__device__ __forceinline__ __half f16_sat(float v, uint32_t* status) {
+  if (fabsf(v) > 65504.f && fabsf(v) < INFINITY) {
+    if (status) atomicAdd(status + STATUS_WORD_F16_RANGE, 1u);
+    v = copysignf(65504.f, v);
+  }
+  return __float2half_rn(v);
+}
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -211,7 +231,7 @@ __device__ __forceinline__ uint32_t umma_idesc_m128(uint32_t n, bool f16) {
 // features.  Columns are handled in pairs: the lower half-warp finishes the even column, the upper half the odd one,
 // so all 32 lanes compute and store.  `f` is the feature index of this lane (same for lane and lane ^ 16).
 __device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], __half* out, long long ldo, int m_first, int M, int f,
-                                               bool f_ok, int lane) {
+                                               bool f_ok, int lane, uint32_t* status) {
   const bool upper = lane >= 16;
 #pragma unroll
   for (int j = 0; j < 16; j += 2) {
@@ -221,7 +241,7 @@ __device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], __half* 
     const float gate = upper ? recv : mine_even;               // upper half: partner's gate of the odd column
     const float up = upper ? mine_odd : recv;                  // lower half: partner's up of the even column
     const int m = m_first + j + (upper ? 1 : 0);
-    if (f_ok && m < M) out[size_t(m) * ldo + f] = __float2half_rn(silu_f(gate) * up);
+    if (f_ok && m < M) out[size_t(m) * ldo + f] = f16_sat(silu_f(gate) * up, status);
   }
 }
 

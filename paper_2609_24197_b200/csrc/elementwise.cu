@@ -39,7 +39,7 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 
 // y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 out.
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __half* __restrict__ y,
-                               int n, float eps) {
+                               int n, float eps, uint32_t* status) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
@@ -62,11 +62,13 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
       const int d4 = threadIdx.x + i * blockDim.x;
       if (d4 < nv) {
         const float4 g = reinterpret_cast<const float4*>(w)[d4];
-        __half2 lo = __floats2half2_rn(v[i].x * inv * g.x, v[i].y * inv * g.y);
-        __half2 hi = __floats2half2_rn(v[i].z * inv * g.z, v[i].w * inv * g.w);
+        // (a normalised value is at most sqrt(n) |w|; the saturating convert still guards a huge gain or a NaN-free
+        // overflow of x * inv)
+        const __half2 lo = __halves2half2(f16_sat(v[i].x * inv * g.x, status), f16_sat(v[i].y * inv * g.y, status));
+        const __half2 hi = __halves2half2(f16_sat(v[i].z * inv * g.z, status), f16_sat(v[i].w * inv * g.w, status));
         uint2 out;
-        out.x = *reinterpret_cast<uint32_t*>(&lo);
-        out.y = *reinterpret_cast<uint32_t*>(&hi);
+        out.x = *reinterpret_cast<const uint32_t*>(&lo);
+        out.y = *reinterpret_cast<const uint32_t*>(&hi);
         reinterpret_cast<uint2*>(yr)[d4] = out;
       }
     }
@@ -76,7 +78,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   for (int d = threadIdx.x; d < n; d += blockDim.x) { const float v = xr[d]; ss += v * v; }
   const float tot = block_sum(ss, red);
   const float inv = rsqrtf(tot / float(n) + eps);
-  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = __float2half_rn(xr[d] * inv * w[d]);
+  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = f16_sat(xr[d] * inv * w[d], status);
 }
 
 // Per (row, head): optional RMSNorm over dh, then rotate-half RoPE at position ctx_len + i.
@@ -167,7 +169,7 @@ __global__ void kv_inject_write_kernel(const float* __restrict__ kv, const float
   }
 }
 
-__global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F, uint32_t* status) {
   pdl_wait();
   pdl_trigger();
   const long long total = (long long)M * F;
@@ -175,7 +177,7 @@ __global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__
        idx += (long long)gridDim.x * blockDim.x) {
     const int m = int(idx / F), f = int(idx % F);
     const float gte = gu[size_t(m) * 2 * F + f], up = gu[size_t(m) * 2 * F + F + f];
-    h[idx] = __float2half_rn(silu_f(gte) * up);
+    h[idx] = f16_sat(silu_f(gte) * up, status);
   }
 }
 
@@ -186,23 +188,26 @@ __global__ void copy_f32_kernel(const float* __restrict__ src, float* __restrict
     dst[i] = src[i];
 }
 
-// inv_freq table per (theta, dh): theta^(-2j/dh) evaluated in double, rounded to fp32, kept on the device.
-struct RopeTable { float theta; int dh; float* dev; };
-RopeTable g_rope[8];
+// inv_freq table per (device, theta, dh): theta^(-2j/dh) evaluated in double, rounded to fp32, kept on that device.
+struct RopeTable { int device; float theta; int dh; float* dev; };
+constexpr int MAX_ROPE_TABLES = 64;
+RopeTable g_rope[MAX_ROPE_TABLES];
 int g_n_rope = 0;
 
-const float* rope_table(float theta, int dh, cudaStream_t stream) {
+const float* rope_table(float theta, int dh) {
+  const int device = current_device();
+  if (device < 0) return nullptr;
+  std::lock_guard<std::mutex> lock(device_setup_mutex());
   for (int i = 0; i < g_n_rope; ++i)
-    if (g_rope[i].theta == theta && g_rope[i].dh == dh) return g_rope[i].dev;
-  if (g_n_rope == 8) return nullptr;
+    if (g_rope[i].device == device && g_rope[i].theta == theta && g_rope[i].dh == dh) return g_rope[i].dev;
+  if (g_n_rope == MAX_ROPE_TABLES) return nullptr;
   float host[128];
   const int half = dh / 2;
   for (int j = 0; j < half; ++j) host[j] = float(pow(double(theta), -2.0 * double(j) / double(dh)));
   float* dev = nullptr;
   if (cudaMalloc(&dev, sizeof(float) * half) != cudaSuccess) return nullptr;
-  if (cudaMemcpy(dev, host, sizeof(float) * half, cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
-  (void)stream;
-  g_rope[g_n_rope++] = RopeTable{theta, dh, dev};
+  if (cudaMemcpy(dev, host, sizeof(float) * half, cudaMemcpyHostToDevice) != cudaSuccess) { cudaFree(dev); return nullptr; }
+  g_rope[g_n_rope++] = RopeTable{device, theta, dh, dev};
   return dev;
 }
 
@@ -219,9 +224,10 @@ cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token,
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream) {
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream,
+                           uint32_t* status) {
   const int threads = n >= 2048 ? 512 : 256;
-  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, (__half*)y_f16, n, eps);
+  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, (__half*)y_f16, n, eps, status);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -229,7 +235,7 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
                                 void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
                                 int qk_norm, cudaStream_t stream) {
   if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
-  const float* tab = rope_table(theta, dh, stream);
+  const float* tab = rope_table(theta, dh);
   if (!tab) return cudaErrorMemoryAllocation;
   const int n_pairs = B * k * (Hq + 2 * Hkv);
   cudaError_t e = launch_pdl(qk_norm_rope_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, qkv, qw, kw, tab, ctx_lens,
@@ -241,7 +247,7 @@ cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32
                                    const int32_t* page_table, int page_table_stride, void* k_pool, void* v_pool, int T,
                                    int Hkv, int dh, int page_size, float theta, float eps, int k_norm, cudaStream_t stream) {
   if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
-  const float* tab = rope_table(theta, dh, stream);
+  const float* tab = rope_table(theta, dh);
   if (!tab) return cudaErrorMemoryAllocation;
   const int n_pairs = T * 2 * Hkv;
   kv_inject_write_kernel<<<(n_pairs + 7) / 8, 256, 0, stream>>>(kv, kw, tab, req, pos, page_table, page_table_stride,
@@ -250,8 +256,9 @@ cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32
   return cudaGetLastError();
 }
 
-cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream) {
-  cudaError_t e = launch_pdl(swiglu_kernel, dim3(grid_for((long long)M * F, 256)), dim3(256), 0, stream, gu, (__half*)h_f16, M, F);
+cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream, uint32_t* status) {
+  cudaError_t e = launch_pdl(swiglu_kernel, dim3(grid_for((long long)M * F, 256)), dim3(256), 0, stream, gu, (__half*)h_f16, M, F,
+                             status);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -11,6 +11,12 @@
 //
 // Epilogues: fp32 / bf16 store, fp32 accumulate-into (residual), fp32 K-slice partial, and the
 // LM-head form that reduces each activation row's (max, index) over the CTA's 128 vocabulary rows.
+//
+// A CTA can also own TWO weight tiles (WT = 2, two accumulators in TMEM) so that one activation fill per k-step feeds
+// two MMAs: 1.5 bytes of shared-memory fill per weight byte instead of 2 at 128 activation rows.  Measured on the
+// state projection at 128 rows it changes nothing (5.55 TB/s either way: the profiler shows L2-to-SM traffic down
+// from 2.0x to 1.5x the weight bytes, DRAM at 73 % and the tensor pipe at 43 % - neither the fill nor a pipe is the
+// limit there), so it stays off unless HSPEC_GEMM_WT=2 asks for it.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -43,12 +49,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // 128-byte swizzle needs 1024-byte aligned tiles
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t b_stage_bytes = g.BN * TILE_K * 2;
-  const uint32_t stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  const uint32_t a_stage_bytes = uint32_t(g.WT) * A_STAGE_BYTES;
+  const uint32_t stage_bytes = a_stage_bytes + b_stage_bytes;
   GemmSmemTail* tail = reinterpret_cast<GemmSmemTail*>(smem + size_t(g.stages) * stage_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile_m = blockIdx.x;            // activation-row tile (fastest: CTAs sharing a weight tile run together)
-  const int tile_n = blockIdx.y;            // weight-row tile
+  const int tile_n = blockIdx.y;            // weight-row tile (WT consecutive 128-row tiles)
   const int split = blockIdx.z;
   const int kt_begin = split * g.k_tiles_per_split;
   const int kt_end = min(g.k_tiles_total, kt_begin + g.k_tiles_per_split);
@@ -93,8 +100,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t full = smem_u32(&tail->full[s]);
         mbar_expect_tx(full, stage_bytes);
         uint8_t* sa = smem + size_t(s) * stage_bytes;
-        tma_load_2d(smem_u32(sa), &tmA, (kt_begin + i) * TILE_K, tile_n * TILE_W, full, pol_w);
-        tma_load_2d(smem_u32(sa + A_STAGE_BYTES), &tmB, (kt_begin + i) * TILE_K, tile_m * g.BN, full, pol_x);
+        for (int w = 0; w < g.WT; ++w)       // (a tile wholly past the last weight row is zero-filled by the copy)
+          tma_load_2d(smem_u32(sa + w * A_STAGE_BYTES), &tmA, (kt_begin + i) * TILE_K, (tile_n * g.WT + w) * TILE_W, full, pol_w);
+        tma_load_2d(smem_u32(sa + a_stage_bytes), &tmB, (kt_begin + i) * TILE_K, tile_m * g.BN, full, pol_x);
       }
     }
   } else if (warp == 1) {
@@ -112,12 +120,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         tc_fence_after();
         const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes);
-        const uint64_t da = umma_desc_kmajor_sw128(sa);
-        const uint64_t db = umma_desc_kmajor_sw128(sa + A_STAGE_BYTES);
+        const uint64_t db = umma_desc_kmajor_sw128(sa + a_stage_bytes);
+        for (int w = 0; w < g.WT; ++w) {
+          const uint64_t da = umma_desc_kmajor_sw128(sa + w * A_STAGE_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < TILE_K / UMMA_K; ++kk) {
-          // advancing K inside the swizzle row: +32 bytes = +2 in the descriptor's 16-byte units
-          umma_bf16(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < TILE_K / UMMA_K; ++kk) {
+            // advancing K inside the swizzle row: +32 bytes = +2 in the descriptor's 16-byte units
+            umma_bf16(tmem_acc + uint32_t(w * g.BN), da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (i > 0 || kk > 0) ? 1u : 0u);
+          }
         }
         umma_commit(smem_u32(&tail->empty[s]));   // stage reusable once these MMAs have read it
       }
@@ -142,12 +152,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (!ok) atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
     tc_fence_after();
     if (*reinterpret_cast<volatile uint32_t*>(&tail->abort_flag)) ok = false;
-    const int n = tile_n * TILE_W + q * 32 + lane;  // output feature (weight row) of this thread
-    const bool n_ok = n < g.N_out;
     const int m0 = tile_m * g.BN;
+    for (int w = 0; w < g.WT; ++w) {                // (WT = 2 is never combined with the arg-max epilogue)
+    const int tile_w = tile_n * g.WT + w;           // 128-row weight tile of this pass
+    const int n = tile_w * TILE_W + q * 32 + lane;  // output feature (weight row) of this thread
+    const bool n_ok = n < g.N_out;
     for (int c0 = 0; c0 < g.BN && ok; c0 += 16) {
       uint32_t r[16];
-      tmem_ld16(tmem_acc + (uint32_t(q * 32) << 16) + uint32_t(c0), r);
+      tmem_ld16(tmem_acc + (uint32_t(q * 32) << 16) + uint32_t(w * g.BN + c0), r);
       tmem_ld_wait();
       if (g.mode == EPI_STORE_F32 || g.mode == EPI_PARTIAL_F32) {
         float* out = reinterpret_cast<float*>(g.out) + (g.mode == EPI_PARTIAL_F32 ? size_t(split) * g.M * g.ldo : 0);
@@ -178,14 +190,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
         }
       } else if (g.mode == EPI_SWIGLU_F16) {
-        const int f = tile_n * 64 + q * 16 + (lane & 15);
-        swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane);
+        const int f = tile_w * 64 + q * 16 + (lane & 15);
+        swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
       } else if (g.mode == EPI_STORE_F16) {
         __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
           const int m = m0 + c0 + j;
-          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2half_rn(__uint_as_float(r[j]));
+          if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = f16_sat(__uint_as_float(r[j]), g.status);
         }
       } else {  // EPI_ARGMAX: logits optional, (max, lowest index) over this warp's 32 vocabulary rows
         float add[16];
@@ -212,6 +224,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         warp_argmax16(v, vi, lane, row);
         if ((lane & 1) == 0) { tail->red_val[q][c0 + row] = v[0]; tail->red_idx[q][c0 + row] = vi[0]; }
       }
+    }
     }
     if (g.mode == EPI_ARGMAX) {
       asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
@@ -243,7 +256,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 // Sum the K-slice partials in slice order (deterministic) and apply the final store.
 __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits, int M, int N, void* out,
-                                     long long ldo, int mode) {
+                                     long long ldo, int mode, uint32_t* status) {
   pdl_wait();
   pdl_trigger();
   const long long total = (long long)M * N;
@@ -254,14 +267,14 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
     for (int s = 0; s < splits; ++s) acc += part[(size_t(s) * M + m) * N + n];
     if (mode == EPI_STORE_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] = acc;
     else if (mode == EPI_ACCUM_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] += acc;
-    else if (mode == EPI_STORE_F16) reinterpret_cast<__half*>(out)[size_t(m) * ldo + n] = __float2half_rn(acc);
+    else if (mode == EPI_STORE_F16) reinterpret_cast<__half*>(out)[size_t(m) * ldo + n] = f16_sat(acc, status);
     else if (mode == EPI_SWIGLU_F16) {
       // n runs over interleaved rows; lower half of each 32-row block = gate, upper half = up of the same 16 features
       if ((n & 31) < 16) {
         float up = 0.f;
         for (int s = 0; s < splits; ++s) up += part[(size_t(s) * M + m) * N + n + 16];
         const int f = (n >> 5) * 16 + (n & 15);
-        reinterpret_cast<__half*>(out)[size_t(m) * ldo + f] = __float2half_rn(silu_f(acc) * up);
+        reinterpret_cast<__half*>(out)[size_t(m) * ldo + f] = f16_sat(silu_f(acc) * up, status);
       }
     }
     else reinterpret_cast<__nv_bfloat16*>(out)[size_t(m) * ldo + n] = __float2bfloat16_rn(acc);
@@ -345,7 +358,8 @@ EncodeTiledFn get_encode() {
   return fn;
 }
 
-int g_smem_optin = -1;
+bool g_attr_done[MAX_DEVICES] = {};
+int g_smem_optin[MAX_DEVICES] = {};
 
 }  // namespace
 
@@ -401,14 +415,16 @@ size_t gemm_splitk_bytes(int M, int n_out, int splits) {
 // Launches y = x W^T.  tmW must describe W with box rows 128; x is described here (box rows BN).
 cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
   if (c.addend == nullptr && gemm2_preferred(c.M, c.n_out)) return gemm2_launch(c, stream, trk, err);
-  if (g_smem_optin < 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&g_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    cudaError_t e = cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         g_smem_optin);
+  {
+    // the opt-in shared-memory limit is a per-device function attribute
+    const cudaError_t e = once_per_device(g_attr_done, [](int dev) {
+      cudaError_t e2 = cudaDeviceGetAttribute(&g_smem_optin[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+      if (e2 != cudaSuccess) return e2;
+      return cudaFuncSetAttribute(gemm_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin[dev]);
+    });
     if (e != cudaSuccess) return e;
   }
+  const int smem_optin = g_smem_optin[current_device()];
   GemmArgs g{};
   g.M = c.M; g.N_out = c.n_out; g.K = c.K;
   g.BN = gemm_pick_bn(c.M);
@@ -417,14 +433,18 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   if (splits > g.k_tiles_total) splits = g.k_tiles_total;
   g.k_tiles_per_split = (g.k_tiles_total + splits - 1) / splits;
   splits = (g.k_tiles_total + g.k_tiles_per_split - 1) / g.k_tiles_per_split;   // no empty slice
+  // Two weight tiles per CTA: only on request (HSPEC_GEMM_WT=2, measurements), see the note at the top of the file.
+  static const int wt_env = [] { const char* e = getenv("HSPEC_GEMM_WT"); return e ? atoi(e) : 0; }();
+  const int n_tiles_w = (c.n_out + TILE_W - 1) / TILE_W;
+  g.WT = (wt_env == 2 && g.BN <= 128 && c.mode != EPI_ARGMAX && c.addend == nullptr) ? 2 : 1;
   uint32_t cols = 32;
-  while (cols < uint32_t(g.BN)) cols <<= 1;
+  while (cols < uint32_t(g.WT * g.BN)) cols <<= 1;
   g.tmem_cols = cols;
-  const size_t stage_bytes = A_STAGE_BYTES + size_t(g.BN) * TILE_K * 2;
+  const size_t stage_bytes = size_t(g.WT) * A_STAGE_BYTES + size_t(g.BN) * TILE_K * 2;
   const size_t fixed = sizeof(GemmSmemTail) + 1024;
   // Weight streaming (narrow activation tile): size the ring so that TWO CTAs fit on an SM; one CTA's prologue and
   // epilogue then overlap the other's stream.  Wide tiles take the whole SM.
-  const size_t budget = (g.BN <= 128) ? size_t(g_smem_optin) / 2 - 1024 : size_t(g_smem_optin);
+  const size_t budget = (g.BN <= 128) ? size_t(smem_optin) / 2 - 1024 : size_t(smem_optin);
   int stages = int((budget - fixed) / stage_bytes);
   if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
   if (stages > g.k_tiles_per_split) stages = g.k_tiles_per_split < 2 ? 2 : g.k_tiles_per_split;
@@ -447,20 +467,22 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   }
   CUtensorMap tmB;
   if (!make_tmap_16bit_2d(&tmB, c.x, c.M, c.K, c.ldx, g.BN, c.f16, err)) return cudaErrorInvalidValue;
-  dim3 grid((c.M + g.BN - 1) / g.BN, (c.n_out + TILE_W - 1) / TILE_W, splits);
+  dim3 grid((c.M + g.BN - 1) / g.BN, (n_tiles_w + g.WT - 1) / g.WT, splits);
   const size_t smem = size_t(stages) * stage_bytes + fixed;
-  trk_begin(trk, c.label ? c.label : "gemm", 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
+  trk_begin(trk, c.label ? c.label : "gemm", 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K,
+            gemm_io_bytes(c.M, c.n_out, c.K, c.mode, c.logits != nullptr));
   cudaError_t e = launch_pdl(gemm_tcgen05_kernel, grid, dim3(192), smem, stream, *c.tmW, tmB, g);
   trk_end(trk);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (splits > 1)
-    e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk);
+    e = splitk_reduce_launch(reinterpret_cast<const float*>(c.splitk_ws), splits, c.M, c.n_out, c.out, c.ldo, c.mode, stream, trk,
+                             c.status);
   return e;
 }
 
 cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, void* out, long long ldo, int mode,
-                                 cudaStream_t stream, Tracker* trk) {
+                                 cudaStream_t stream, Tracker* trk, uint32_t* status) {
   const long long total = (long long)M * N;
   trk_begin(trk, "splitk_reduce", 0, double(splits + 1) * M * N * 4);
   const bool f32 = mode == EPI_STORE_F32 || mode == EPI_ACCUM_F32;
@@ -475,7 +497,7 @@ cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, vo
   } else {
     int blocks = int((total + 255) / 256);
     if (blocks > 148 * 8) blocks = 148 * 8;
-    launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, part, splits, M, N, out, ldo, mode);
+    launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, part, splits, M, N, out, ldo, mode, status);
   }
   trk_end(trk);
   return cudaGetLastError();

@@ -276,13 +276,13 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           }
         } else if (mode == EPI_SWIGLU_F16) {
           const int f = tile_n128 * 64 + q * 16 + (lane & 15);
-          swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane);
+          swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
         } else if (mode == EPI_STORE_F16) {
           __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll
           for (int j = 0; j < 16; ++j) {
             const int m = m0 + c0 + j;
-            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2half_rn(__uint_as_float(r[j]));
+            if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = f16_sat(__uint_as_float(r[j]), g.status);
           }
         } else if (mode == EPI_STORE_BF16) {
           __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(g.out);
@@ -372,19 +372,20 @@ gemm2_tail_reduce_kernel(Gemm2Args g) {
       if (sp < g.tail_splits) acc += v[sp][j];
     if (g.mode == EPI_SWIGLU_F16) {
       const float up = __shfl_xor_sync(0xffffffffu, acc, 16);
-      if (lane < 16 && 2 * f < g.N_out) reinterpret_cast<__half*>(g.out)[size_t(m) * g.ldo + f] = __float2half_rn(silu_f(acc) * up);
+      if (lane < 16 && 2 * f < g.N_out) reinterpret_cast<__half*>(g.out)[size_t(m) * g.ldo + f] = f16_sat(silu_f(acc) * up, g.status);
       continue;
     }
     if (n >= g.N_out) continue;
     const size_t o = size_t(m) * g.ldo + n;
     if (g.mode == EPI_STORE_F32) reinterpret_cast<float*>(g.out)[o] = acc;
     else if (g.mode == EPI_ACCUM_F32) reinterpret_cast<float*>(g.out)[o] += acc;
-    else if (g.mode == EPI_STORE_F16) reinterpret_cast<__half*>(g.out)[o] = __float2half_rn(acc);
+    else if (g.mode == EPI_STORE_F16) reinterpret_cast<__half*>(g.out)[o] = f16_sat(acc, g.status);
     else reinterpret_cast<__nv_bfloat16*>(g.out)[o] = __float2bfloat16_rn(acc);
   }
 }
 
-int g_smem_optin2 = -1;
+bool g_attr_done2[MAX_DEVICES] = {};
+int g_smem_optin2[MAX_DEVICES] = {};
 
 }  // namespace
 
@@ -430,13 +431,15 @@ void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out
 size_t gemm2_tail_bytes() { return size_t(74) * 256 * 256 * 4; }
 
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err) {
-  if (g_smem_optin2 < 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&g_smem_optin2, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    cudaError_t e = cudaFuncSetAttribute(gemm_2sm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin2);
+  {
+    const cudaError_t e = once_per_device(g_attr_done2, [](int dev) {
+      cudaError_t e2 = cudaDeviceGetAttribute(&g_smem_optin2[dev], cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+      if (e2 != cudaSuccess) return e2;
+      return cudaFuncSetAttribute(gemm_2sm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, g_smem_optin2[dev]);
+    });
     if (e != cudaSuccess) return e;
   }
+  const int smem_optin2 = g_smem_optin2[current_device()];
   Gemm2Args g{};
   g.M = c.M; g.N_out = c.n_out; g.K = c.K;
   int splits = 1;
@@ -462,7 +465,7 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
   const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
   const size_t fixed = sizeof(Tail2) + 1024;
-  int stages = int((size_t(g_smem_optin2) - fixed) / stage_bytes);
+  int stages = int((size_t(smem_optin2) - fixed) / stage_bytes);
   if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
   if (stages < 2) { if (err) *err = "shared memory too small for the 2-SM GEMM pipeline"; return cudaErrorInvalidValue; }
   g.stages = stages;
@@ -474,7 +477,8 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   // profile name "gemm2:<what>" tells this kernel's launches from the one-CTA kernel's "gemm:<what>"
   std::string label = "gemm2:";
   if (c.label) { const char* colon = strchr(c.label, ':'); label += colon ? colon + 1 : c.label; }
-  trk_begin(trk, label.c_str(), 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K);
+  trk_begin(trk, label.c_str(), 2.0 * c.M * c.n_out * c.K, 2.0 * c.n_out * c.K,
+            gemm_io_bytes(c.M, c.n_out, c.K, c.mode, c.logits != nullptr));
   cudaError_t e = launch_pdl(gemm_2sm_kernel, dim3(2 * clusters), dim3(192), smem, stream, *c.tmW, tmB, g);
   trk_end(trk);
   if (e == cudaSuccess) e = cudaGetLastError();

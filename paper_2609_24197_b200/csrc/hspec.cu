@@ -137,14 +137,7 @@ const char* check_config(const hspec_config& c) {
   return nullptr;
 }
 
-uint32_t* g_status = nullptr;   // status word for the handle-less single-op entry points
-uint32_t* global_status() {
-  if (!g_status) {
-    if (cudaMalloc(&g_status, 256) != cudaSuccess) return nullptr;
-    cudaMemset(g_status, 0, 256);
-  }
-  return g_status;
-}
+uint32_t* g_status[MAX_DEVICES] = {};   // status blocks of the handle-less single-op entry points, one per device
 
 int fail(hspec_handle* h, int code, const std::string& msg);
 
@@ -154,7 +147,25 @@ namespace hspec {
 
 void set_last_error(const std::string& msg) { g_err = msg; }
 
-void Tracker::begin(const char* name, double flops, double bytes) {
+std::mutex& device_setup_mutex() {
+  static std::mutex m;
+  return m;
+}
+
+uint32_t* global_status() {
+  const int d = current_device();
+  if (d < 0) return nullptr;
+  std::lock_guard<std::mutex> lock(device_setup_mutex());
+  if (!g_status[d]) {
+    uint32_t* p = nullptr;
+    if (cudaMalloc(&p, STATUS_WORDS * 4) != cudaSuccess) return nullptr;
+    if (cudaMemset(p, 0, STATUS_WORDS * 4) != cudaSuccess) { cudaFree(p); return nullptr; }
+    g_status[d] = p;
+  }
+  return g_status[d];
+}
+
+void Tracker::begin(const char* name, double flops, double bytes, double io_bytes) {
   ++launches;
   if (!profiling) return;
   if (used == entries.size()) {
@@ -166,7 +177,7 @@ void Tracker::begin(const char* name, double flops, double bytes) {
   Entry& e = entries[used];
   memset(e.name, 0, sizeof(e.name));
   strncpy(e.name, name, sizeof(e.name) - 1);
-  e.flops = flops; e.bytes = bytes;
+  e.flops = flops; e.bytes = bytes; e.io_bytes = io_bytes;
   cudaEventRecord(e.a, stream);
 }
 
@@ -266,22 +277,24 @@ std::vector<std::string> required_names(const hspec_config& c) {
   return n;
 }
 
-__global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n) {
+__global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n,
+                                   uint32_t* status) {
   pdl_wait();
   pdl_trigger();
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < n; i += size_t(gridDim.x) * blockDim.x)
-    dst[i] = __float2half_rn(__bfloat162float(src[i]));
+    dst[i] = f16_sat(__bfloat162float(src[i]), status);
 }
 
 // w_gate_up [2F, K] bf16 (rows gate | up) -> fp16 with rows interleaved in blocks of 16:
 // dst rows [32j, 32j+16) = gate rows [16j, 16j+16), dst rows [32j+16, 32j+32) = up rows [16j, 16j+16).
-__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int F, int K) {
+__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int F, int K,
+                                          uint32_t* status) {
   const size_t total = size_t(2) * F * K;
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < total; i += size_t(gridDim.x) * blockDim.x) {
     const size_t r = i / K, c = i % K;
     const size_t blk = r >> 5, w = r & 31;
     const size_t src_row = (w < 16) ? blk * 16 + w : size_t(F) + blk * 16 + (w - 16);
-    dst[i] = __float2half_rn(__bfloat162float(src[src_row * K + c]));
+    dst[i] = f16_sat(__bfloat162float(src[src_row * K + c]), status);
   }
 }
 
@@ -297,12 +310,12 @@ __global__ void wait_selftest_kernel(uint32_t* status, unsigned long long limit_
 }
 
 __global__ void cvt_cols_f16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
-                                    __half* __restrict__ dst) {
+                                    __half* __restrict__ dst, uint32_t* status) {
   pdl_wait();
   pdl_trigger();
   const int total = M * ncols;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x)
-    dst[i] = __float2half_rn(src[size_t(i / ncols) * ld + col0 + i % ncols]);
+    dst[i] = f16_sat(src[size_t(i / ncols) * ld + col0 + i % ncols], status);
 }
 
 }  // namespace
@@ -347,8 +360,8 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
   if (cudaGetDeviceCount(&dev_count) != cudaSuccess || dev_count < 1)
     return fail(h, HSPEC_ERR_CUDA, "hspec_load_weights: no CUDA device; this library has no CPU path");
   if (!h->d_status) {
-    CUDA_TRY(h, cudaMalloc(&h->d_status, 256));
-    CUDA_TRY(h, cudaMemset(h->d_status, 0, 256));
+    CUDA_TRY(h, cudaMalloc(&h->d_status, STATUS_WORDS * 4));
+    CUDA_TRY(h, cudaMemset(h->d_status, 0, STATUS_WORDS * 4));
   }
   for (int i = 0; i < n; ++i) {
     if (!t[i].name || !t[i].data) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_load_weights: tensor without name or data");
@@ -372,10 +385,10 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
       const int blocks = int(std::min<size_t>((count + 255) / 256, 148 * 32));
       if (name.size() >= 13 && name.compare(name.size() - 13, 13, "mlp.w_gate_up") == 0 && h->cfg.F % 16 == 0)
         interleave_gate_up_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
-                                                   reinterpret_cast<__half*>(w.data), h->cfg.F, int(cols));
+                                                   reinterpret_cast<__half*>(w.data), h->cfg.F, int(cols), h->d_status);
       else
         bf16_to_f16_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
-                                            reinterpret_cast<__half*>(w.data), count);
+                                            reinterpret_cast<__half*>(w.data), count, h->d_status);
       CUDA_TRY(h, cudaGetLastError());
       if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, true, &errtxt)) {
         cudaFree(w.data);
@@ -405,12 +418,23 @@ int hspec_get_stats(hspec_handle* h, hspec_stats* out) {
   out->kernel_launches = h->trk.launches;
   out->launches_last_step = h->launches_last_step;
   out->device_status = 0;
+  out->attn_rescales = out->f16_range_events = out->bad_inputs = 0;
   if (h->d_status) {
     std::string errtxt;
+    uint32_t words[4] = {0, 0, 0, 0};
     CUDA_TRY(h, cudaStreamSynchronize(h->last_stream));
-    CUDA_TRY(h, cudaMemcpy(&out->device_status, h->d_status, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(h, cudaMemcpy(words, h->d_status, sizeof(words), cudaMemcpyDeviceToHost));
+    out->device_status = words[STATUS_WORD_CODE];
+    out->attn_rescales = words[STATUS_WORD_RESCALES];
+    out->f16_range_events = words[STATUS_WORD_F16_RANGE];
+    out->bad_inputs = words[STATUS_WORD_BAD_INPUT];
   }
-  return out->device_status ? HSPEC_ERR_TIMEOUT : HSPEC_OK;
+  if (out->device_status) return fail(h, HSPEC_ERR_TIMEOUT, "a bounded in-kernel wait gave up (device status word is set)");
+  if (out->bad_inputs)
+    return fail(h, HSPEC_ERR_PAGE_OUT_OF_RANGE, "a kernel met a context length or page id out of range (clamped / read as zeros)");
+  if (out->f16_range_events)
+    return fail(h, HSPEC_ERR_F16_RANGE, "finite values left the fp16 range and were clamped to +-65504");
+  return HSPEC_OK;
 }
 
 int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* out) {
@@ -499,7 +523,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     const size_t n_lh = size_t(B) * c.n_fuse * c.D;
     trk->begin("cvt_last_hidden", 0, double(n_lh) * 4);
     bf16_to_f16_kernel<<<int(std::min<size_t>((n_lh + 255) / 256, 148 * 8)), 256, 0, st>>>(
-        reinterpret_cast<const __nv_bfloat16*>(in->last_hidden), reinterpret_cast<__half*>(LH), n_lh);
+        reinterpret_cast<const __nv_bfloat16*>(in->last_hidden), reinterpret_cast<__half*>(LH), n_lh, h->d_status);
     trk->end();
     CUDA_TRY(h, cudaGetLastError());
   }
@@ -509,13 +533,13 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   for (int l = 0; l < c.L; ++l) {
     const std::string pre = "layers." + std::to_string(l) + ".";
     // ---- Mamba-2 mixer from the injected state
-    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
     CUDA_TRY(h, gemm(pre + "mamba.in_proj", "gemm:in_proj", U, M, EPI_STORE_F32, BIG, d.d_in_proj));
     const float* dt_raw = nullptr;
     if (c.dt_rank > 0) {
       trk->begin("cvt_dt_cols", 0, Md * c.dt_rank * 6);
       cvt_cols_f16_kernel<<<(M * c.dt_rank + 255) / 256, 256, 0, st>>>(BIG, d.d_in_proj, c.Di + d.d_xBC, c.dt_rank, M,
-                                                                     reinterpret_cast<__half*>(DTL));
+                                                                     reinterpret_cast<__half*>(DTL), h->d_status);
       trk->end();
       CUDA_TRY(h, cudaGetLastError());
       CUDA_TRY(h, gemm(pre + "mamba.dt_up", "gemm:dt_up", DTL, M, EPI_STORE_F32, DT, d.H));
@@ -528,11 +552,11 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     sc.y_gated = YG; sc.B = B; sc.k = k; sc.Di = c.Di; sc.P = c.P; sc.N = c.N; sc.G = c.G; sc.d_conv = c.d_conv;
     sc.ws = ws + p.SCAN; sc.ws_bytes = p.scan_bytes;
     CUDA_TRY(h, scan_launch(sc, st, trk, &errtxt));
-    EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st));
+    EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st, h->d_status));
     CUDA_TRY(h, gemm(pre + "mamba.out_proj", "gemm:out_proj", U, M, EPI_ACCUM_F32, X, c.D));
     // ---- attention over the target's KV (in place) + the block
     if (c.has_attn[l]) {
-      EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st));
+      EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
       CUDA_TRY(h, gemm(pre + "attn.wqkv", "gemm:wqkv", U, M, EPI_STORE_F32, BIG, d.d_qkv));
       EW("qk_norm_rope", Md * d.d_qkv * 6,
          qk_norm_rope_launch(BIG, fptr(pre + "attn.q_norm"), fptr(pre + "attn.k_norm"), in->ctx_lens, Q, KB, VB, B, k, c.Hq,
@@ -549,20 +573,20 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
       CUDA_TRY(h, gemm(pre + "attn.wo", "gemm:wo", U, M, EPI_ACCUM_F32, X, c.D));
     }
     // ---- SwiGLU MLP
-    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
     if (c.F % 16 == 0) {
       // gate/up rows were interleaved at load: the GEMM epilogue applies SiLU(gate) * up and writes h directly.
       // U is both the GEMM's input (D columns) and h's home (F columns), so h goes to a second fp16 buffer.
       CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_SWIGLU_F16, U2, c.F));
     } else {
       CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
-      EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U2, M, c.F, st));
+      EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U2, M, c.F, st, h->d_status));
     }
     CUDA_TRY(h, gemm(pre + "mlp.w_down", "gemm:down", U2, M, EPI_ACCUM_F32, X, c.D));
   }
   if (out->hidden) EW("copy_hidden", Md * c.D * 8, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st));
   // ---- final norm, LM head fused with the per-row arg-max
-  EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st));
+  EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st, h->d_status));
   const int* id_map = c.V_draft > 0 ? reinterpret_cast<const int*>(W("vocab_map").data) : nullptr;
   if (c.markov_rank > 0) {
     // ---- LM head to fp32 logits, then the causal correction position by position (Sec. 3.3.3)
@@ -596,8 +620,8 @@ int hspec_debug_wait_selftest(hspec_handle* h, int32_t limit_ms, void* stream) {
   if (!h || limit_ms < 1 || limit_ms > 2000) return fail(h, HSPEC_ERR_INVALID_ARG, "hspec_debug_wait_selftest: bad argument");
   std::string errtxt;
   if (!h->d_status) {
-    CUDA_TRY(h, cudaMalloc(&h->d_status, 256));
-    CUDA_TRY(h, cudaMemset(h->d_status, 0, 256));
+    CUDA_TRY(h, cudaMalloc(&h->d_status, STATUS_WORDS * 4));
+    CUDA_TRY(h, cudaMemset(h->d_status, 0, STATUS_WORDS * 4));
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   h->last_stream = st;
@@ -611,7 +635,7 @@ int hspec_clear_status(hspec_handle* h) {
   std::string errtxt;
   if (h->d_status) {
     CUDA_TRY(h, cudaStreamSynchronize(h->last_stream));
-    CUDA_TRY(h, cudaMemset(h->d_status, 0, 256));
+    CUDA_TRY(h, cudaMemset(h->d_status, 0, STATUS_WORDS * 4));
   }
   return HSPEC_OK;
 }
@@ -634,7 +658,7 @@ int hspec_get_profile(hspec_handle* h, hspec_prof_entry* out, int32_t max_entrie
     CUDA_TRY(h, cudaEventElapsedTime(&ms, e.a, e.b));
     memset(out[n].name, 0, sizeof(out[n].name));
     strncpy(out[n].name, e.name, sizeof(out[n].name) - 1);
-    out[n].ms = ms; out[n].flops = e.flops; out[n].bytes = e.bytes;
+    out[n].ms = ms; out[n].flops = e.flops; out[n].bytes = e.bytes; out[n].io_bytes = e.io_bytes;
   }
   return n;
 }
@@ -723,6 +747,32 @@ int hspec_op_kv_inject_write(const float* kv, const float* k_norm_w, const int32
   return HSPEC_OK;
 }
 
+int hspec_op_device_status(uint32_t* words4, int32_t clear) {
+  std::string errtxt;
+  uint32_t total[4] = {0, 0, 0, 0};
+  OP_TRY(cudaDeviceSynchronize());
+  uint32_t* blocks[2] = {nullptr, noalloc_status_if_resolved()};
+  {
+    const int d = current_device();
+    if (d < 0) return fail(nullptr, HSPEC_ERR_CUDA, "hspec_op_device_status: no current CUDA device");
+    std::lock_guard<std::mutex> lock(device_setup_mutex());
+    blocks[0] = g_status[d];
+  }
+  for (uint32_t* blk : blocks) {
+    if (!blk) continue;
+    uint32_t w[4];
+    OP_TRY(cudaMemcpy(w, blk, sizeof(w), cudaMemcpyDeviceToHost));
+    if (total[0] == 0) total[0] = w[0];
+    for (int i = 1; i < 4; ++i) total[i] += w[i];
+    if (clear) OP_TRY(cudaMemset(blk, 0, STATUS_WORDS * 4));
+  }
+  if (words4) memcpy(words4, total, sizeof(total));
+  if (total[STATUS_WORD_CODE]) return fail(nullptr, HSPEC_ERR_TIMEOUT, "a bounded in-kernel wait gave up (device status word is set)");
+  if (total[STATUS_WORD_BAD_INPUT]) return fail(nullptr, HSPEC_ERR_PAGE_OUT_OF_RANGE, "a kernel met a context length or page id out of range");
+  if (total[STATUS_WORD_F16_RANGE]) return fail(nullptr, HSPEC_ERR_F16_RANGE, "finite values left the fp16 range and were clamped");
+  return HSPEC_OK;
+}
+
 size_t hspec_markov_workspace_bytes(int32_t B, int32_t Vd, int32_t r) {
   if (B < 1 || Vd < 1 || r < 1) return 0;
   return markov_workspace_bytes(B, Vd, r);
@@ -753,7 +803,7 @@ int hspec_op_markov_head(float* logits, int64_t ld, const void* W_in, const void
 int hspec_op_rmsnorm(const float* x, const float* w, void* y, int32_t M, int32_t n, float eps, void* stream) {
   if (!x || !w || !y || M < 1 || n < 1) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_rmsnorm: bad argument");
   std::string errtxt;
-  OP_TRY(rmsnorm_launch(x, w, y, M, n, eps, reinterpret_cast<cudaStream_t>(stream)));
+  OP_TRY(rmsnorm_launch(x, w, y, M, n, eps, reinterpret_cast<cudaStream_t>(stream), global_status()));
   return HSPEC_OK;
 }
 
@@ -832,7 +882,7 @@ int hspec_debug_gather_kv(const void* pool, const int32_t* page_table_row, int32
 int hspec_op_swiglu(const float* gu, void* h_f16, int32_t M, int32_t F, void* stream) {
   if (!gu || !h_f16 || M < 1 || F < 1) return fail(nullptr, HSPEC_ERR_INVALID_ARG, "hspec_op_swiglu: bad argument");
   std::string errtxt;
-  OP_TRY(swiglu_launch(gu, h_f16, M, F, reinterpret_cast<cudaStream_t>(stream)));
+  OP_TRY(swiglu_launch(gu, h_f16, M, F, reinterpret_cast<cudaStream_t>(stream), global_status()));
   return HSPEC_OK;
 }
 

@@ -5,6 +5,7 @@
 #include <stdint.h>
 
 #include <cstdlib>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -15,13 +16,39 @@ constexpr int GEMM_MAX_STAGES = 8;
 // Records the message hspec_last_error(NULL) returns (calling thread).
 void set_last_error(const std::string& msg);
 
+// State that CUDA keeps per device (function attributes, small device-side tables, the status block of the
+// handle-less entry points) is cached per device index, so one process may drive several GPUs.
+constexpr int MAX_DEVICES = 64;
+std::mutex& device_setup_mutex();
+inline int current_device() {
+  int d = -1;
+  return (cudaGetDevice(&d) == cudaSuccess && d >= 0 && d < MAX_DEVICES) ? d : -1;
+}
+// Runs `fn` (returning cudaError_t) once per device, for the current device; a failure is returned and retried on the
+// next call.
+template <class F>
+inline cudaError_t once_per_device(bool (&done)[MAX_DEVICES], F fn) {
+  const int d = current_device();
+  if (d < 0) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(device_setup_mutex());
+  if (done[d]) return cudaSuccess;
+  const cudaError_t e = fn(d);
+  if (e == cudaSuccess) done[d] = true;
+  return e;
+}
+// Status block (STATUS_WORDS x uint32, zeroed) of the current device for entry points that take no handle.
+uint32_t* global_status();
+// Status block inside the allocation-free entry point's built-in array, once a call on the current device has
+// resolved its address (else null).
+uint32_t* noalloc_status_if_resolved();
+
 // Counts kernel launches and, when profiling is on, brackets each launch with a pair of CUDA events
 // recorded on the launching stream (read back with elapsed() after the stream is synchronised).
 struct Tracker {
   struct Entry {
     char name[40];
     cudaEvent_t a = nullptr, b = nullptr;
-    double flops = 0, bytes = 0;
+    double flops = 0, bytes = 0, io_bytes = 0;
   };
   uint64_t launches = 0;
   bool profiling = false;
@@ -29,11 +56,26 @@ struct Tracker {
   std::vector<Entry> entries;
   size_t used = 0;
   void begin_step(cudaStream_t st) { used = 0; stream = st; }
-  void begin(const char* name, double flops = 0, double bytes = 0);   // call right before a launch
+  void begin(const char* name, double flops = 0, double bytes = 0, double io_bytes = 0);   // call right before a launch
   void end();                                                         // call right after it
   void destroy();
 };
-inline void trk_begin(Tracker* t, const char* name, double flops = 0, double bytes = 0) { if (t) t->begin(name, flops, bytes); }
+inline void trk_begin(Tracker* t, const char* name, double flops = 0, double bytes = 0, double io_bytes = 0) {
+  if (t) t->begin(name, flops, bytes, io_bytes);
+}
+// Activation bytes a GEMM launch reads and writes besides its weights: x [M, K] 16-bit in, y [M, n_out] out (a
+// residual epilogue reads y as well; the LM-head arg-max epilogue writes logits only when asked).
+inline double gemm_io_bytes(int M, int n_out, int K, int mode, bool logits) {
+  double out = 0;
+  switch (mode) {
+    case 0: case 3: out = 4.0 * M * n_out; break;            // fp32 store / K-slice partial
+    case 1: case 5: out = 2.0 * M * n_out; break;            // bf16 / fp16 store
+    case 2: out = 8.0 * M * n_out; break;                    // fp32 read-modify-write
+    case 6: out = 1.0 * M * n_out; break;                    // SwiGLU: fp16 [M, n_out / 2]
+    default: out = logits ? 4.0 * M * n_out : 0; break;      // arg-max
+  }
+  return 2.0 * M * K + out;
+}
 inline void trk_end(Tracker* t) { if (t) t->end(); }
 
 // Launch with programmatic stream serialisation: the kernel MUST call pdl_wait() before it touches global data.
@@ -62,6 +104,7 @@ enum GemmEpilogue : int {
 struct GemmArgs {       // kernel argument block
   int M, N_out, K;
   int BN;               // activation rows per CTA = UMMA N (multiple of 16, <= 256)
+  int WT;               // 128-row weight tiles per CTA (1 or 2): with 2, one activation tile fill feeds two MMAs
   int k_tiles_total, k_tiles_per_split;
   int stages;
   uint32_t tmem_cols;
@@ -110,7 +153,7 @@ bool gemm2_preferred(int M, int n_out);        // many rows and at least one ful
 size_t gemm2_tail_bytes();                     // scratch the 2-SM kernel's K-sliced tail wave may use
 void gemm2_pick(int M, int n_out, int K, int mode, int* bnt, int* splits);   // tile width and K-slices of the 2-SM kernel
 cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, void* out, long long ldo, int mode,
-                                 cudaStream_t stream, Tracker* trk);
+                                 cudaStream_t stream, Tracker* trk, uint32_t* status);
 cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, std::string* err);
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk, const int* id_map = nullptr);
@@ -178,11 +221,12 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
 // ---- element-wise kernels (elementwise.cu)
 cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
                               int D, cudaStream_t stream);
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream);
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream,
+                           uint32_t* status);
 cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
                                 void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
                                 int qk_norm, cudaStream_t stream);
-cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream);
+cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream, uint32_t* status);
 cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream);
 
 }  // namespace hspec

@@ -56,6 +56,19 @@ int scratch_for_current_device(NoAllocScratch** out, std::string* why) {
   return HSPEC_OK;
 }
 
+}  // namespace
+
+namespace hspec {
+uint32_t* noalloc_status_if_resolved() {
+  const int dev = current_device();
+  if (dev < 0 || dev >= NA_MAX_DEVICES) return nullptr;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  return g_scratch_ptr[dev] ? reinterpret_cast<NoAllocScratch*>(g_scratch_ptr[dev])->status : nullptr;
+}
+}  // namespace hspec
+
+namespace {
+
 int na_fail(int code, const std::string& msg) {
   hspec::set_last_error("hspec_op_lm_head_argmax_noalloc: " + msg);
   return code;

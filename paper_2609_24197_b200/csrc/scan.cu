@@ -568,13 +568,13 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
     launch_pdl(scan_cb_kernel, dim3(c.G, c.B), dim3(256), 0, stream, a, xact, (float*)cbw);
     trk_end(trk);
     const size_t smem_s = two ? scan_stream_smem<2>() : scan_stream_smem<1>();
-    static bool sset1 = false, sset2 = false;
-    bool& was = two ? sset2 : sset1;
-    if (!was) {
-      cudaError_t e = two ? cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s))
-                          : cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s));
+    static bool sset[2][MAX_DEVICES] = {};
+    {
+      const cudaError_t e = once_per_device(sset[two ? 1 : 0], [two, smem_s](int) {
+        return two ? cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s))
+                   : cudaFuncSetAttribute(mamba_scan_stream_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_s));
+      });
       if (e != cudaSuccess) return e;
-      was = true;
     }
     dim3 grid_s(a.H / 4, c.B);
     trk_begin(trk, "mamba_scan", 2.0 * c.B * c.k * a.H * c.P * c.N, double(c.B) * a.H * c.P * c.N * 2);
@@ -586,13 +586,13 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
   if (c.P == 64 && c.N == 128 && (a.H / c.G) % 4 == 0 && c.ld_in % 2 == 0 && c.Di % 2 == 0) {
     const bool two = c.k > 16;
     const size_t smem_f = two ? scan_mma_smem<2>() : scan_mma_smem<1>();
-    static bool set1 = false, set2 = false;
-    bool& was_set = two ? set2 : set1;
-    if (!was_set) {
-      cudaError_t e = two ? cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f))
-                          : cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f));
+    static bool fset[2][MAX_DEVICES] = {};
+    {
+      const cudaError_t e = once_per_device(fset[two ? 1 : 0], [two, smem_f](int) {
+        return two ? cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f))
+                   : cudaFuncSetAttribute(mamba_scan_mma_kernel<64, 128, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem_f));
+      });
       if (e != cudaSuccess) return e;
-      was_set = true;
     }
     dim3 grid_f(a.H / 4, c.B);
     trk_begin(trk, "mamba_scan", 2.0 * c.B * c.k * a.H * c.P * c.N, double(c.B) * a.H * c.P * c.N * 2);
@@ -603,11 +603,17 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
   }
   const size_t smem = sizeof(float) * (size_t(KMAX) * c.P + 2 * size_t(KMAX) * c.N + KMAX * KMAX + 3 * KMAX +
                                        size_t(c.P) * a.NP);
-  static size_t smem_set = 0;
-  if (smem > 48 * 1024 && smem > smem_set) {
-    cudaError_t e = cudaFuncSetAttribute(mamba_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-    if (e != cudaSuccess) { if (err) *err = "scan: state tile does not fit in shared memory"; return e; }
-    smem_set = smem;
+  if (smem > 48 * 1024) {
+    // the largest size asked for so far, per device (the attribute is a per-device property of the function)
+    static size_t smem_set[MAX_DEVICES] = {};
+    const int dev = current_device();
+    if (dev < 0) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(device_setup_mutex());
+    if (smem > smem_set[dev]) {
+      cudaError_t e = cudaFuncSetAttribute(mamba_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+      if (e != cudaSuccess) { if (err) *err = "scan: state tile does not fit in shared memory"; return e; }
+      smem_set[dev] = smem;
+    }
   }
   dim3 grid(a.H, c.B);
   trk_begin(trk, "mamba_scan", 0, double(c.B) * a.H * c.P * c.N * 2);

@@ -37,7 +37,6 @@ _MODEL_PAPER_8B = dict(
 )
 
 CONFIGS = {
-    # index i = BASELINE config i+1
     "tiny": dict(_MODEL_TINY, name="tiny", B=1, k=8, ctx=("const", 256, 256)),
     "latency_8b": dict(_MODEL_8B, name="latency_8b", B=1, k=16, ctx=("const", 2048, 2048)),
     "serving_8b": dict(_MODEL_8B, name="serving_8b", B=32, k=16, ctx=("uniform", 512, 8192)),

@@ -202,7 +202,38 @@ def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state, with_scratch):
 
 
 # ------------------------------------------------------------------------------ attention
-def _attn_case(hs, B, k, Hq, Hkv, dh, ctxs, window, chunk, seed=0, poison=True):
+def _peak_the_scores(batch, ctxs, q, kb, k, Hq, Hkv, dh, ramp=12.0, targets=(25.0, 45.0, 70.0, 110.0)):
+    """Makes the score rows peaked the way a real target cache is (attention sinks, a few dominant keys), in place:
+    the stored keys of every request grow by a factor rising from 1 at position 0 to `ramp` at the end of the context,
+    so every row's running maximum keeps climbing from tile to tile and from chunk to chunk; and a few keys late in
+    the context, and a few of the block's own keys, are set to a multiple of one query row chosen so that this row's
+    scaled score q.k/sqrt(dh) reaches `targets` (natural-log units: 70 is 101 in the kernel's base-2 units, 110 is
+    159, which no fp32 weight 2^(s - m) could hold relative to the first tiles' maximum without moving the reference)."""
+    kp = batch["k_pools"][0]
+    pt = batch["page_table"].cpu()
+    rep = Hq // Hkv
+    g = torch.Generator().manual_seed(99)
+    for b, ctx in enumerate(ctxs):
+        if ctx > 0:
+            pos = torch.arange(ctx)
+            pages = pt[b, pos // 16].long().cuda()
+            slots = (pos % 16).cuda()
+            factor = (1.0 + (ramp - 1.0) * pos.float() / max(ctx - 1, 1)).cuda()
+            kp[pages, slots] = (kp[pages, slots].float() * factor[:, None, None]).to(torch.bfloat16)
+        for n, tgt in enumerate(targets):
+            i = int(torch.randint(0, k, (1,), generator=g))
+            hq = int(torch.randint(0, Hq, (1,), generator=g))
+            qv = q[b * k + i, hq].float()
+            key = (qv * (tgt * dh ** 0.5 / float(qv @ qv))).to(torch.bfloat16)
+            if n % 2 == 0 and ctx > 0:                  # a stored key in the last quarter of the context
+                p = int(torch.randint(ctx - max(1, ctx // 4), ctx, (1,), generator=g))
+                kp[int(pt[b, p // 16]), p % 16, hq // rep] = key
+            else:                                       # one of the block's own keys, visible to row i (j <= i)
+                j = int(torch.randint(0, i + 1, (1,), generator=g))
+                kb[b * k + j, hq // rep] = key
+
+
+def _attn_case(hs, B, k, Hq, Hkv, dh, ctxs, window, chunk, seed=0, poison=True, peaked=False):
     cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
     batch = synth.make_request_batch(cfg, ctx_lens=ctxs, device="cuda", poison_tail=poison, extra_pages=3,
                                      seed_offset=seed)
@@ -210,6 +241,8 @@ def _attn_case(hs, B, k, Hq, Hkv, dh, ctxs, window, chunk, seed=0, poison=True):
     q = _randn((M, Hq, dh), 41 + seed, 1.0, torch.bfloat16)
     kb = _randn((M, Hkv, dh), 42 + seed, 1.0, torch.bfloat16)
     vb = _randn((M, Hkv, dh), 43 + seed, 1.0, torch.bfloat16)
+    if peaked:
+        _peak_the_scores(batch, ctxs, q, kb, k, Hq, Hkv, dh)
     o = torch.full((M, Hq * dh), float("nan"), dtype=torch.float16, device="cuda")
     max_ctx = max(ctxs + [1])
     ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, max_ctx, window, chunk), dtype=torch.uint8,
@@ -251,6 +284,58 @@ def test_attention_many_short_requests_fill_the_work_list(hs):
     ctxs[7], ctxs[123], ctxs[299] = 0, 3000, 1537
     _attn_case(hs, 300, 4, 8, 4, 128, ctxs, 0, 256, seed=4, poison=False)
     _attn_case(hs, 300, 4, 8, 4, 128, ctxs, 100, 128, seed=5, poison=False)
+
+
+@pytest.mark.parametrize("k,Hq,Hkv,dh", [(16, 16, 2, 128), (16, 32, 8, 128), (32, 8, 1, 128), (8, 4, 2, 64)])
+@pytest.mark.parametrize("window,chunk", [(0, 0), (0, 512), (2048, 0)])
+def test_attention_peaked_scores_move_the_reference_maximum(hs, k, Hq, Hkv, dh, window, chunk):
+    """Row maxima that grow by far more than 2^8 between key tiles and between chunks (R = 128, 64 and 256 query rows
+    per KV head on the tensor-core path, plus the dh = 64 path).  On the tensor-core path the reference maximum is
+    lazy: it moves, and the accumulator row is rescaled in tensor memory, only when a tile's row maximum outgrows it by
+    2^8 - with N(0,1) keys that never happens, with these inputs it must, and the kernel counts the events."""
+    hs.hspec_op_device_status(clear=True)
+    _attn_case(hs, 3, k, Hq, Hkv, dh, [700, 4099, 9000], window, chunk, seed=6, peaked=True)
+    st = hs.hspec_op_device_status(clear=True)
+    assert st["device_status"] == 0 and st["bad_inputs"] == 0 and st["f16_range_events"] == 0
+    if dh == 128:
+        assert st["attn_rescales"] > 0, "the rescale branch of the tensor-core kernel did not run"
+
+
+def test_attention_bad_page_id_and_context_length_are_caught_not_followed(hs):
+    """A stale page-table entry (id past the pool, or negative) and a context length beyond the host's bound must not
+    turn into an address: the kernels read such a page as zeros, clamp the length, count the event, and the status call
+    reports HSPEC_ERR_PAGE_OUT_OF_RANGE.  Nothing faults; the next call on clean inputs is correct again."""
+    B, k, Hq, Hkv = 3, 4, 8, 2
+    for dh in (128, 64):
+        cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16)
+        ctxs = [300, 77, 520]
+        batch = synth.make_request_batch(cfg, ctx_lens=ctxs, device="cuda", extra_pages=2)
+        q = _randn((B * k, Hq, dh), 61, 1.0, torch.bfloat16)
+        kb, vb = _randn((B * k, Hkv, dh), 62, 1.0, torch.bfloat16), _randn((B * k, Hkv, dh), 63, 1.0, torch.bfloat16)
+        ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, 520, 0, 0), dtype=torch.uint8, device="cuda")
+        o = torch.empty((B * k, Hq * dh), dtype=torch.float16, device="cuda")
+
+        def run(pt, cl):
+            hs.hspec_op_attention(q, kb, vb, batch["k_pools"][0], batch["v_pools"][0], pt, cl, 520, o, B, k, Hq, Hkv, dh,
+                                  16, 0, 0, ws)
+            return hs.hspec_op_device_status(clear=True)
+        hs.hspec_op_device_status(clear=True)
+        assert run(batch["page_table"], batch["ctx_lens"])["rc"] == 0
+        good = o.clone()
+        pt = batch["page_table"].clone()
+        pt[0, 3] = batch["num_pages"] + 5            # a full page of a full tile (fetched by TMA on the tcgen05 path)
+        pt[1, 4] = -7                                # the ragged last page of request 1 (fetched by plain loads)
+        st = run(pt, batch["ctx_lens"])
+        assert st["rc"] == -5 and st["bad_inputs"] >= 2 and st["device_status"] == 0
+        assert torch.isfinite(o.float()).all()
+        assert torch.equal(o[2 * k:], good[2 * k:])               # request 2 has clean pages: untouched by the others
+        cl = batch["ctx_lens"].clone()
+        cl[2] = 100000                               # far beyond max_ctx = 520 and beyond the page-table row
+        st = run(batch["page_table"], cl)
+        assert st["rc"] == -5 and st["bad_inputs"] >= 1
+        assert torch.equal(o[:2 * k], good[:2 * k])
+        assert run(batch["page_table"], batch["ctx_lens"])["rc"] == 0
+        assert torch.equal(o, good)
 
 
 def test_attention_page_permutation_is_bit_exact(hs):

@@ -97,14 +97,21 @@ def test_request_independence_across_batch_sizes():
 
 
 def _full_size(name, n_check, **over):
+    """The workload at its full size, in the launch configuration bench.py times, compared with the oracle on `n_check`
+    sampled requests (requests are independent, so each is a complete comparison): the longest, the shortest and the
+    median context, then seeded random ones.  The shortest is a request whose visible context is a single chunk
+    (finished inside the attention kernel, no partials), the longest has the most chunks."""
     cfg = synth.get_config(name, **over)
     drafter, w, batch = cuda_setup(cfg, poison_tail=False, extra_pages=0)
     B = cfg["B"]
-    # longest, shortest and (if asked) a seeded random request
     order = np.argsort(batch["ctx_lens_host"])
-    pick = sorted(set([int(order[-1]), int(order[0])][:n_check]))
-    r = check_step(cfg, drafter, w, batch, cfg["k"], requests=pick, dtype=np.float32, what=name)
-    print(name, "requests", pick, r)
+    pick = [int(order[-1]), int(order[0]), int(order[B // 2])]
+    rnd = np.random.default_rng(synth.BASE_SEED + 17).permutation(B).tolist()
+    pick = list(dict.fromkeys(pick + [int(b) for b in rnd]))[:max(1, min(n_check, B))]
+    r = check_step(cfg, drafter, w, batch, cfg["k"], requests=sorted(pick), dtype=np.float32, what=name)
+    st = drafter.stats()
+    assert st["rc"] == 0, st
+    print(name, "requests", sorted(pick), "contexts", [batch["ctx_lens_host"][b] for b in sorted(pick)], r)
     drafter.close()
     del w, batch
     torch.cuda.empty_cache()
@@ -116,21 +123,32 @@ def test_latency_8b_full_size():
 
 
 def test_serving_8b_full_size_sampled_requests():
-    _full_size("serving_8b", 2)
+    _full_size("serving_8b", 8)
 
 
-def test_conc128_32b_full_size_sampled_request():
-    _full_size("conc128_32b", 1)
+def test_conc128_32b_full_size_sampled_requests():
+    _full_size("conc128_32b", 8)
+
+
+def test_serving_8b_and_conc128_32b_with_the_2048_token_window():
+    # the paper's sliding window (App. B.1) on the two serving workloads: the variant bench.py reports beside the
+    # full-context headline
+    _full_size("serving_8b", 2, window=2048)
+    _full_size("conc128_32b", 2, window=2048)
 
 
 def test_paper_shape_drafter_sampled_requests():
     # the paper's own drafter shape (App. B.1): 48 Mamba heads x 64 with state = groups = conv = 4, five fused target
     # layers, three attention layers + one Mamba-MLP layer, 2048-token window
-    _full_size("paper_8b", 2)
+    _full_size("paper_8b", 3)
 
 
-def test_sweep_cell_8b_B128_k8_sampled_request():
-    _full_size("sweep_8b_B128_k8", 1)
+def test_sweep_cells_8b_sampled_requests():
+    # cells of the concurrency x block-size sweep: 64 query rows per KV head at k = 16, 32 at k = 8, and at k = 32 the
+    # only shape that runs two 128-row tiles per KV head at full size
+    _full_size("sweep_8b_B128_k8", 2)
+    _full_size("sweep_8b_B256_k16", 8)
+    _full_size("sweep_8b_B128_k32", 5)
 
 
 def test_mid_config_pruned_drafter_vocabulary():
@@ -164,8 +182,8 @@ def test_mid_config_markov_head(over):
     drafter.close()
 
 
-def test_conc128_32b_markov_full_size_sampled_request():
-    _full_size("conc128_32b_markov", 1)
+def test_conc128_32b_markov_full_size_sampled_requests():
+    _full_size("conc128_32b_markov", 2)
 
 
 def test_bounded_wait_gives_up_and_reports_without_killing_the_context():
