@@ -577,7 +577,7 @@ def _randn(shape, seed, std, dtype):
     return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std).to(dtype)
 
 
-def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16):
+def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16, window=0):
     """One attention layer of the serving shapes: dh = 128, contexts uniform in [lo, hi]."""
     import paper_2609_24197_b200 as hs
     dh = 128
@@ -588,17 +588,17 @@ def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16):
     q, kb, vb = (_randn((M, h, dh), s, 1.0, torch.bfloat16) for h, s in ((Hq, 1), (Hkv, 2), (Hkv, 3)))
     o = torch.empty((M, Hq * dh), dtype=torch.float16, device="cuda")
     mc = max(ctx)
-    ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, mc, 0, 0), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(hs.hspec_attention_workspace_bytes(B, k, Hq, Hkv, dh, mc, window, 0), dtype=torch.uint8, device="cuda")
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
     ev[0].record()
     for i in range(reps):
         hs.hspec_op_attention(q, kb, vb, batch["k_pools"][0], batch["v_pools"][0], batch["page_table"],
-                              batch["ctx_lens"], mc, o, B, k, Hq, Hkv, dh, 16, 0, 0, ws)
+                              batch["ctx_lens"], mc, o, B, k, Hq, Hkv, dh, 16, window, 0, ws)
         ev[i + 1].record()
     torch.cuda.synchronize()
-    kv_bytes = sum(ctx) * Hkv * dh * 2 * 2
+    kv_bytes = sum(min(c, window - 1) if window > 0 else c for c in ctx) * Hkv * dh * 2 * 2
     us = [ev[i].elapsed_time(ev[i + 1]) * 1e3 for i in range(reps)]
-    print(f"attention: B={B} k={k} Hq={Hq} Hkv={Hkv} sum ctx={sum(ctx)} target-KV bytes per launch={kv_bytes} "
+    print(f"attention: B={B} k={k} Hq={Hq} Hkv={Hkv} window={window} sum ctx={sum(ctx)} target-KV bytes per launch={kv_bytes} "
           f"us per call={[round(u, 1) for u in us]} -> {kv_bytes / (min(us) * 1e-6) / 1e12:.2f} TB/s")
 
 
@@ -640,6 +640,7 @@ CASES = {
     # name: (function, keyword arguments) - each runs ONE kernel family a few times on inputs larger than L2
     "attention": (case_attention, {}),                                             # 8B-class, 64 query rows per KV head
     "attention32b": (case_attention, dict(Hq=64, Hkv=8, B=16, lo=2048, hi=16384)),  # 32B-class, 128 rows per KV head
+    "attention32b_w2048": (case_attention, dict(Hq=64, Hkv=8, B=128, lo=2048, hi=16384, window=2048)),   # the paper's window
     "gemm": (case_gemm, {}),                                                       # the 2-SM kernel, M = 2048
     "gemm_skinny": (case_gemm, dict(M=32, n_out=65536, K=4096)),                   # weight streaming, Proj_dS class
     "gemm_skinny64": (case_gemm, dict(M=64, n_out=262144, K=5120)),                # Proj_dS at concurrency 64 (a fifth of it)

@@ -293,7 +293,9 @@ int rows_per_cta(int R) { int rt = ((R + 15) / 16) * 16; return rt > 128 ? 128 :
 }  // namespace
 
 int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms) {
-  int lmax = (window > 0 && window < max_ctx) ? window : max_ctx;
+  // with a window the visible range starts on a page boundary, up to 15 tokens before the window itself: size the
+  // chunks for window + 15 tokens, or a request's last few tokens become a chunk (and a merge) of their own
+  int lmax = (window > 0 && window + 15 < max_ctx) ? window + 15 : max_ctx;
   if (lmax < 1) lmax = 1;
   int nsplit = (2 * num_sms + B * Hkv - 1) / (B * Hkv);
   if (nsplit < 1) nsplit = 1;
