@@ -577,11 +577,11 @@ def _randn(shape, seed, std, dtype):
     return (torch.randn(shape, generator=g, device="cuda", dtype=torch.float32) * std).to(dtype)
 
 
-def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16, window=0):
-    """One attention layer of the serving shapes: dh = 128, contexts uniform in [lo, hi]."""
+def case_attention(reps, Hq=32, Hkv=8, B=32, lo=512, hi=8192, k=16, window=0, dist="uniform"):
+    """One attention layer of the serving shapes: dh = 128, contexts drawn from [lo, hi]."""
     import paper_2609_24197_b200 as hs
     dh = 128
-    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16, B=B, ctx=("uniform", lo, hi))
+    cfg = dict(page_size=16, Hkv=Hkv, dh=dh, n_slots=1, n_fuse=1, D=8, V=16, B=B, ctx=(dist, lo, hi))
     ctx = synth.make_ctx_lens(cfg)
     batch = synth.make_request_batch(cfg, ctx_lens=ctx, device="cuda")
     M = B * k
@@ -636,16 +636,59 @@ def case_scan(reps):
     print(f"scan: B={B} H={H} S_init bytes per launch={B * H * P * N * 2}")
 
 
+def case_overlap(reps):
+    """Does the weight-streaming state projection (HBM-bound) overlap with a tensor-bound GEMM when both are in flight?
+    Proj_dS of the 32B-class drafter at 128 rows (a fifth of it) on one stream, the layer's in-projection at 2048 rows
+    on another: serial time vs the time with both streams fed at once."""
+    import paper_2609_24197_b200 as hs
+    xs, Ws = _randn((128, 5120), 11, 1.0, torch.float16), _randn((262144, 5120), 12, 0.02, torch.float16)
+    ys = torch.empty((128, 262144), dtype=torch.float16, device="cuda")
+    xg, Wg = _randn((2048, 5120), 13, 1.0, torch.float16), _randn((21664, 5120), 14, 0.02, torch.float16)
+    yg = torch.empty((2048, 21664), dtype=torch.float32, device="cuda")
+    ws_s = torch.empty(hs.hspec_gemm_workspace_bytes(128, 262144, 5120), dtype=torch.uint8, device="cuda")
+    ws_g = torch.empty(hs.hspec_gemm_workspace_bytes(2048, 21664, 5120), dtype=torch.uint8, device="cuda")
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    n_g = 5                                         # five in-projections ~ the tensor-bound work next to one projection
+
+    def run(parallel):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        s1.wait_stream(torch.cuda.current_stream())
+        s2.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s1):
+            hs.hspec_op_gemm(xs, Ws, ys, workspace=ws_s)
+        if not parallel:
+            s2.wait_stream(s1)
+        with torch.cuda.stream(s2):
+            for _ in range(n_g):
+                hs.hspec_op_gemm(xg, Wg, yg, workspace=ws_g)
+        torch.cuda.current_stream().wait_stream(s1)
+        torch.cuda.current_stream().wait_stream(s2)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e3
+    for _ in range(2):
+        run(False), run(True)
+    ser = [round(run(False), 1) for _ in range(reps)]
+    par = [round(run(True), 1) for _ in range(reps)]
+    print(f"overlap: state projection (128 x 262144 x 5120) + {n_g} x in-projection (2048 x 21664 x 5120): one after the other "
+          f"{ser} us, both streams at once {par} us")
+
+
 CASES = {
     # name: (function, keyword arguments) - each runs ONE kernel family a few times on inputs larger than L2
     "attention": (case_attention, {}),                                             # 8B-class, 64 query rows per KV head
     "attention32b": (case_attention, dict(Hq=64, Hkv=8, B=16, lo=2048, hi=16384)),  # 32B-class, 128 rows per KV head
+    "attention32b_full": (case_attention, dict(Hq=64, Hkv=8, B=128, lo=1024, hi=32768, dist="loguniform")),  # conc128_32b's layer
+    "attention8b_full": (case_attention, dict(Hq=32, Hkv=8, B=128, lo=1024, hi=16384)),                       # sweep B = 128, k = 16
     "attention32b_w2048": (case_attention, dict(Hq=64, Hkv=8, B=128, lo=2048, hi=16384, window=2048)),   # the paper's window
     "gemm": (case_gemm, {}),                                                       # the 2-SM kernel, M = 2048
     "gemm_skinny": (case_gemm, dict(M=32, n_out=65536, K=4096)),                   # weight streaming, Proj_dS class
     "gemm_skinny64": (case_gemm, dict(M=64, n_out=262144, K=5120)),                # Proj_dS at concurrency 64 (a fifth of it)
     "gemm_skinny128": (case_gemm, dict(M=128, n_out=262144, K=5120)),              # Proj_dS at concurrency 128 (a fifth of it)
     "scan": (case_scan, {}),
+    "overlap": (case_overlap, {}),
 }
 
 

@@ -452,6 +452,8 @@ void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out
       if (cost < best_cost) { best_cost = cost; best_bnt = bnt; best_s = s; }
     }
   }
+  static const int bnt_env = [] { const char* e = getenv("HSPEC_GEMM2_BNT"); return e ? atoi(e) : 0; }();   // measurements only
+  if (bnt_env == 128 || bnt_env == 256) { best_bnt = bnt_env; best_s = 1; }
   *bnt_out = best_bnt;
   *splits_out = best_s;
 }
