@@ -801,6 +801,18 @@ def main_ours(args):
                 print(f"[bench] window row of {name} skipped: {exc}", file=sys.stderr)
             torch.cuda.empty_cache()
         line["window_2048"] = win
+        # the same headline workload with bf16 tensor-core operands (act_bf16 = 1: the caller's bf16 matrices used in place,
+        # bf16 activations) beside the default fp16 operands
+        try:
+            r = run_workload(args.workload, args.steps, args.warmup, rank, clock_gpu=torch.cuda.current_device(),
+                             want_e2e=False, settle_s=min(args.settle_s, 1.0), want_graph=False, act_bf16=1)
+            t = summarize(r, peaks, traffic)
+            line["bf16_operands"] = dict(brief(t, r), workload=args.workload, gemm=t["gemm"],
+                                         note="act_bf16 = 1; parity bound 5e-2 of the output RMS instead of 2e-2 (8-bit operands)")
+            del r
+        except Exception as exc:
+            print(f"[bench] bf16-operand row skipped: {exc}", file=sys.stderr)
+        torch.cuda.empty_cache()
         if not args.no_sweep:
             try:
                 line["sweep"] = run_sweep(args.sweep_steps, args.warmup, peaks, rank)

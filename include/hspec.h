@@ -99,10 +99,17 @@ typedef struct {
   int32_t markov_rank;       /* 0, or the rank of the causal-correction head applied after the LM head (Sec. 3.3.3; 256 in
                                 App. B.1): tensors `markov_in` [V, rank] and `markov_out` [V or V_draft, rank] are then
                                 required and the draft ids follow hspec_op_markov_head's rule */
+  int32_t act_bf16;          /* 0 (default): fp16 tensor-core operands, see "Precision".  1: bf16 operands - the GEMM
+                                matrices are used where the caller put them (no library copy, except w_gate_up, whose rows
+                                the fused SwiGLU epilogue needs interleaved), activations are stored as bf16; no fp16
+                                range limit, but 8 instead of 11 significant bits on every GEMM input (measured on the
+                                mid-size test step: 2.0e-2 of the hidden state's RMS and 2.3e-2 of the logits' RMS at the
+                                maximum, against 4.6e-3 and 5.0e-3 with fp16 operands) */
 } hspec_config;
 
 /* A named tensor in DEVICE memory.  hspec_load_weights copies it (converting GEMM matrices to fp16), so
- * the caller may free or reuse it afterwards.  Names (l = layer index):
+ * the caller may free or reuse it afterwards - except with act_bf16 = 1, where the bf16 GEMM matrices are BORROWED:
+ * they must stay valid and unchanged until hspec_destroy.  Names (l = layer index):
  *   embed [V,D]  proj_r [r, n_fuse*D]  proj_ds [H*P*N, r]  final_norm [D]  lm_head [V,D] (or [V_draft,D])
  *   vocab_map [V_draft] int32 (only if V_draft > 0: target token id of each LM-head row, ascending)
  *   markov_in [V, markov_rank]  markov_out [V or V_draft, markov_rank]  (only if markov_rank > 0)

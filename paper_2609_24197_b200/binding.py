@@ -40,7 +40,7 @@ class hspec_config(C.Structure):
         ("rope_theta", C.c_float), ("window", C.c_int32), ("qk_norm", C.c_int32), ("F", C.c_int32),
         ("V", C.c_int32), ("V_draft", C.c_int32), ("mask_id", C.c_int32), ("rms_eps", C.c_float), ("page_size", C.c_int32),
         ("max_batch", C.c_int32), ("max_k", C.c_int32), ("max_pages_per_req", C.c_int32),
-        ("markov_rank", C.c_int32),
+        ("markov_rank", C.c_int32), ("act_bf16", C.c_int32),
     ]
 
 
@@ -155,6 +155,7 @@ def make_config(cfg, max_batch=None, max_k=None, max_pages_per_req=None):
         setattr(c, name, int(cfg[name]))
     c.V_draft = int(cfg.get("V_draft", 0))
     c.markov_rank = int(cfg.get("markov_rank", 0))
+    c.act_bf16 = int(cfg.get("act_bf16", 0))
     c.rope_theta = float(cfg["rope_theta"])
     c.rms_eps = float(cfg["rms_eps"])
     for l in range(int(cfg["L"])):
@@ -392,6 +393,7 @@ class Drafter:
         if not torch.cuda.is_available():
             raise HSpecError("no CUDA device: the H-Spec draft step has no CPU path")
         self.cfg = cfg
+        self.weights = weights if cfg.get("act_bf16", 0) else None     # bf16 mode borrows the GEMM matrices: keep them alive
         ps = cfg["page_size"]
         self.max_pages = max(1, (max_ctx + ps - 1) // ps)
         self.config = make_config(cfg, max_batch, max_k, self.max_pages)

@@ -25,7 +25,8 @@ struct AttnArgs {
   const int32_t* ctx_lens;
   float* ws_o;       // [B, Hkv, max_chunks, R, DH]
   float* ws_ml;      // [B, Hkv, max_chunks, R, 2]
-  __half* o;         // [B*k, Hq*DH]
+  void* o;           // [B*k, Hq*DH] fp16 (or bf16 when o_bf16)
+  int o_bf16;
   uint32_t* status;
   int page_table_stride;
   int B, k, Hq, Hkv, rep, R, RT, n_row_tiles;
@@ -272,7 +273,7 @@ __global__ void attn_merge_kernel(AttnArgs a) {
       L += ml[1] * w;
       acc += a.ws_o[((slab0 + c) * a.R + r) * DH + d] * w;
     }
-    a.o[(size_t(m) * a.Hq + hq) * DH + d] = f16_sat(acc / L, a.status);
+    store_act16(a.o, (size_t(m) * a.Hq + hq) * DH + d, acc / L, a.o_bf16 != 0, a.status);
   }
 }
 
@@ -330,7 +331,7 @@ cudaError_t attention_launch(const AttnCall& c, cudaStream_t stream, Tracker* tr
   AttnArgs a{};
   a.q = (const __nv_bfloat16*)c.q; a.kb = (const __nv_bfloat16*)c.kb; a.vb = (const __nv_bfloat16*)c.vb;
   a.k_pool = (const __nv_bfloat16*)c.k_pool; a.v_pool = (const __nv_bfloat16*)c.v_pool;
-  a.page_table = c.page_table; a.ctx_lens = c.ctx_lens; a.o = (__half*)c.o;
+  a.page_table = c.page_table; a.ctx_lens = c.ctx_lens; a.o = c.o; a.o_bf16 = c.o_bf16 ? 1 : 0;
   a.page_table_stride = c.page_table_stride;
   a.B = c.B; a.k = c.k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.rep = c.Hq / c.Hkv;
   a.R = c.k * a.rep; a.RT = rows_per_cta(a.R); a.n_row_tiles = (a.R + a.RT - 1) / a.RT;

@@ -46,7 +46,9 @@ struct AttnTcArgs {
   const int32_t* ctx_lens;
   float* ws_o;
   float* ws_ml;
-  __half* o_final;       // [B*k, Hq, dh] fp16: requests whose context is one chunk are finished here, without partials
+  uint16_t* o_final;     // [B*k, Hq, dh] fp16 (or bf16 when o_bf16): requests whose context is one chunk are finished
+                         // here, without partials; the merge kernel writes the others
+  int o_bf16;
   uint32_t* status;
   int page_table_stride;
   int B, k, Hq, Hkv, rep, R, n_row_tiles;
@@ -668,7 +670,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       } else if (whole) {
         // (the last chunk always holds the row's own block key, so the row sum is positive)
         const float inv = 1.f / l_row;
-        __half* dsth = a.o_final + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH + hf * 64;
+        uint16_t* dsth = a.o_final + ((size_t(b) * a.k + (row_ok ? i_blk : 0)) * a.Hq + kvh * a.rep + (row_ok ? rg % a.rep : 0)) * DH + hf * 64;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           uint32_t o[32];
@@ -680,9 +682,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
               uint32_t h[4];
 #pragma unroll
               for (int q2 = 0; q2 < 4; ++q2) {
-                const __half2 v = __halves2half2(f16_sat(__uint_as_float(o[e + 2 * q2]) * inv, a.status),
-                                                 f16_sat(__uint_as_float(o[e + 2 * q2 + 1]) * inv, a.status));
-                h[q2] = *reinterpret_cast<const uint32_t*>(&v);
+                const float v0 = __uint_as_float(o[e + 2 * q2]) * inv, v1 = __uint_as_float(o[e + 2 * q2 + 1]) * inv;
+                if (a.o_bf16) {
+                  h[q2] = pack_bf16(v0, v1);
+                } else {
+                  const __half2 v = __halves2half2(f16_sat(v0, a.status), f16_sat(v1, a.status));
+                  h[q2] = *reinterpret_cast<const uint32_t*>(&v);
+                }
               }
               *reinterpret_cast<uint4*>(dsth + j * 32 + e) = make_uint4(h[0], h[1], h[2], h[3]);
             }
@@ -731,7 +737,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 }
 
 // One block per (row of the block, query head): merge the chunk partials in chunk order (page-aligned chunk geometry).
-__global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n_pairs) {
+__global__ void attn_tc_merge_kernel(AttnTcArgs a, uint16_t* __restrict__ o, int n_pairs) {
   pdl_wait();
   pdl_trigger();
   // one warp per (row, head): each lane merges four adjacent head-dim columns with 16-byte loads
@@ -757,11 +763,16 @@ __global__ void attn_tc_merge_kernel(AttnTcArgs a, __half* __restrict__ o, int n
     acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
   }
   const float inv = 1.f / L;
-  const __half2 lo = __halves2half2(f16_sat(acc.x * inv, a.status), f16_sat(acc.y * inv, a.status));
-  const __half2 hi = __halves2half2(f16_sat(acc.z * inv, a.status), f16_sat(acc.w * inv, a.status));
   uint2 out;
-  out.x = *reinterpret_cast<const uint32_t*>(&lo);
-  out.y = *reinterpret_cast<const uint32_t*>(&hi);
+  if (a.o_bf16) {
+    out.x = pack_bf16(acc.x * inv, acc.y * inv);
+    out.y = pack_bf16(acc.z * inv, acc.w * inv);
+  } else {
+    const __half2 lo = __halves2half2(f16_sat(acc.x * inv, a.status), f16_sat(acc.y * inv, a.status));
+    const __half2 hi = __halves2half2(f16_sat(acc.z * inv, a.status), f16_sat(acc.w * inv, a.status));
+    out.x = *reinterpret_cast<const uint32_t*>(&lo);
+    out.y = *reinterpret_cast<const uint32_t*>(&hi);
+  }
   reinterpret_cast<uint2*>(o + (size_t(m) * a.Hq + hq) * DH)[d4] = out;
 }
 
@@ -814,7 +825,8 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   a.scale_log2 = 1.4426950408889634f / sqrtf(float(c.dh));
   const size_t slabs = size_t(c.B) * c.Hkv * max_chunks;
   a.ws_o = reinterpret_cast<float*>(c.ws);
-  a.o_final = reinterpret_cast<__half*>(c.o);
+  a.o_final = reinterpret_cast<uint16_t*>(c.o);
+  a.o_bf16 = c.o_bf16 ? 1 : 0;
   a.ws_ml = a.ws_o + slabs * a.R * c.dh;
   CUtensorMap tmK, tmV;
   if (!make_pool_tmap(&tmK, c.k_pool, c.num_pages, c.Hkv, err) || !make_pool_tmap(&tmV, c.v_pool, c.num_pages, c.Hkv, err))
@@ -846,7 +858,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   if (e != cudaSuccess) return e;
   const int n_pairs = c.B * c.k * c.Hq;
   trk_begin(trk, "attn_merge");
-  launch_pdl(attn_tc_merge_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, a, reinterpret_cast<__half*>(c.o), n_pairs);
+  launch_pdl(attn_tc_merge_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, a, reinterpret_cast<uint16_t*>(c.o), n_pairs);
   trk_end(trk);
   return cudaGetLastError();
 }

@@ -53,6 +53,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // (fast exponential and fast division: ~2 ulp each, far inside every tolerance that follows an fp16 or bf16 rounding)
 __device__ __forceinline__ float silu_f(float v) { return __fdividef(v, 1.0f + __expf(-v)); }
 
+// Stores v into a 16-bit activation buffer: fp16 with saturation (counted), or bf16 (fp32's range: nothing to clamp).
+__device__ __forceinline__ void store_act16(void* base, size_t idx, float v, bool bf16, uint32_t* status) {
+  if (bf16) reinterpret_cast<__nv_bfloat16*>(base)[idx] = __float2bfloat16_rn(v);
+  else reinterpret_cast<__half*>(base)[idx] = f16_sat(v, status);
+}
+
 // ------------------------------------------------------------------ programmatic dependent launch
 // A kernel launched with launch_pdl() may start while the kernel before it on the stream is still running: its CTAs
 // run their set-up and then block in pdl_wait() until that kernel has finished and its writes are visible.  Nothing
@@ -230,7 +236,7 @@ __device__ __forceinline__ uint32_t umma_idesc_m128(uint32_t n, bool f16) {
 // of 16: lanes 0..15 of a warp hold the gate pre-activation of 16 features, lanes 16..31 the up projection of the same
 // features.  Columns are handled in pairs: the lower half-warp finishes the even column, the upper half the odd one,
 // so all 32 lanes compute and store.  `f` is the feature index of this lane (same for lane and lane ^ 16).
-__device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], __half* out, long long ldo, int m_first, int M, int f,
+__device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], void* out, bool bf16, long long ldo, int m_first, int M, int f,
                                                bool f_ok, int lane, uint32_t* status) {
   const bool upper = lane >= 16;
 #pragma unroll
@@ -241,7 +247,7 @@ __device__ __forceinline__ void swiglu_store16(const uint32_t (&r)[16], __half* 
     const float gate = upper ? recv : mine_even;               // upper half: partner's gate of the odd column
     const float up = upper ? mine_odd : recv;                  // lower half: partner's up of the even column
     const int m = m_first + j + (upper ? 1 : 0);
-    if (f_ok && m < M) out[size_t(m) * ldo + f] = f16_sat(silu_f(gate) * up, status);
+    if (f_ok && m < M) store_act16(out, size_t(m) * ldo + f, silu_f(gate) * up, bf16, status);
   }
 }
 

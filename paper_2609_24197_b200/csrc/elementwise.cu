@@ -37,14 +37,14 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return r;
 }
 
-// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 out.
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, __half* __restrict__ y,
-                               int n, float eps, uint32_t* status) {
+// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 (or bf16) out.
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, void* __restrict__ y,
+                               int n, float eps, uint32_t* status, int bf16_out) {
   pdl_wait();
   pdl_trigger();
   __shared__ float red[32];
   const float* xr = x + size_t(blockIdx.x) * n;
-  __half* yr = y + size_t(blockIdx.x) * n;
+  uint16_t* yr = reinterpret_cast<uint16_t*>(y) + size_t(blockIdx.x) * n;      // a row of 16-bit values, either type
   if ((n & 3) == 0 && n <= 4 * 6 * int(blockDim.x)) {
     // 16-byte loads, the row stays in registers between the two passes
     float4 v[6];
@@ -64,11 +64,16 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
         const float4 g = reinterpret_cast<const float4*>(w)[d4];
         // (a normalised value is at most sqrt(n) |w|; the saturating convert still guards a huge gain or a NaN-free
         // overflow of x * inv)
-        const __half2 lo = __halves2half2(f16_sat(v[i].x * inv * g.x, status), f16_sat(v[i].y * inv * g.y, status));
-        const __half2 hi = __halves2half2(f16_sat(v[i].z * inv * g.z, status), f16_sat(v[i].w * inv * g.w, status));
         uint2 out;
-        out.x = *reinterpret_cast<const uint32_t*>(&lo);
-        out.y = *reinterpret_cast<const uint32_t*>(&hi);
+        if (bf16_out) {
+          out.x = pack_bf16(v[i].x * inv * g.x, v[i].y * inv * g.y);
+          out.y = pack_bf16(v[i].z * inv * g.z, v[i].w * inv * g.w);
+        } else {
+          const __half2 lo = __halves2half2(f16_sat(v[i].x * inv * g.x, status), f16_sat(v[i].y * inv * g.y, status));
+          const __half2 hi = __halves2half2(f16_sat(v[i].z * inv * g.z, status), f16_sat(v[i].w * inv * g.w, status));
+          out.x = *reinterpret_cast<const uint32_t*>(&lo);
+          out.y = *reinterpret_cast<const uint32_t*>(&hi);
+        }
         reinterpret_cast<uint2*>(yr)[d4] = out;
       }
     }
@@ -78,7 +83,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   for (int d = threadIdx.x; d < n; d += blockDim.x) { const float v = xr[d]; ss += v * v; }
   const float tot = block_sum(ss, red);
   const float inv = rsqrtf(tot / float(n) + eps);
-  for (int d = threadIdx.x; d < n; d += blockDim.x) yr[d] = f16_sat(xr[d] * inv * w[d], status);
+  for (int d = threadIdx.x; d < n; d += blockDim.x) store_act16(yr, d, xr[d] * inv * w[d], bf16_out != 0, status);
 }
 
 // Per (row, head): optional RMSNorm over dh, then rotate-half RoPE at position ctx_len + i.
@@ -169,7 +174,7 @@ __global__ void kv_inject_write_kernel(const float* __restrict__ kv, const float
   }
 }
 
-__global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__ h, int M, int F, uint32_t* status) {
+__global__ void swiglu_kernel(const float* __restrict__ gu, void* __restrict__ h, int M, int F, uint32_t* status, int bf16_out) {
   pdl_wait();
   pdl_trigger();
   const long long total = (long long)M * F;
@@ -177,7 +182,7 @@ __global__ void swiglu_kernel(const float* __restrict__ gu, __half* __restrict__
        idx += (long long)gridDim.x * blockDim.x) {
     const int m = int(idx / F), f = int(idx % F);
     const float gte = gu[size_t(m) * 2 * F + f], up = gu[size_t(m) * 2 * F + F + f];
-    h[idx] = f16_sat(silu_f(gte) * up, status);
+    store_act16(h, size_t(idx), silu_f(gte) * up, bf16_out != 0, status);
   }
 }
 
@@ -224,10 +229,10 @@ cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token,
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream,
-                           uint32_t* status) {
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_16, int M, int n, float eps, cudaStream_t stream,
+                           uint32_t* status, bool bf16_out) {
   const int threads = n >= 2048 ? 512 : 256;
-  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, (__half*)y_f16, n, eps, status);
+  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, y_16, n, eps, status, bf16_out ? 1 : 0);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
@@ -256,9 +261,9 @@ cudaError_t kv_inject_write_launch(const float* kv, const float* kw, const int32
   return cudaGetLastError();
 }
 
-cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream, uint32_t* status) {
-  cudaError_t e = launch_pdl(swiglu_kernel, dim3(grid_for((long long)M * F, 256)), dim3(256), 0, stream, gu, (__half*)h_f16, M, F,
-                             status);
+cudaError_t swiglu_launch(const float* gu, void* h_16, int M, int F, cudaStream_t stream, uint32_t* status, bool bf16_out) {
+  cudaError_t e = launch_pdl(swiglu_kernel, dim3(grid_for((long long)M * F, 256)), dim3(256), 0, stream, gu, h_16, M, F,
+                             status, bf16_out ? 1 : 0);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 

@@ -189,9 +189,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const int m = m0 + c0 + j;
           if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = __float2bfloat16_rn(__uint_as_float(r[j]));
         }
-      } else if (g.mode == EPI_SWIGLU_F16) {
+      } else if (g.mode == EPI_SWIGLU_F16 || g.mode == EPI_SWIGLU_BF16) {
         const int f = tile_w * 64 + q * 16 + (lane & 15);
-        swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
+        swiglu_store16(r, g.out, g.mode == EPI_SWIGLU_BF16, g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
       } else if (g.mode == EPI_STORE_F16) {
         __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll
@@ -268,13 +268,13 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ part, int splits,
     if (mode == EPI_STORE_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] = acc;
     else if (mode == EPI_ACCUM_F32) reinterpret_cast<float*>(out)[size_t(m) * ldo + n] += acc;
     else if (mode == EPI_STORE_F16) reinterpret_cast<__half*>(out)[size_t(m) * ldo + n] = f16_sat(acc, status);
-    else if (mode == EPI_SWIGLU_F16) {
+    else if (mode == EPI_SWIGLU_F16 || mode == EPI_SWIGLU_BF16) {
       // n runs over interleaved rows; lower half of each 32-row block = gate, upper half = up of the same 16 features
       if ((n & 31) < 16) {
         float up = 0.f;
         for (int s = 0; s < splits; ++s) up += part[(size_t(s) * M + m) * N + n + 16];
         const int f = (n >> 5) * 16 + (n & 15);
-        reinterpret_cast<__half*>(out)[size_t(m) * ldo + f] = f16_sat(silu_f(acc) * up, status);
+        store_act16(out, size_t(m) * ldo + f, silu_f(acc) * up, mode == EPI_SWIGLU_BF16, status);
       }
     }
     else reinterpret_cast<__nv_bfloat16*>(out)[size_t(m) * ldo + n] = __float2bfloat16_rn(acc);

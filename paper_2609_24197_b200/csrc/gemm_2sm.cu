@@ -296,9 +296,9 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int m = m0 + c0 + j;
             if (n_ok && m < g.M) out[size_t(m) * g.ldo + n] = old[j] + __uint_as_float(r[j]);
           }
-        } else if (mode == EPI_SWIGLU_F16) {
+        } else if (mode == EPI_SWIGLU_F16 || mode == EPI_SWIGLU_BF16) {
           const int f = tile_n128 * 64 + q * 16 + (lane & 15);
-          swiglu_store16(r, reinterpret_cast<__half*>(g.out), g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
+          swiglu_store16(r, g.out, mode == EPI_SWIGLU_BF16, g.ldo, m0 + c0, g.M, f, 2 * f < g.N_out, lane, g.status);
         } else if (mode == EPI_STORE_F16) {
           __half* out = reinterpret_cast<__half*>(g.out);
 #pragma unroll
@@ -399,9 +399,9 @@ gemm2_tail_reduce_kernel(Gemm2Args g) {
 #pragma unroll
     for (int sp = 0; sp < TAIL_MAX_SPLITS; ++sp)
       if (sp < g.tail_splits) acc += v[sp][j];
-    if (g.mode == EPI_SWIGLU_F16) {
+    if (g.mode == EPI_SWIGLU_F16 || g.mode == EPI_SWIGLU_BF16) {
       const float up = __shfl_xor_sync(0xffffffffu, acc, 16);
-      if (lane < 16 && 2 * f < g.N_out) reinterpret_cast<__half*>(g.out)[size_t(m) * g.ldo + f] = f16_sat(silu_f(acc) * up, g.status);
+      if (lane < 16 && 2 * f < g.N_out) store_act16(g.out, size_t(m) * g.ldo + f, silu_f(acc) * up, g.mode == EPI_SWIGLU_BF16, g.status);
       continue;
     }
     if (n >= g.N_out) continue;

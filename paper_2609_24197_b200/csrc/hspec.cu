@@ -23,7 +23,9 @@ constexpr int kNumSMs = 148;   // B200; only used to size grids and K-slices
 thread_local std::string g_err;
 
 struct Weight {
-  void* data = nullptr;      // library-owned device copy (GEMM matrices as fp16, everything else as given)
+  void* data = nullptr;      // library-owned device copy (GEMM matrices as fp16, everything else as given); with bf16
+                             // activations the GEMM matrices are the caller's own (owned = false)
+  bool owned = true;
   int dtype = 0;
   int64_t rows = 0, cols = 0;
   bool has_tm = false;
@@ -287,14 +289,15 @@ __global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half
 
 // w_gate_up [2F, K] bf16 (rows gate | up) -> fp16 with rows interleaved in blocks of 16:
 // dst rows [32j, 32j+16) = gate rows [16j, 16j+16), dst rows [32j+16, 32j+32) = up rows [16j, 16j+16).
-__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int F, int K,
-                                          uint32_t* status) {
+__global__ void interleave_gate_up_kernel(const __nv_bfloat16* __restrict__ src, void* __restrict__ dst, int F, int K,
+                                          uint32_t* status, int keep_bf16) {
   const size_t total = size_t(2) * F * K;
   for (size_t i = blockIdx.x * size_t(blockDim.x) + threadIdx.x; i < total; i += size_t(gridDim.x) * blockDim.x) {
     const size_t r = i / K, c = i % K;
     const size_t blk = r >> 5, w = r & 31;
     const size_t src_row = (w < 16) ? blk * 16 + w : size_t(F) + blk * 16 + (w - 16);
-    dst[i] = f16_sat(__bfloat162float(src[src_row * K + c]), status);
+    if (keep_bf16) reinterpret_cast<__nv_bfloat16*>(dst)[i] = src[src_row * K + c];
+    else reinterpret_cast<__half*>(dst)[i] = f16_sat(__bfloat162float(src[src_row * K + c]), status);
   }
 }
 
@@ -310,12 +313,12 @@ __global__ void wait_selftest_kernel(uint32_t* status, unsigned long long limit_
 }
 
 __global__ void cvt_cols_f16_kernel(const float* __restrict__ src, long long ld, int col0, int ncols, int M,
-                                    __half* __restrict__ dst, uint32_t* status) {
+                                    void* __restrict__ dst, uint32_t* status, int bf16_out) {
   pdl_wait();
   pdl_trigger();
   const int total = M * ncols;
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x)
-    dst[i] = f16_sat(src[size_t(i / ncols) * ld + col0 + i % ncols], status);
+    store_act16(dst, size_t(i), src[size_t(i / ncols) * ld + col0 + i % ncols], bf16_out != 0, status);
 }
 
 }  // namespace
@@ -374,23 +377,35 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
       return fail(h, HSPEC_ERR_BAD_SHAPE, "hspec_load_weights: '" + name + "' has the wrong shape or dtype (expected [" +
                                               std::to_string(rows) + (cols ? "," + std::to_string(cols) : "") + "])");
     auto old = h->w.find(name);
-    if (old != h->w.end()) { cudaFree(old->second.data); h->w.erase(old); }
+    if (old != h->w.end()) { if (old->second.owned) cudaFree(old->second.data); h->w.erase(old); }
     Weight w;
     w.dtype = dtype; w.rows = rows; w.cols = cols;
     const size_t count = size_t(rows) * size_t(cols ? cols : 1);
     const size_t bytes = count * ((dtype == HSPEC_F32 || dtype == HSPEC_I32) ? 4 : 2);
+    const bool bf16_mode = h->cfg.act_bf16 != 0;
+    const bool is_gate_up = name.size() >= 13 && name.compare(name.size() - 13, 13, "mlp.w_gate_up") == 0 && h->cfg.F % 16 == 0;
+    if (gemm && bf16_mode && !is_gate_up) {
+      // bf16 operands: the matrix is used where it lies (borrowed until hspec_destroy)
+      w.data = const_cast<void*>(t[i].data);
+      w.owned = false;
+      if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, false, &errtxt))
+        return fail(h, HSPEC_ERR_BAD_SHAPE, "hspec_load_weights: '" + name + "': " + errtxt);
+      w.has_tm = true;
+      h->w[name] = w;
+      continue;
+    }
     CUDA_TRY(h, cudaMalloc(&w.data, bytes));
     if (gemm) {
       // bf16 -> fp16: exact for every value with |w| in [2^-17, 65504]; smaller ones lose at most 2^-25
       const int blocks = int(std::min<size_t>((count + 255) / 256, 148 * 32));
-      if (name.size() >= 13 && name.compare(name.size() - 13, 13, "mlp.w_gate_up") == 0 && h->cfg.F % 16 == 0)
-        interleave_gate_up_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
-                                                   reinterpret_cast<__half*>(w.data), h->cfg.F, int(cols), h->d_status);
+      if (is_gate_up)
+        interleave_gate_up_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data), w.data, h->cfg.F,
+                                                   int(cols), h->d_status, bf16_mode ? 1 : 0);
       else
         bf16_to_f16_kernel<<<blocks, 256>>>(reinterpret_cast<const __nv_bfloat16*>(t[i].data),
                                             reinterpret_cast<__half*>(w.data), count, h->d_status);
       CUDA_TRY(h, cudaGetLastError());
-      if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, true, &errtxt)) {
+      if (!make_tmap_16bit_2d(&w.tm, w.data, rows, cols, cols, 128, !bf16_mode, &errtxt)) {
         cudaFree(w.data);
         return fail(h, HSPEC_ERR_BAD_SHAPE, "hspec_load_weights: '" + name + "': " + errtxt);
       }
@@ -407,7 +422,7 @@ int hspec_load_weights(hspec_handle* h, const hspec_tensor* t, int32_t n) {
 int hspec_destroy(hspec_handle* h) {
   if (!h) return HSPEC_ERR_INVALID_ARG;
   if (h->d_status) cudaFree(h->d_status);
-  for (auto& kv : h->w) cudaFree(kv.second.data);
+  for (auto& kv : h->w) if (kv.second.owned) cudaFree(kv.second.data);
   h->trk.destroy();
   delete h;
   return HSPEC_OK;
@@ -501,13 +516,14 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
   const uint64_t launches0 = trk->launches;
   const double Md = double(M);
 
+  const bool bf = c.act_bf16 != 0;                 // bf16 tensor-core operands instead of fp16
   auto W = [&](const std::string& nm) -> const Weight& { return h->w.at(nm); };
   auto fptr = [&](const std::string& nm) { return reinterpret_cast<const float*>(h->w.at(nm).data); };
   auto gemm = [&](const std::string& wname, const char* label, const void* x, int rows, int mode, void* o,
                   long long ldo) -> cudaError_t {
     const Weight& w = W(wname);
     GemmCall g{};
-    g.tmW = &w.tm; g.x = x; g.f16 = true; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
+    g.tmW = &w.tm; g.x = x; g.f16 = !bf; g.ldx = w.cols; g.M = rows; g.n_out = int(w.rows); g.K = int(w.cols);
     g.mode = mode; g.out = o; g.ldo = ldo;
     g.splits = gemm_pick_splits(rows, g.n_out, g.K, kNumSMs, mode);
     g.splitk_ws = ws + p.SPLITK; g.splitk_ws_bytes = p.splitk_bytes;
@@ -519,27 +535,32 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
 
   EW("embed_rows", Md * c.D * 6, embed_rows_launch(W("embed").data, in->last_token, c.mask_id, X, B, k, c.D, st));
   // S_init = Proj_dS(Proj_r(concat h)): once per step, shared by all layers
-  {
+  const void* lh_in = LH;
+  if (bf && (reinterpret_cast<uintptr_t>(in->last_hidden) & 15) == 0) {
+    lh_in = in->last_hidden;                       // already the operand type: read in place
+  } else {
     const size_t n_lh = size_t(B) * c.n_fuse * c.D;
     trk->begin("cvt_last_hidden", 0, double(n_lh) * 4);
-    bf16_to_f16_kernel<<<int(std::min<size_t>((n_lh + 255) / 256, 148 * 8)), 256, 0, st>>>(
+    if (bf) CUDA_TRY(h, cudaMemcpyAsync(LH, in->last_hidden, n_lh * 2, cudaMemcpyDeviceToDevice, st));
+    else bf16_to_f16_kernel<<<int(std::min<size_t>((n_lh + 255) / 256, 148 * 8)), 256, 0, st>>>(
         reinterpret_cast<const __nv_bfloat16*>(in->last_hidden), reinterpret_cast<__half*>(LH), n_lh, h->d_status);
     trk->end();
     CUDA_TRY(h, cudaGetLastError());
   }
-  CUDA_TRY(h, gemm("proj_r", "gemm:proj_r", LH, B, EPI_STORE_F16, Fv, c.r));
+  CUDA_TRY(h, gemm("proj_r", "gemm:proj_r", lh_in, B, bf ? EPI_STORE_BF16 : EPI_STORE_F16, Fv, c.r));
+  // (S_init is an output the scan consumes, not a GEMM operand: it stays fp16 in both modes)
   CUDA_TRY(h, gemm("proj_ds", "gemm:proj_ds", Fv, B, EPI_STORE_F16, SINIT, d.d_S));
 
   for (int l = 0; l < c.L; ++l) {
     const std::string pre = "layers." + std::to_string(l) + ".";
     // ---- Mamba-2 mixer from the injected state
-    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mamba.norm"), U, M, c.D, c.rms_eps, st, h->d_status, bf));
     CUDA_TRY(h, gemm(pre + "mamba.in_proj", "gemm:in_proj", U, M, EPI_STORE_F32, BIG, d.d_in_proj));
     const float* dt_raw = nullptr;
     if (c.dt_rank > 0) {
       trk->begin("cvt_dt_cols", 0, Md * c.dt_rank * 6);
       cvt_cols_f16_kernel<<<(M * c.dt_rank + 255) / 256, 256, 0, st>>>(BIG, d.d_in_proj, c.Di + d.d_xBC, c.dt_rank, M,
-                                                                     reinterpret_cast<__half*>(DTL), h->d_status);
+                                                                     DTL, h->d_status, bf ? 1 : 0);
       trk->end();
       CUDA_TRY(h, cudaGetLastError());
       CUDA_TRY(h, gemm(pre + "mamba.dt_up", "gemm:dt_up", DTL, M, EPI_STORE_F32, DT, d.H));
@@ -552,11 +573,11 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     sc.y_gated = YG; sc.B = B; sc.k = k; sc.Di = c.Di; sc.P = c.P; sc.N = c.N; sc.G = c.G; sc.d_conv = c.d_conv;
     sc.ws = ws + p.SCAN; sc.ws_bytes = p.scan_bytes;
     CUDA_TRY(h, scan_launch(sc, st, trk, &errtxt));
-    EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st, h->d_status));
+    EW("rmsnorm_gated", Md * c.Di * 6, rmsnorm_launch(YG, fptr(pre + "mamba.gnorm"), U, M, c.Di, c.rms_eps, st, h->d_status, bf));
     CUDA_TRY(h, gemm(pre + "mamba.out_proj", "gemm:out_proj", U, M, EPI_ACCUM_F32, X, c.D));
     // ---- attention over the target's KV (in place) + the block
     if (c.has_attn[l]) {
-      EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
+      EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "attn.norm"), U, M, c.D, c.rms_eps, st, h->d_status, bf));
       CUDA_TRY(h, gemm(pre + "attn.wqkv", "gemm:wqkv", U, M, EPI_STORE_F32, BIG, d.d_qkv));
       EW("qk_norm_rope", Md * d.d_qkv * 6,
          qk_norm_rope_launch(BIG, fptr(pre + "attn.q_norm"), fptr(pre + "attn.k_norm"), in->ctx_lens, Q, KB, VB, B, k, c.Hq,
@@ -566,45 +587,45 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
       a.k_pool = in->k_pools[c.kv_slot[l]]; a.v_pool = in->v_pools[c.kv_slot[l]];
       a.num_pages = in->num_pages; a.status = h->d_status;
       a.page_table = in->page_table; a.page_table_stride = in->page_table_stride; a.ctx_lens = in->ctx_lens;
-      a.max_ctx = max_ctx; a.o = U; a.B = B; a.k = k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.dh = c.dh;
+      a.max_ctx = max_ctx; a.o = U; a.o_bf16 = bf; a.B = B; a.k = k; a.Hq = c.Hq; a.Hkv = c.Hkv; a.dh = c.dh;
       a.page_size = c.page_size; a.window = c.window; a.chunk_tokens = p.attn_chunk;
       a.ws = ws + p.ATT; a.ws_bytes = p.att_bytes;
       CUDA_TRY(h, attention_launch(a, st, trk, &errtxt));
       CUDA_TRY(h, gemm(pre + "attn.wo", "gemm:wo", U, M, EPI_ACCUM_F32, X, c.D));
     }
     // ---- SwiGLU MLP
-    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st, h->d_status));
+    EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr(pre + "mlp.norm"), U, M, c.D, c.rms_eps, st, h->d_status, bf));
     if (c.F % 16 == 0) {
       // gate/up rows were interleaved at load: the GEMM epilogue applies SiLU(gate) * up and writes h directly.
       // U is both the GEMM's input (D columns) and h's home (F columns), so h goes to a second fp16 buffer.
-      CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_SWIGLU_F16, U2, c.F));
+      CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, bf ? EPI_SWIGLU_BF16 : EPI_SWIGLU_F16, U2, c.F));
     } else {
       CUDA_TRY(h, gemm(pre + "mlp.w_gate_up", "gemm:gate_up", U, M, EPI_STORE_F32, BIG, 2 * c.F));
-      EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U2, M, c.F, st, h->d_status));
+      EW("swiglu", Md * c.F * 10, swiglu_launch(BIG, U2, M, c.F, st, h->d_status, bf));
     }
     CUDA_TRY(h, gemm(pre + "mlp.w_down", "gemm:down", U2, M, EPI_ACCUM_F32, X, c.D));
   }
   if (out->hidden) EW("copy_hidden", Md * c.D * 8, copy_f32_launch(X, out->hidden, size_t(M) * c.D, st));
   // ---- final norm, LM head fused with the per-row arg-max
-  EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st, h->d_status));
+  EW("rmsnorm", Md * c.D * 6, rmsnorm_launch(X, fptr("final_norm"), U, M, c.D, c.rms_eps, st, h->d_status, bf));
   const int* id_map = c.V_draft > 0 ? reinterpret_cast<const int*>(W("vocab_map").data) : nullptr;
   if (c.markov_rank > 0) {
     // ---- LM head to fp32 logits, then the causal correction position by position (Sec. 3.3.3)
     float* logits = out->logits ? out->logits : reinterpret_cast<float*>(ws + p.LOGITS);
     const Weight& w = W("lm_head");
     GemmCall g{};
-    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_STORE_F32; g.splits = 1;
+    g.tmW = &w.tm; g.x = U; g.f16 = !bf; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_STORE_F32; g.splits = 1;
     g.out = logits; g.ldo = d.Vd; g.status = h->d_status; g.label = "gemm:lm_head";
     CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
     MarkovCall mc{};
-    mc.logits = logits; mc.ld = d.Vd; mc.W_in = W("markov_in").data; mc.tmW_out = &W("markov_out").tm; mc.f16 = true;
+    mc.logits = logits; mc.ld = d.Vd; mc.W_in = W("markov_in").data; mc.tmW_out = &W("markov_out").tm; mc.f16 = !bf;
     mc.last_token = in->last_token; mc.id_map = id_map; mc.ids = out->draft_ids; mc.B = B; mc.k = k; mc.Vd = d.Vd;
     mc.r = c.markov_rank; mc.write_logits = out->logits != nullptr; mc.ws = ws + p.MARKOV; mc.status = h->d_status;
     CUDA_TRY(h, markov_launch(mc, st, trk, &errtxt));
   } else {
     const Weight& w = W("lm_head");
     GemmCall g{};
-    g.tmW = &w.tm; g.x = U; g.f16 = true; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
+    g.tmW = &w.tm; g.x = U; g.f16 = !bf; g.ldx = c.D; g.M = M; g.n_out = d.Vd; g.K = c.D; g.mode = EPI_ARGMAX; g.splits = 1;
     g.logits = out->logits; g.ldo = d.Vd;
     g.part_val = reinterpret_cast<float*>(ws + p.AMAXV); g.part_idx = reinterpret_cast<int*>(ws + p.AMAXI);
     g.status = h->d_status; g.label = "gemm:lm_head_argmax";

@@ -71,7 +71,7 @@ inline double gemm_io_bytes(int M, int n_out, int K, int mode, bool logits) {
     case 0: case 3: out = 4.0 * M * n_out; break;            // fp32 store / K-slice partial
     case 1: case 5: out = 2.0 * M * n_out; break;            // bf16 / fp16 store
     case 2: out = 8.0 * M * n_out; break;                    // fp32 read-modify-write
-    case 6: out = 1.0 * M * n_out; break;                    // SwiGLU: fp16 [M, n_out / 2]
+    case 6: case 7: out = 1.0 * M * n_out; break;            // SwiGLU: 16-bit [M, n_out / 2]
     default: out = logits ? 4.0 * M * n_out : 0; break;      // arg-max
   }
   return 2.0 * M * K + out;
@@ -98,8 +98,10 @@ enum GemmEpilogue : int {
   EPI_PARTIAL_F32 = 3,  // K-slice partial (internal)
   EPI_ARGMAX = 4,
   EPI_STORE_F16 = 5,    // y fp16 = acc
-  EPI_SWIGLU_F16 = 6,   // weight rows interleaved in blocks of 16 (gate | up): h fp16 [M, n_out/2] = SiLU(gate) * up       // per activation row (max, lowest index) over the CTA's 128 weight rows (+ optional logits)
+  EPI_SWIGLU_F16 = 6,   // weight rows interleaved in blocks of 16 (gate | up): h fp16 [M, n_out/2] = SiLU(gate) * up
+  EPI_SWIGLU_BF16 = 7,  // the same with h stored as bf16
 };
+inline bool epi_is_swiglu(int mode) { return mode == EPI_SWIGLU_F16 || mode == EPI_SWIGLU_BF16; }
 
 struct GemmArgs {       // kernel argument block
   int M, N_out, K;
@@ -190,7 +192,8 @@ struct AttnCall {
   int page_table_stride;
   const int32_t* ctx_lens;
   int max_ctx;                      // host bound on ctx_lens
-  void* o;                          // fp16 [B*k, Hq*dh]
+  void* o;                          // fp16 (or bf16 when o_bf16) [B*k, Hq*dh]
+  bool o_bf16;
   int B, k, Hq, Hkv, dh, page_size, window;
   int chunk_tokens;                 // <= 0: choose
   void* ws;
@@ -221,12 +224,12 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
 // ---- element-wise kernels (elementwise.cu)
 cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token, int mask_id, float* X, int B, int k,
                               int D, cudaStream_t stream);
-cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_f16, int M, int n, float eps, cudaStream_t stream,
-                           uint32_t* status);
+cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_16, int M, int n, float eps, cudaStream_t stream,
+                           uint32_t* status, bool bf16_out = false);
 cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* kw, const int32_t* ctx_lens, void* q,
                                 void* kb, void* vb, int B, int k, int Hq, int Hkv, int dh, float theta, float eps,
                                 int qk_norm, cudaStream_t stream);
-cudaError_t swiglu_launch(const float* gu, void* h_f16, int M, int F, cudaStream_t stream, uint32_t* status);
+cudaError_t swiglu_launch(const float* gu, void* h_16, int M, int F, cudaStream_t stream, uint32_t* status, bool bf16_out = false);
 cudaError_t copy_f32_launch(const float* src, float* dst, size_t n, cudaStream_t stream);
 
 }  // namespace hspec

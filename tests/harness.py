@@ -55,7 +55,7 @@ def oracle_step(cfg, weights, batch, k, requests=None, dtype=np.float64, **kw):
                          to_np(batch["last_token"]), k, dtype=dtype, requests=requests, **kw)
 
 
-def check_step(cfg, drafter, weights, batch, k, requests=None, dtype=np.float64, what="step"):
+def check_step(cfg, drafter, weights, batch, k, requests=None, dtype=np.float64, what="step", tol=TOL):
     """Run the CUDA step for the whole batch and the oracle for `requests`; compare."""
     ids, logits, hidden = drafter.draft(batch, k, want_logits=True, want_hidden=True,
                                         max_ctx=max(batch["ctx_lens_host"] + [1]))
@@ -71,7 +71,7 @@ def check_step(cfg, drafter, weights, batch, k, requests=None, dtype=np.float64,
     if "vocab_map" in weights:
         own = weights["vocab_map"].cpu().numpy()[own]
     np.testing.assert_array_equal(ids, own)
-    e_h = assert_close(hidden[requests], ref["hidden"], what + " hidden")
+    e_h = assert_close(hidden[requests], ref["hidden"], what + " hidden", tol)
     sure = ref["margin"] > MARGIN
     if "markov_in" in weights:
         # the correction at position i depends on the token chosen at i - 1: after a near-tie the two sides may
@@ -79,10 +79,10 @@ def check_step(cfg, drafter, weights, batch, k, requests=None, dtype=np.float64,
         chain_ok = np.ones_like(sure)
         chain_ok[:, 1:] = np.cumprod(sure[:, :-1], axis=1).astype(bool)
         assert sure.shape[1] == 1 or chain_ok[:, 1:].any(), what + ": no chained position is comparable"
-        e_l = assert_close(logits[requests][chain_ok], ref["logits"][chain_ok], what + " logits")
+        e_l = assert_close(logits[requests][chain_ok], ref["logits"][chain_ok], what + " logits", tol)
         sure &= chain_ok
     else:
-        e_l = assert_close(logits[requests], ref["logits"], what + " logits")
+        e_l = assert_close(logits[requests], ref["logits"], what + " logits", tol)
     assert np.array_equal(ids[requests][sure], ref["draft_ids"][sure]), what + " draft ids differ above the margin"
     return dict(err_hidden=e_h, err_logits=e_l, ids_compared=int(sure.sum()), ids_total=int(sure.size))
 

@@ -43,6 +43,26 @@ def test_mid_config_window_and_attentionless_layer():
     drafter.close()
 
 
+TOL_BF16 = 5e-2    # bf16 tensor-core operands: 8 significant bits on every GEMM input (fp16 mode: 11 bits, bar 2e-2)
+
+
+@pytest.mark.parametrize("over", [dict(), dict(markov_rank=64, V_draft=700), dict(window=256, has_attn=[1, 0], kv_slot=[1, -1])])
+def test_mid_config_bf16_operand_mode(over):
+    """act_bf16 = 1: the GEMMs run bf16 x bf16 on the caller's own matrices (borrowed, no library copy) and every
+    activation the library feeds to a GEMM is bf16.  Same step, same oracle; the bound is the looser one that 8-bit
+    operands allow, and the measured error is printed so the two modes can be compared."""
+    cfg = synth.derived(dict(MID, act_bf16=1, **over))
+    drafter, w, batch = cuda_setup(cfg, ctx_lens=[0, 1, 17, 1000, 2999], max_k=32)
+    r16 = check_step(cfg, drafter, w, batch, 16, what="mid bf16 operands", tol=TOL_BF16)
+    drafter.close()
+    cfg_h = synth.derived(dict(MID, **over))
+    d_h, _, _ = cuda_setup(cfg_h, ctx_lens=[0, 1, 17, 1000, 2999], max_k=32, weights=w)
+    rh = check_step(cfg_h, d_h, w, batch, 16, what="mid fp16 operands")
+    d_h.close()
+    print("bf16 operands:", r16, "fp16 operands:", rh)
+    assert r16["ids_compared"] > 0 and rh["err_logits"] <= r16["err_logits"] * 1.5
+
+
 def test_properties_bit_exact():
     cfg = synth.derived(dict(MID))
     drafter, w, batch = cuda_setup(cfg, ctx_lens=[33, 700, 16, 2100])
