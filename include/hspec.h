@@ -242,8 +242,12 @@ int hspec_op_lm_head_argmax(const void* x, const void* W, int32_t in_dtype, int3
  * a fixed array inside the library's device image: 8 MiB + 256 B on every GPU that loads the library, held until the
  * process exits.  Limits: M <= 512 rows, V <= 262144; larger sizes are rejected with HSPEC_ERR_BAD_SHAPE.
  * The call allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).  Its FIRST call on a device
- * resolves the array's device address (cudaGetSymbolAddress, with that device current); make that first call before
- * any stream capture begins.  All calls share the array: calls that overlap on the GPU (e.g. on two streams) race.
+ * resolves the array's device address (cudaGetSymbolAddress, with that device current) and, with CUDA's lazy module
+ * loading, is also the moment the driver places the array and the kernels' code in device memory: make that first
+ * call at start-up - before the host hands the remaining HBM to its pool, and before any stream capture begins; from
+ * the second call on, free device memory does not move (the test checks it).  All calls share the array: calls that
+ * overlap on the GPU (e.g. on two streams) race.  A bounded wait that gives up inside the call shows in
+ * hspec_op_device_status (the ids of such a call are 0x7fffffff).
  * Inputs and outputs are the caller's, as in hspec_op_lm_head_argmax; results are identical to it. */
 int hspec_op_lm_head_argmax_noalloc(const void* x, const void* W, int32_t in_dtype, int32_t* ids, float* logits, int32_t M,
                                     int32_t V, int32_t K, void* stream);

@@ -12,10 +12,15 @@
 //   warps 2..5  epilogue (both CTAs, their own 128 accumulator lanes)
 // No TMA load is multicast; the only cluster-wide signal is tcgen05.commit to both CTAs' barriers.
 //
+// A pipeline stage holds TWO 64-column k-steps (64 KB per CTA at 256-wide tiles, three stages): every barrier round of
+// the MMA thread (wait for "full", commit to "empty") costs the tensor pipe about 150 clocks whatever the order of the
+// operations, so it is paid once per eight MMAs instead of once per four.
+//
 // Measurement builds (HSPEC_NVCC_FLAGS): -DHSPEC_GEMM2_NOLOAD (no operand is fetched), -DHSPEC_GEMM2_NOEPI (accumulators
-// are not read out), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time).  On M = 2048, n_out = 25600,
-// K = 5120 the MMA issue alone (no loads, no read-out) takes 167 SM clocks per 256 x 256 x 16 instruction (76 % of 8192
-// flop per clock and SM), 182 clocks with loads and read-out (70 %); a library GEMM on the same shape runs at ~85 %.
+// are not read out), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time); HSPEC_GEMM2_KSUB=1 in the
+// environment goes back to one k-step per stage.  On M = 2048, n_out = 25600, K = 5120, SM clocks per 256 x 256 x 16
+// instruction (the arithmetic needs 128): MMA issue alone, no barrier at all 128; one k-step per stage 167 alone and
+// 182 with loads and read-out; two k-steps per stage 146 and 160.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -34,6 +39,7 @@ struct Gemm2Args {
   int M, N_out, K;
   int BNT;                 // activation rows per cluster tile (128 or 256); each CTA stages BNT/2
   int k_tiles, stages;
+  int ksub;                // 64-column k-steps per pipeline stage (1 or 2): one barrier round per stage
   int n_tiles_w, n_tiles_m;
   // Work units: the first n_full_tiles tiles run whole (full waves of the SM pairs); each of the remaining "tail" tiles
   // is cut into tail_splits K-slices so that the last, partly filled wave keeps every pair busy.  A slice stores an
@@ -121,7 +127,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const uint32_t b_bytes = uint32_t(g.BNT / 2) * TILE_K * 2;
-  const uint32_t stage_bytes = A_BYTES + b_bytes;
+  const uint32_t sub_bytes = A_BYTES + b_bytes;                    // one k-step: this CTA's weight rows + its half of the activations
+  const uint32_t stage_bytes = uint32_t(g.ksub) * sub_bytes;
   Tail2* tail = reinterpret_cast<Tail2*>(smem + size_t(g.stages) * stage_bytes);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -183,7 +190,7 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         int tile, sp, kt_begin, kt_end;
         decode(unit, tile, sp, kt_begin, kt_end);
         const int tn = tile / g.n_tiles_m, tm = tile % g.n_tiles_m;
-        for (int kt = kt_begin; kt < kt_end; ++kt, ++it) {
+        for (int kt = kt_begin; kt < kt_end; kt += g.ksub, ++it) {
           const int s = it % g.stages;
           const uint32_t lap = it / g.stages;
           if (lap > 0 && !mbar_wait(smem_u32(&tail->empty[s]), (lap - 1) & 1)) {
@@ -192,17 +199,20 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             ok = false;
             break;
           }
+          const int n_sub = min(g.ksub, kt_end - kt);
           const uint32_t full = smem_u32(&tail->full[s]);
 #ifdef HSPEC_GEMM2_NOLOAD
           // measurement build: no operand is fetched, the MMAs run on whatever the stage holds (results are garbage);
           // shows the rate of the MMA issue + epilogue alone
           if (rank == 0) mbar_arrive(full);
-          (void)pol_w; (void)pol_x; (void)tn; (void)tm;
+          (void)pol_w; (void)pol_x; (void)tn; (void)tm; (void)n_sub;
 #else
-          if (rank == 0) mbar_expect_tx(full, 2 * stage_bytes);       // both CTAs' bytes land on the leader's barrier
-          uint8_t* sa = smem + size_t(s) * stage_bytes;
-          tma_load_2d_pair(smem_u32(sa), &tmA, kt * TILE_K, tn * 256 + int(rank) * 128, full, pol_w);
-          tma_load_2d_pair(smem_u32(sa + A_BYTES), &tmB, kt * TILE_K, tm * g.BNT + int(rank) * (g.BNT / 2), full, pol_x);
+          if (rank == 0) mbar_expect_tx(full, 2 * uint32_t(n_sub) * sub_bytes);   // both CTAs' bytes land on the leader's barrier
+          for (int sub = 0; sub < n_sub; ++sub) {
+            uint8_t* sa = smem + size_t(s) * stage_bytes + size_t(sub) * sub_bytes;
+            tma_load_2d_pair(smem_u32(sa), &tmA, (kt + sub) * TILE_K, tn * 256 + int(rank) * 128, full, pol_w);
+            tma_load_2d_pair(smem_u32(sa + A_BYTES), &tmB, (kt + sub) * TILE_K, tm * g.BNT + int(rank) * (g.BNT / 2), full, pol_x);
+          }
 #endif
         }
       }
@@ -219,16 +229,21 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (use > 0 && !mbar_wait(smem_u32(&tail->tmem_empty[acc]), (use - 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const uint32_t tmem_acc = tmem_base + acc * uint32_t(g.BNT);
-        for (int kt = kt_begin; kt < kt_end; ++kt, ++it) {
+        for (int kt = kt_begin; kt < kt_end; kt += g.ksub, ++it) {
           const int s = it % g.stages;
           const uint32_t lap = it / g.stages;
+          // (every barrier round in this thread costs the tensor pipe ~150 clocks: with two k-steps per stage it is
+          // paid once per eight MMAs instead of once per four)
           if (!mbar_wait(smem_u32(&tail->full[s]), lap & 1)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes);
-          const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
+          const int n_sub = min(g.ksub, kt_end - kt);
+          for (int sub = 0; sub < n_sub; ++sub) {
+            const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes + size_t(sub) * sub_bytes);
+            const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
 #pragma unroll
-          for (int kk = 0; kk < TILE_K / 16; ++kk)
-            umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > kt_begin || kk > 0) ? 1u : 0u);
+            for (int kk = 0; kk < TILE_K / 16; ++kk)
+              umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > kt_begin || sub > 0 || kk > 0) ? 1u : 0u);
+          }
           umma_commit_pair(smem_u32(&tail->empty[s]));
         }
         if (ok) umma_commit_pair(smem_u32(&tail->tmem_full[acc]));
@@ -494,7 +509,9 @@ cudaError_t gemm2_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, s
   g.f16 = c.f16 ? 1 : 0; g.mode = c.mode; g.out = c.out; g.ldo = c.ldo;
   if (c.addend != nullptr) { if (err) *err = "the 2-SM kernel has no addend epilogue"; return cudaErrorInvalidValue; }
   g.logits = c.logits; g.part_val = c.part_val; g.part_idx = c.part_idx; g.status = c.status;
-  const size_t stage_bytes = A_BYTES + size_t(g.BNT / 2) * TILE_K * 2;
+  static const int ksub_env = [] { const char* e = getenv("HSPEC_GEMM2_KSUB"); return e ? atoi(e) : 0; }();   // measurements only
+  g.ksub = (ksub_env == 1 || ksub_env == 2) ? ksub_env : 2;
+  const size_t stage_bytes = size_t(g.ksub) * (A_BYTES + size_t(g.BNT / 2) * TILE_K * 2);
   const size_t fixed = sizeof(Tail2) + 1024;
   int stages = int((size_t(smem_optin2) - fixed) / stage_bytes);
   if (stages > GEMM_MAX_STAGES) stages = GEMM_MAX_STAGES;
