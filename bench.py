@@ -417,11 +417,16 @@ def summarize(res, peaks, traffic=None):
     hbm_time_ms = (a["weight_bytes"] + a["kv_bytes"]) / (hbm * 1e9) * 1e3
     tensor_time_ms = (a["gemm_flops"] + a["attn_flops"]) / (tf * 1e12) * 1e3
 
-    def group(prefix):
-        vs = [v for n, v in res["prof"].items() if n.startswith(prefix)]
-        t = sum(v["ms"] for v in vs) / steps
-        return dict(ms=t, flops=sum(v["flops"] for v in vs) / steps, bytes=sum(v["bytes"] for v in vs) / steps,
-                    io_bytes=sum(v["io_bytes"] for v in vs) / steps, launches=sum(v["n"] for v in vs) // steps)
+    def tensor_bound(v):
+        return v["flops"] / (tf * 1e12) >= v["bytes"] / (hbm * 1e9)
+
+    def group(prefix, want=None):
+        """Launches of one GEMM kernel (by profile-label prefix), all of them or only those on one side of the ridge."""
+        vs = {n: v for n, v in res["prof"].items() if n.startswith(prefix) and (want is None or tensor_bound(v) == want)}
+        t = sum(v["ms"] for v in vs.values()) / steps
+        return dict(ms=t, flops=sum(v["flops"] for v in vs.values()) / steps, bytes=sum(v["bytes"] for v in vs.values()) / steps,
+                    io_bytes=sum(v["io_bytes"] for v in vs.values()) / steps, launches=sum(v["n"] for v in vs.values()) // steps,
+                    labels=sorted(n.split(":", 1)[1] for n in vs))
     g1, g2 = group("gemm:"), group("gemm2:")          # one-CTA kernel (few rows), 2-CTA persistent kernel (many rows)
     gemm_ms, gemm_flops, gemm_bytes = g1["ms"] + g2["ms"], g1["flops"] + g2["flops"], g1["bytes"] + g2["bytes"]
     att = res["prof"].get("attn_partial")
@@ -441,16 +446,20 @@ def summarize(res, peaks, traffic=None):
         return round(t["ratio"] * algorithmic_bytes_per_launch), \
             f"{t['ratio']:.3f} x algorithmic bytes per launch (ncu dram__bytes_read+write on {t['case']})"
 
-    def gemm_roof(kernel, grp):
-        """Roofline of one GEMM kernel over its launches in a step: the bound is the roofline that takes longer."""
+    def gemm_roof(kernel, grp, is_tensor):
+        """Roofline of one GEMM kernel over those of its launches in a step that sit on one side of the ridge (a launch
+        is tensor-bound when its flops at the tensor peak take longer than its weight bytes at the HBM peak)."""
         if grp["ms"] <= 0:
             return None
         tfs, gbs = grp["flops"] / (grp["ms"] * 1e-3) / 1e12, grp["bytes"] / (grp["ms"] * 1e-3) / 1e9
-        tr, tr_note = dram_traffic(kernel, (grp["bytes"] + grp["io_bytes"]) / max(1, grp["launches"]))
-        base = dict(kernel=kernel, traffic=tr, traffic_note=tr_note, ms_per_step=round(grp["ms"], 4),
+        # (captures on record: the pair kernel on a tensor-bound case and on a streaming case, the one-CTA kernel streaming)
+        bound = "tensor" if is_tensor else "hbm"
+        key = kernel + ":" + bound if kernel + ":" + bound in traffic else kernel
+        tr, tr_note = dram_traffic(key, (grp["bytes"] + grp["io_bytes"]) / max(1, grp["launches"]))
+        base = dict(kernel=kernel, launches=grp["labels"], traffic=tr, traffic_note=tr_note, ms_per_step=round(grp["ms"], 4),
                     launches_per_step=grp["launches"],
                     algorithmic_bytes_per_launch=round((grp["bytes"] + grp["io_bytes"]) / max(1, grp["launches"])))
-        if grp["flops"] / (tf * 1e12) >= grp["bytes"] / (hbm * 1e9):
+        if is_tensor:
             r = dict(base, bound="tensor", achieved=round(tfs, 1), peak=tf, unit="TFLOP/s", frac=round(tfs / tf, 4),
                      note=f"sum over its launches per step: 2*M*N*K flops / CUDA-event time; peak = cuBLAS bf16 sustained, "
                           f"of {peaks['source']} (fp16 has the same nominal rate)")
@@ -464,7 +473,9 @@ def summarize(res, peaks, traffic=None):
         return dict(base, bound="hbm", achieved=round(gbs, 1), peak=hbm, unit="GB/s", frac=round(gbs / hbm, 4),
                     note=f"sum over its launches per step: weight bytes / CUDA-event time; peak = copy bandwidth, of "
                          f"{peaks['source']}")
-    roofs = [r for r in (gemm_roof("gemm_2sm_kernel", g2), gemm_roof("gemm_tcgen05_kernel", g1)) if r]
+    roofs = [r for r in (gemm_roof(kern, group(prefix, want), want)
+                         for kern, prefix in (("gemm_2sm_kernel", "gemm2:"), ("gemm_tcgen05_kernel", "gemm:"))
+                         for want in (True, False)) if r]
     if att_ms > 0:
         tr, tr_note = dram_traffic("attn_tc_kernel", a["kv_bytes"] / n_attn)
         roofs.append(dict(kernel="attn_tc_kernel", bound="hbm", achieved=round(att_gbs, 1), peak=hbm, unit="GB/s",
@@ -686,7 +697,7 @@ CASES = {
     "gemm": (case_gemm, {}),                                                       # the 2-SM kernel, M = 2048
     "gemm_skinny": (case_gemm, dict(M=32, n_out=65536, K=4096)),                   # weight streaming, Proj_dS class
     "gemm_skinny64": (case_gemm, dict(M=64, n_out=262144, K=5120)),                # Proj_dS at concurrency 64 (a fifth of it)
-    "gemm_skinny128": (case_gemm, dict(M=128, n_out=262144, K=5120)),              # Proj_dS at concurrency 128 (a fifth of it)
+    "gemm_skinny128": (case_gemm, dict(M=128, n_out=262144, K=5120)),              # Proj_dS at concurrency 128 (a fifth of it; the 2-SM kernel)
     "scan": (case_scan, {}),
     "overlap": (case_overlap, {}),
 }

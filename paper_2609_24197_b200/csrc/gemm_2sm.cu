@@ -183,7 +183,8 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
       // short isolated runs, but ncu showed 2.4x the algorithmic DRAM reads (the clusters that share a weight tile
       // drift apart and fetch it again), and in a long power-capped step the extra DRAM traffic costs clock:
       // 13.5 vs 13.75 ms per step at conc128_32b.
-      const uint64_t pol_w = policy_evict_normal(), pol_x = policy_evict_last();
+      // (With a single activation tile nobody shares a weight tile: the weights stream through once, evict-first.)
+      const uint64_t pol_w = g.n_tiles_m == 1 ? policy_evict_first() : policy_evict_normal(), pol_x = policy_evict_last();
       uint32_t it = 0;
       bool ok = true;
       for (int unit = cluster_id; unit < total_units && ok; unit += n_clusters) {
@@ -435,10 +436,14 @@ int g_smem_optin2[MAX_DEVICES] = {};
 
 bool gemm2_preferred(int M, int n_out) {
   static const bool off = [] { const char* e = getenv("HSPEC_GEMM_1SM"); return e && e[0] == '1'; }();
-  // from 256 rows on the contractions are tensor-bound; even a partly filled wave of pair tiles beats the one-CTA
-  // kernel with K-slices and its reduction pass
-  (void)n_out;
-  return !off && M >= 256;
+  static const int min_m = [] { const char* e = getenv("HSPEC_GEMM2_MIN_M"); return e ? atoi(e) : 0; }();   // measurements only
+  if (off) return false;
+  if (min_m > 0) return M >= min_m;
+  // From 256 rows on the contractions are tensor-bound; even a partly filled wave of pair tiles beats the one-CTA
+  // kernel with K-slices and its reduction pass.  At 128..255 rows only a matrix of 2^18 weight rows or more (the
+  // state projection) goes this way: streaming it, the pair kernel measured 5.65 against 5.51 TB/s at 128 rows (at 64
+  // rows the one-CTA kernel wins, 6.24 against 6.01), and the step's small matrices keep the kernel they are tuned for.
+  return M >= 256 || (M >= 128 && n_out >= (1 << 18));
 }
 
 // Tile width (activation rows per pair tile) and the number of K-slices for the tiles of the last, partly filled wave,

@@ -74,6 +74,20 @@ def test_gemm(hs, M, n_out, K, mode):
     assert_close(y.float().cpu().numpy(), ref, f"gemm {M}x{n_out}x{K} {mode}", tol=2e-2 if mode == "bf16" else 3e-3 if mode == "f16_out" else 1e-4)   # bf16 output: 2^-9 of the largest element
 
 
+@pytest.mark.parametrize("M,mode", [(128, "f16_out"), (200, "f32")])
+def test_gemm_quarter_million_weight_rows_at_128_rows_takes_the_pair_kernel(hs, M, mode):
+    """The state projection's class: a weight matrix of over 2^18 rows met by 128..255 activation rows streams through
+    the 2-SM kernel (one or two activation tiles, K ragged against its two-k-step stages, a ragged last weight tile)."""
+    n_out, K = (1 << 18) + 300, 448
+    x, W = _randn((M, K), 21, 1.0, torch.float16), _randn((n_out, K), 22, 0.05, torch.float16)
+    ref = O.gemm(x.double().cpu().numpy(), W.double().cpu().numpy())
+    ws = torch.empty(hs.hspec_gemm_workspace_bytes(M, n_out, K), dtype=torch.uint8, device="cuda")
+    y = torch.full((M, n_out), float("nan"), dtype=torch.float16 if mode == "f16_out" else torch.float32, device="cuda")
+    hs.hspec_op_gemm(x, W, y, workspace=ws)
+    torch.cuda.synchronize()
+    assert_close(y.float().cpu().numpy(), ref, f"gemm {M}x{n_out}x{K} {mode}", tol=3e-3 if mode == "f16_out" else 1e-4)
+
+
 def test_gemm_strided_output_and_exact_small_integers(hs):
     # integer-valued operands: fp32 accumulation is exact, so the result must be bit-exact
     M, n_out, K = 20, 260, 192
