@@ -306,7 +306,8 @@ int attn_pick_chunk(int B, int Hkv, int max_ctx, int window, int num_sms) {
   if (chunk < 256) chunk = 256;
   // long chunks mean fewer partials to write and merge; they need enough (request, head) pairs to keep every SM's
   // share of the work list even
-  const int cap = (B * Hkv >= 4 * num_sms) ? 8192 : 4096;
+  static const int cap_env = [] { const char* e = getenv("HSPEC_ATTN_CHUNK_CAP"); return e ? atoi(e) : 0; }();   // measurements only
+  const int cap = cap_env >= 256 ? cap_env : (B * Hkv >= 4 * num_sms) ? 8192 : 4096;
   if (chunk > cap) chunk = cap;
   return chunk;
 }

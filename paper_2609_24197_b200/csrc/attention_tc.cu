@@ -17,15 +17,18 @@
 //               maxima through shared memory.  Each reads its S half-row, masks by selection, keeps a
 //               reference maximum that only moves when the row maximum outgrows it by 2^8 (then, rarely, rescales
 //               its O row in TMEM), and writes P (bf16, two keys per 32-bit column) over the first half of the S
-//               buffer it came from.  At the end of an item they put the next item's Q tile into shared memory
-//               first (the tensor core starts on its scores), then read O out: as a finished fp16 row when the
-//               request has a single chunk, else as an fp32 partial for the merge kernel.
+//               buffer it came from.  During an item's last tile they copy the next item's Q tile into shared
+//               memory (cp.async, no registers); at its end they read O out: as a finished fp16 row when the request
+//               has a single chunk, else as an fp32 partial for the merge kernel.
 //
-// The MMA warp issues S_{t+1} and S_{t+2} before it waits for P_t (O and three score buffers fill the 512 TMEM
-// columns): the softmax warps always find the next tile's scores waiting, and the time the issuing thread spends on a
-// score product (barrier round included) is off the P_t -> P V -> S -> softmax chain.  Measured against two buffers
-// and one tile of lookahead: 3 % less time on every shape.  Every wait is bounded; a timed-out role sets a status word
-// and the CTA unwinds.
+// The MMA warp keeps the scores two tiles ahead of the softmax warps (O and three score buffers fill the 512 TMEM
+// columns): S_{t+1} and S_{t+2} are issued before it waits for P_t, so the softmax warps always find the next tile's
+// scores waiting and the issuing thread's time on a score product is off the P_t -> P V -> S -> softmax chain (-3 %
+// against two buffers).  The lookahead crosses item boundaries: the softmax warps copy the next item's Q tile into
+// shared memory while they work on the current item's last tile - every product that reads the old Q has finished by
+// then - so the next item's first scores are computed during the current item's last P V product and read-out
+// (another -3 % at 32B-class shapes, -5..8 % where the items are short).  Every wait is bounded; a timed-out role sets
+// a status word and the CTA unwinds.
 #include "common.cuh"
 #include "kernels.h"
 
@@ -414,12 +417,36 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #else
 #define MCLK(i)
 #endif
-      // S = Q K^T of tile g_t into S buffer g_t % NSB.  The buffer last held P of tile g_t - NSB, whose P V product this
+      // Two cursors walk this CTA's tiles in the same order.  The P V cursor (item n, global tile gt) follows the softmax
+      // warps.  The score cursor (item n_s, tile t_s of T_s, global tile gts) runs up to two tiles ahead of it, ACROSS
+      // item boundaries: the softmax warps put the next item's Q tile in place while they work on this item's last tile
+      // (every score product of the item has finished by then), so the next item's first scores are computed while this
+      // item's last P V product and its read-out are still under way.
+      // S = Q K^T of tile gts into S buffer gts % NSB.  The buffer last held P of tile gts - NSB, whose P V product this
       // thread issued earlier; the tensor pipe runs one thread's MMAs in issue order.
-      auto issue_s = [&](uint32_t g_t) -> bool {
-        const int s = g_t % NSK;
+      uint32_t gts = 0, n_s = 0;
+      int t_s = 0;
+      int4 ws_next = items[item_at(0)];
+      bool s_valid = true;
+      int T_s;
+      {
+        const Item w0 = unpack_item(ws_next);
+        T_s = make_range(w0.ctx, a.window, a.chunk, w0.c, a.k).T;
+        if (item_at(1) < n_items) ws_next = items[item_at(1)];
+      }
+      // returns 1 = issued, 0 = the item's Q tile is not there yet (only when it may come back later), -1 = timed out
+      auto issue_s = [&](bool must) -> int {
+        if (t_s == 0) {
+          const uint32_t qb = smem_u32(&bars->q_ready);
+          MCLK(0)
+          if (must) { if (!mbar_wait(qb, n_s & 1)) return -1; }
+          else if (!mbar_test(qb, n_s & 1)) return 0;
+          MCLK(4)
+          tc_fence_after();
+        }
+        const int s = gts % NSK;
         MCLK(0)
-        if (!mbar_wait(smem_u32(&bars->k_full[s]), (g_t / NSK) & 1)) return false;
+        if (!mbar_wait(smem_u32(&bars->k_full[s]), (gts / NSK) & 1)) return -1;
         MCLK(1)
         tc_fence_after();
         const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
@@ -427,27 +454,37 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         for (int ks = 0; ks < DH / 16; ++ks) {
           const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
           const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
-          umma_bf16(tmem_s0 + (g_t % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
+          umma_bf16(tmem_s0 + (gts % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
         }
         umma_commit(smem_u32(&bars->k_empty[s]));
-        umma_commit(smem_u32(&bars->s_ready[g_t % NSB]));
-        return true;
+        umma_commit(smem_u32(&bars->s_ready[gts % NSB]));
+        ++gts;
+        if (++t_s == T_s) {                            // on to the next item (its descriptor was fetched an item ago)
+          t_s = 0;
+          ++n_s;
+          if (item_at(int(n_s)) < n_items) {
+            const Item wn = unpack_item(ws_next);
+            T_s = make_range(wn.ctx, a.window, a.chunk, wn.c, a.k).T;
+            if (item_at(int(n_s) + 1) < n_items) ws_next = items[item_at(int(n_s) + 1)];
+          } else {
+            s_valid = false;
+          }
+        }
+        return 1;
       };
       int4 w_next = items[item_at(0)];
       for (; item_at(int(n)) < n_items && ok; ++n) {
         const Item wi = unpack_item(w_next);
         if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
         const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
-        MCLK(0)
-        if (!mbar_wait(smem_u32(&bars->q_ready), n & 1)) { ok = false; break; }      // this item's Q tile is in place
-        MCLK(4)
-        tc_fence_after();
-        ok = issue_s(gt);
-        if (ok && g.T > 1) ok = issue_s(gt + 1);
         for (int t = 0; t < g.T && ok; ++t, ++gt) {
-          // the scores run two tiles ahead of the softmax warps: by the time they have turned tile t into P, the
-          // scores of tile t + 1 have long been there, and this thread's issue time is off their critical path
-          if (t + 2 < g.T) ok = issue_s(gt + 2);
+          // the scores of this tile must be under way (the softmax warps wait for them); the next two are issued as soon
+          // as their K tile and, at an item's first tile, its Q tile are there
+          while (ok && s_valid && gts <= gt + 2) {
+            const int r = issue_s(gts <= gt);
+            if (r < 0) ok = false;
+            if (r <= 0) break;
+          }
           if (!ok) break;
           const int s = gt % NSV;
           MCLK(0)
@@ -510,17 +547,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       const __nv_bfloat16* src = q_half(wi, row_ok);
       if (row_ok) asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
     };
-    auto load_q = [&](const Item& wi, uint4 (&qv)[8]) {
+    // Q tile -> shared memory in the swizzled K-major operand layout (zeros for padding rows), by 16-byte asynchronous
+    // copies that need no registers: they are issued once the item's last score product has finished and are waited
+    // for after the thread has dealt with that tile.
+    auto q_copy_issue = [&](const Item& wi) {
       bool row_ok;
       const __nv_bfloat16* src = q_half(wi, row_ok);
 #pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8)
-        qv[c8] = row_ok ? __ldg(reinterpret_cast<const uint4*>(src + c8 * 8)) : make_uint4(0, 0, 0, 0);
+      for (int c8 = 0; c8 < 8; ++c8) cp_async16(smem_u32(sQ + tile_off<KV_HALF>(r_local, hf * 8 + c8)), src + c8 * 8, row_ok);
+      cp_async_commit();
     };
-    // Q tile -> shared memory in the swizzled K-major operand layout (zeros for padding rows)
-    auto store_q = [&](const uint4 (&qv)[8]) {
-#pragma unroll
-      for (int c8 = 0; c8 < 8; ++c8) *reinterpret_cast<uint4*>(sQ + tile_off<KV_HALF>(r_local, hf * 8 + c8)) = qv[c8];
+    auto q_copy_finish = [&]() {
+      cp_async_wait<0>();
       fence_proxy_async();
       tc_fence_before();
       __syncwarp();
@@ -528,11 +566,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     };
     int4 w_cur = items[item_at(0)];
     int4 w_next = (item_at(1) < n_items) ? items[item_at(1)] : w_cur;
-    {
-      uint4 qv[8];
-      load_q(unpack_item(w_cur), qv);
-      store_q(qv);
-    }
+    q_copy_issue(unpack_item(w_cur));
+    q_copy_finish();
     for (; item_at(int(n)) < n_items && ok; ++n) {
       const Item wi = unpack_item(w_cur);
       const int b = wi.b, kvh = wi.kvh, c = wi.c, ctx = wi.ctx;
@@ -552,6 +587,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
       for (int t = 0; t < g.T && ok; ++t, ++gt) {
         const uint32_t t_s = tmem_s0 + (gt % NSB) * 128 + lane_base;
         if (!mbar_wait(smem_u32(&bars->s_ready[gt % NSB]), (gt / NSB) & 1)) { ok = false; break; }
+        // The scores of the item's last tile are there: every product that reads this item's Q tile has finished, and
+        // the next item's Q goes in now, so that the tensor core can start on its scores before this item is done.
+        const bool q_now = has_next && t == g.T - 1;
+        if (q_now) q_copy_issue(unpack_item(w_next));
         if (!warp_live) {
           // The scores run up to two tiles ahead, and the exchange barrier has two slots: this warp must not arrive for
           // tile t + 2 on the slot the live warps still use for tile t, so it waits for the exchange like they do.
@@ -559,6 +598,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
             mbar_arrive(smem_u32(&bars->x_ready[gt & 1]));
             mbar_arrive(smem_u32(&bars->p_ready[gt % NSB]));
           }
+          if (q_now) q_copy_finish();
           if (!mbar_wait(smem_u32(&bars->x_ready[gt & 1]), (gt >> 1) & 1)) { ok = false; break; }
           continue;
         }
@@ -649,27 +689,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&bars->p_ready[gt % NSB]));   // one arrival per warp, after all its lanes' stores
+        if (q_now) q_copy_finish();
         TCLK(5)
       }
       if (!ok) break;
-      // ---- the row sum is the sum of the two halves: the threads of a row swap theirs.
-      // The exchange buffer of parity gt & 1 was last used two tiles ago, and a thread's slot is not written again
-      // before every softmax warp has signalled q_ready for the next item, i.e. after the partner's read.
+      // ---- the row sum is the sum of the two halves: the threads of a row swap theirs through the exchange buffer of
+      // parity gt & 1, last used two tiles ago.  The next tile (the next item's first) writes the same slots, so a second
+      // round of the barrier keeps every thread from going on before its partner has read.
       bars->xmax[gt & 1][hf][r_local] = l_sum;
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->l_ready));
-      if (!mbar_wait(smem_u32(&bars->l_ready), n & 1)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&bars->l_ready), 0)) { ok = false; break; }
       const float l_row = l_sum + bars->xmax[gt & 1][hf ^ 1][r_local];
-      {
-        // every MMA of the item has finished (so has every read of Q): the next item's Q goes in at once and the
-        // tensor core starts on its scores during the read-out
-        uint4 qv[8];
-        if (has_next) load_q(unpack_item(w_next), qv);
-        if (!mbar_wait(smem_u32(&bars->o_done), n & 1) || *abort_flag) { ok = false; break; }
-        tc_fence_after();
-        TCLK(6)
-        if (has_next) store_q(qv);
-      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->l_ready));
+      if (!mbar_wait(smem_u32(&bars->l_ready), 1)) { ok = false; break; }
+      // every MMA of the item has finished once o_done completes
+      if (!mbar_wait(smem_u32(&bars->o_done), n & 1) || *abort_flag) { ok = false; break; }
+      tc_fence_after();
+      TCLK(6)
       const size_t slab = (size_t(b) * a.Hkv + kvh) * a.max_chunks + c;
       const bool whole = g.n_chunks == 1;            // the request's only chunk: normalise and finish here
       if (!warp_live) {
