@@ -343,7 +343,7 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
 
 // Persistent: one CTA per SM walks the work list (items item_at(0), item_at(1), ...).  All ring and buffer indices
 // count tiles across items (gt): K slot = gt % NSK, V slot = gt % NSV, S / P buffer = gt % NSB.
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(384, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a,
                const int* __restrict__ count, const int4* __restrict__ items) {
   pdl_wait();
@@ -403,8 +403,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     produce_operand(a, is_v ? &tmV : &tmK, is_v ? a.v_pool : a.k_pool, is_v ? a.vb : a.kb, sKV + (is_v ? NSK * KV_BYTES : 0),
                     is_v ? bars->v_full : bars->k_full, is_v ? bars->v_empty : bars->k_empty, abort_flag, items, n_items, lane,
                     is_v ? NSV : NSK);
-  } else if (warp == 9) {
-    // ================================================================= MMA issuer
+  } else if (warp == 9 || warp == 11) {
+    // ================================================================= MMA issuers: warp 9 the scores, warp 11 the P V products
+    // Two threads, because an issuing thread is held while the tensor pipe's queue is full: with one thread, a P that
+    // became ready while the scores two tiles ahead were being issued waited behind them, and the scores waited behind
+    // every P.  The pipe runs one thread's MMAs in issue order but not two threads', so the score thread waits for the
+    // COMPLETION of the P V product that last read the buffer it is about to overwrite (the barrier that frees that
+    // tile's V slot: same index, same phase, since both rings have three slots).
+    static_assert(NSB == NSV, "the score thread reuses the V ring's release barriers");
     if (lane == 0) {
       // fp32 accumulate, bf16 x bf16, M = 128, N = 128; scores: A = Q, B = K tile, both K-major in shared memory;
       // P V: A = P from tensor memory, B = V tile (MN-major)
@@ -417,106 +423,76 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #else
 #define MCLK(i)
 #endif
-      // Two cursors walk this CTA's tiles in the same order.  The P V cursor (item n, global tile gt) follows the softmax
-      // warps.  The score cursor (item n_s, tile t_s of T_s, global tile gts) runs up to two tiles ahead of it, ACROSS
-      // item boundaries: the softmax warps put the next item's Q tile in place while they work on this item's last tile
-      // (every score product of the item has finished by then), so the next item's first scores are computed while this
-      // item's last P V product and its read-out are still under way.
-      // S = Q K^T of tile gts into S buffer gts % NSB.  The buffer last held P of tile gts - NSB, whose P V product this
-      // thread issued earlier; the tensor pipe runs one thread's MMAs in issue order.
-      uint32_t gts = 0, n_s = 0;
-      int t_s = 0;
-      int4 ws_next = items[item_at(0)];
-      bool s_valid = true;
-      int T_s;
-      {
-        const Item w0 = unpack_item(ws_next);
-        T_s = make_range(w0.ctx, a.window, a.chunk, w0.c, a.k).T;
-        if (item_at(1) < n_items) ws_next = items[item_at(1)];
-      }
-      // returns 1 = issued, 0 = the item's Q tile is not there yet (only when it may come back later), -1 = timed out
-      auto issue_s = [&](bool must) -> int {
-        if (t_s == 0) {
-          const uint32_t qb = smem_u32(&bars->q_ready);
-          MCLK(0)
-          if (must) { if (!mbar_wait(qb, n_s & 1)) return -1; }
-          else if (!mbar_test(qb, n_s & 1)) return 0;
-          MCLK(4)
-          tc_fence_after();
-        }
-        const int s = gts % NSK;
-        MCLK(0)
-        if (!mbar_wait(smem_u32(&bars->k_full[s]), (gts / NSK) & 1)) return -1;
-        MCLK(1)
-        tc_fence_after();
-        const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
-          const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
-          umma_bf16(tmem_s0 + (gts % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
-        }
-        umma_commit(smem_u32(&bars->k_empty[s]));
-        umma_commit(smem_u32(&bars->s_ready[gts % NSB]));
-        ++gts;
-        if (++t_s == T_s) {                            // on to the next item (its descriptor was fetched an item ago)
-          t_s = 0;
-          ++n_s;
-          if (item_at(int(n_s)) < n_items) {
-            const Item wn = unpack_item(ws_next);
-            T_s = make_range(wn.ctx, a.window, a.chunk, wn.c, a.k).T;
-            if (item_at(int(n_s) + 1) < n_items) ws_next = items[item_at(int(n_s) + 1)];
-          } else {
-            s_valid = false;
-          }
-        }
-        return 1;
-      };
       int4 w_next = items[item_at(0)];
-      for (; item_at(int(n)) < n_items && ok; ++n) {
-        const Item wi = unpack_item(w_next);
-        if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
-        const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
-        for (int t = 0; t < g.T && ok; ++t, ++gt) {
-          // the scores of this tile must be under way (the softmax warps wait for them); the next two are issued as soon
-          // as their K tile and, at an item's first tile, its Q tile are there
-          while (ok && s_valid && gts <= gt + 2) {
-            const int r = issue_s(gts <= gt);
-            if (r < 0) ok = false;
-            if (r <= 0) break;
-          }
-          if (!ok) break;
-          const int s = gt % NSV;
+      if (warp == 9) {
+        // S = Q K^T of tile gt into S buffer gt % NSB, as far ahead of the softmax warps as the three buffers, the K
+        // ring and the Q tile allow; this runs across item boundaries (the softmax warps put the next item's Q tile in
+        // place while they work on this item's last tile: every score product of the item has finished by then).
+        for (; item_at(int(n)) < n_items && ok; ++n) {
+          const Item wi = unpack_item(w_next);
+          if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
+          const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
           MCLK(0)
-          if (!mbar_wait(smem_u32(&bars->p_ready[gt % NSB]), (gt / NSB) & 1)) { ok = false; break; }
-          MCLK(2)
-          if (!mbar_wait(smem_u32(&bars->v_full[s]), (gt / NSV) & 1)) { ok = false; break; }
-          MCLK(3)
-          // the first P V product of an item overwrites O: the previous item's accumulator must have been read out
-          if (t == 0 && n > 0 && !mbar_wait(smem_u32(&bars->o_free), (n - 1) & 1)) { ok = false; break; }
-          MCLK(5)
-          tc_fence_after();
-          const uint32_t vbase = smem_u32(sKV + (NSK + s) * KV_BYTES);
+          if (!mbar_wait(smem_u32(&bars->q_ready), n & 1)) { ok = false; break; }      // this item's Q tile is in place
+          MCLK(4)
+          for (int t = 0; t < g.T && ok; ++t, ++gt) {
+            const int s = gt % NSK;
+            MCLK(0)
+            if (!mbar_wait(smem_u32(&bars->k_full[s]), (gt / NSK) & 1)) { ok = false; break; }
+            MCLK(1)
+            // the buffer last held P of tile gt - NSB: its P V product must be complete
+            if (gt >= uint32_t(NSB) && !mbar_wait(smem_u32(&bars->v_empty[gt % NSV]), ((gt / NSV) - 1) & 1)) { ok = false; break; }
+            MCLK(2)
+            tc_fence_after();
+            const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
 #pragma unroll
-          for (int ks = 0; ks < KT / 16; ++ks) {
-            // A = 16 keys of P = 8 TMEM columns; B = the same 16 keys (rows) of V
-            const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
-            umma_bf16_ts(tmem_o, tmem_s0 + (gt % NSB) * 128 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+            for (int ks = 0; ks < DH / 16; ++ks) {
+              const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+              const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+              umma_bf16(tmem_s0 + (gt % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bars->k_empty[s]));
+            umma_commit(smem_u32(&bars->s_ready[gt % NSB]));
           }
-          umma_commit(smem_u32(&bars->v_empty[s]));
         }
-        if (ok) umma_commit(smem_u32(&bars->o_done));
+      } else {
+        for (; item_at(int(n)) < n_items && ok; ++n) {
+          const Item wi = unpack_item(w_next);
+          if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
+          const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
+          for (int t = 0; t < g.T && ok; ++t, ++gt) {
+            const int s = gt % NSV;
+            MCLK(0)
+            if (!mbar_wait(smem_u32(&bars->p_ready[gt % NSB]), (gt / NSB) & 1)) { ok = false; break; }
+            MCLK(2)
+            if (!mbar_wait(smem_u32(&bars->v_full[s]), (gt / NSV) & 1)) { ok = false; break; }
+            MCLK(3)
+            // the first P V product of an item overwrites O: the previous item's accumulator must have been read out
+            if (t == 0 && n > 0 && !mbar_wait(smem_u32(&bars->o_free), (n - 1) & 1)) { ok = false; break; }
+            MCLK(5)
+            tc_fence_after();
+            const uint32_t vbase = smem_u32(sKV + (NSK + s) * KV_BYTES);
+#pragma unroll
+            for (int ks = 0; ks < KT / 16; ++ks) {
+              // A = 16 keys of P = 8 TMEM columns; B = the same 16 keys (rows) of V
+              const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
+              umma_bf16_ts(tmem_o, tmem_s0 + (gt % NSB) * 128 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bars->v_empty[s]));
+          }
+          if (ok) umma_commit(smem_u32(&bars->o_done));
+        }
       }
 #ifdef HSPEC_ATTN_TIMING
       MCLK(0)
       if (blockIdx.x == 0 || blockIdx.x == 147)
-        printf("cta %d mma: total %lld | issue %lld wait_k %lld wait_p %lld wait_v %lld wait_q %lld wait_ofree %lld\n",
-               blockIdx.x, clock64() - m_start, mk[0], mk[1], mk[2], mk[3], mk[4], mk[5]);
+        printf("cta %d mma warp %d: total %lld | issue %lld wait_k %lld wait_p_or_buffer %lld wait_v %lld wait_q %lld wait_ofree %lld\n",
+               blockIdx.x, warp, clock64() - m_start, mk[0], mk[1], mk[2], mk[3], mk[4], mk[5]);
 #endif
       if (!ok) {
         atomicExch(a.status, STATUS_TIMEOUT_MMA);
         *abort_flag = 1;
-        mbar_arrive(smem_u32(&bars->o_done));
+        if (warp == 11) mbar_arrive(smem_u32(&bars->o_done));
       }
     }
   } else {
@@ -740,7 +716,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           }
         }
       } else {
-        float* dst = a.ws_o + (slab * a.R + (row_ok ? rg : 0)) * DH + hf * 64;
+        // partial layout [slab][group of 4 head-dim columns][row][4]: a thread owns a row, so for one column group the
+        // 32 lanes of a warp write 32 consecutive rows = 512 contiguous bytes (row-major partials would scatter every
+        // 16-byte store of a warp over 32 lines, and the item's read-out took 4 000 clocks of the load/store unit)
+        float* dst = a.ws_o + slab * a.R * DH + size_t(row_ok ? rg : 0) * 4;
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
           uint32_t o[32];
@@ -749,7 +728,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
           if (row_ok) {
 #pragma unroll
             for (int e = 0; e < 32; e += 4)
-              *reinterpret_cast<uint4*>(dst + j * 32 + e) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
+              *reinterpret_cast<uint4*>(dst + size_t(hf * 16 + j * 8 + e / 4) * a.R * 4) = make_uint4(o[e], o[e + 1], o[e + 2], o[e + 3]);
           }
         }
       }
@@ -781,44 +760,73 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
   }
 }
 
-// One block per (row of the block, query head): merge the chunk partials in chunk order (page-aligned chunk geometry).
-__global__ void attn_tc_merge_kernel(AttnTcArgs a, uint16_t* __restrict__ o, int n_pairs) {
+// Merges the chunk partials in chunk order (page-aligned chunk geometry).  One block per (request, KV head, group of
+// 32 of its k * rep rows): lane = row, warp w = head-dim columns [16 w, 16 w + 16), so the loads follow the partials'
+// [column group][row][4] layout (512 contiguous bytes per warp) and the finished rows go through shared memory to leave
+// as whole 256-byte rows.
+constexpr int MERGE_ROW_BYTES = DH * 2 + 16;         // padded: the 32 lanes' 16-byte writes spread over the banks
+__global__ void __launch_bounds__(256)
+attn_tc_merge_kernel(AttnTcArgs a, uint16_t* __restrict__ o) {
   pdl_wait();
   pdl_trigger();
-  // one warp per (row, head): each lane merges four adjacent head-dim columns with 16-byte loads
-  const int pair = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (pair >= n_pairs) return;
-  const int m = pair / a.Hq, hq = pair % a.Hq;
-  const int b = m / a.k, i = m % a.k;
-  const int kvh = hq / a.rep, r = i * a.rep + hq % a.rep;
+  __shared__ __align__(16) uint8_t tile[32 * MERGE_ROW_BYTES];
+  const int groups = (a.R + 31) / 32;
+  const int b = blockIdx.x / (a.Hkv * groups), kvh = (blockIdx.x / groups) % a.Hkv, r0 = (blockIdx.x % groups) * 32;
   const Range g = make_range(clamped_ctx(a, b), a.window, a.chunk, 0, a.k);
-  if (g.n_chunks == 1) return;                     // finished by the attention kernel itself
+  if (g.n_chunks == 1) return;                     // finished by the attention kernel itself (uniform for the block)
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int r = r0 + lane;
+  const bool row_ok = r < a.R;
   const size_t slab0 = (size_t(b) * a.Hkv + kvh) * a.max_chunks;
-  float m_tot = -INFINITY;
-  for (int c = 0; c < g.n_chunks; ++c) m_tot = fmaxf(m_tot, a.ws_ml[((slab0 + c) * a.R + r) * 2]);
-  const float ref = (m_tot == -INFINITY) ? 0.f : m_tot;
-  const int d4 = threadIdx.x & 31;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float L = 0.f;
-  for (int c = 0; c < g.n_chunks; ++c) {
-    const float* ml = a.ws_ml + ((slab0 + c) * a.R + r) * 2;
-    const float w = exp2f(ml[0] - ref);
-    L += ml[1] * w;
-    const float4 v = reinterpret_cast<const float4*>(a.ws_o + ((slab0 + c) * a.R + r) * DH)[d4];
-    acc.x += v.x * w; acc.y += v.y * w; acc.z += v.z * w; acc.w += v.w * w;
+  if (row_ok) {
+    float m_tot = -INFINITY;
+    for (int c = 0; c < g.n_chunks; ++c) m_tot = fmaxf(m_tot, a.ws_ml[((slab0 + c) * a.R + r) * 2]);
+    const float ref = (m_tot == -INFINITY) ? 0.f : m_tot;
+    float4 acc[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float L = 0.f;
+    for (int c = 0; c < g.n_chunks; ++c) {
+      const float* ml = a.ws_ml + ((slab0 + c) * a.R + r) * 2;
+      const float wgt = exp2f(ml[0] - ref);
+      L += ml[1] * wgt;
+      const float* src = a.ws_o + (slab0 + c) * a.R * DH + size_t(r) * 4;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(src + size_t(w * 4 + q) * a.R * 4);
+        acc[q].x += v.x * wgt; acc[q].y += v.y * wgt; acc[q].z += v.z * wgt; acc[q].w += v.w * wgt;
+      }
+    }
+    const float inv = 1.f / L;
+    uint32_t h[8];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (a.o_bf16) {
+        h[2 * q] = pack_bf16(acc[q].x * inv, acc[q].y * inv);
+        h[2 * q + 1] = pack_bf16(acc[q].z * inv, acc[q].w * inv);
+      } else {
+        const __half2 lo = __halves2half2(f16_sat(acc[q].x * inv, a.status), f16_sat(acc[q].y * inv, a.status));
+        const __half2 hi = __halves2half2(f16_sat(acc[q].z * inv, a.status), f16_sat(acc[q].w * inv, a.status));
+        h[2 * q] = *reinterpret_cast<const uint32_t*>(&lo);
+        h[2 * q + 1] = *reinterpret_cast<const uint32_t*>(&hi);
+      }
+    }
+    uint4* dst = reinterpret_cast<uint4*>(tile + lane * MERGE_ROW_BYTES + w * 32);
+    dst[0] = make_uint4(h[0], h[1], h[2], h[3]);
+    dst[1] = make_uint4(h[4], h[5], h[6], h[7]);
   }
-  const float inv = 1.f / L;
-  uint2 out;
-  if (a.o_bf16) {
-    out.x = pack_bf16(acc.x * inv, acc.y * inv);
-    out.y = pack_bf16(acc.z * inv, acc.w * inv);
-  } else {
-    const __half2 lo = __halves2half2(f16_sat(acc.x * inv, a.status), f16_sat(acc.y * inv, a.status));
-    const __half2 hi = __halves2half2(f16_sat(acc.z * inv, a.status), f16_sat(acc.w * inv, a.status));
-    out.x = *reinterpret_cast<const uint32_t*>(&lo);
-    out.y = *reinterpret_cast<const uint32_t*>(&hi);
+  __syncthreads();
+  // 16 lanes write one 256-byte row: row rr of the group is block position rr / rep, query head kvh * rep + rr % rep
+#pragma unroll
+  for (int p = 0; p < 2; ++p) {
+    const int rl = w * 4 + p * 2 + (lane >> 4);
+    const int rr = r0 + rl;
+    if (rr < a.R) {
+      const int i = rr / a.rep, hq = kvh * a.rep + rr % a.rep;
+      const uint4 v = *reinterpret_cast<const uint4*>(tile + rl * MERGE_ROW_BYTES + (lane & 15) * 16);
+      *reinterpret_cast<uint4*>(o + ((size_t(b) * a.k + i) * a.Hq + hq) * DH + (lane & 15) * 8) = v;
+    }
   }
-  reinterpret_cast<uint2*>(o + (size_t(m) * a.Hq + hq) * DH)[d4] = out;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -897,13 +905,12 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   trk_begin(trk, "attn_partial");
-  launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(352), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
+  launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(384), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
   trk_end(trk);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int n_pairs = c.B * c.k * c.Hq;
   trk_begin(trk, "attn_merge");
-  launch_pdl(attn_tc_merge_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, a, reinterpret_cast<uint16_t*>(c.o), n_pairs);
+  launch_pdl(attn_tc_merge_kernel, dim3(c.B * c.Hkv * ((a.R + 31) / 32)), dim3(256), 0, stream, a, reinterpret_cast<uint16_t*>(c.o));
   trk_end(trk);
   return cudaGetLastError();
 }
