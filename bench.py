@@ -407,6 +407,16 @@ def kernel_table(res):
     return rows
 
 
+def serial_roofline_ms(launches, kv_bytes, peaks):
+    """The kernels of a step run one after another, so the step cannot beat the SUM of its kernels' own rooflines: each
+    GEMM launch at the slower of its two (weight bytes at the HBM peak, flops at the tensor peak), the attention and the
+    scan at their HBM bytes.  Tighter than max(HBM, tensor) of the step's totals when a step mixes a weight-streaming
+    projection with tensor-bound layers.  `launches`: (name, flops, bytes) of one step's launches."""
+    hbm, tf = peaks["hbm_gbs"] * 1e9, peaks["bf16_tflops_sustained"] * 1e12
+    t = sum(max(f / tf, b / hbm) for n, f, b in launches if n.startswith(("gemm:", "gemm2:", "mamba_scan")))
+    return (t + kv_bytes / hbm) * 1e3
+
+
 def summarize(res, peaks, traffic=None):
     """Roofline numbers of one workload from the per-launch event times."""
     traffic = traffic or {}
@@ -483,11 +493,14 @@ def summarize(res, peaks, traffic=None):
                           launches_per_step=n_attn, algorithmic_bytes_per_launch=round(a["kv_bytes"] / n_attn),
                           note=f"visible target-KV bytes / CUDA-event time over its launches per step, of {peaks['source']}"))
     roof = max(roofs, key=lambda r: r["ms_per_step"])            # the dominant kernel of this workload
+    serial_ms = serial_roofline_ms([(n, v["flops"] / steps, v["bytes"] / steps) for n, v in res["prof"].items()],
+                                   a["kv_bytes"], peaks)
     return dict(
         ms_per_step=round(ms, 4), draft_tokens_per_s=round(res["B"] * res["k"] / (ms * 1e-3), 1),
         hbm_roofline_ms=round(hbm_time_ms, 4), hbm_roofline_frac=round(hbm_time_ms / ms, 4),
         tensor_roofline_ms=round(tensor_time_ms, 4),
         max_roofline_frac=round(max(hbm_time_ms, tensor_time_ms) / ms, 4),
+        serial_roofline_ms=round(serial_ms, 4), serial_roofline_frac=round(serial_ms / ms, 4),
         weight_GB=round(a["weight_bytes"] / 1e9, 3), kv_GB=round(a["kv_bytes"] / 1e9, 3),
         attention=dict(ms_per_step=round(att_ms, 4), achieved_GBs=round(att_gbs, 1), frac_of_hbm=round(att_gbs / hbm, 4),
                        launches_per_step=n_attn),
@@ -505,6 +518,7 @@ def brief(s, r=None):
     """The few figures of a summarised workload that the side tables of the bench line carry."""
     out = dict(draft_tokens_per_s=s["draft_tokens_per_s"], ms_per_step=s["ms_per_step"],
                hbm_roofline_frac=s["hbm_roofline_frac"], max_roofline_frac=s["max_roofline_frac"],
+               serial_roofline_frac=s["serial_roofline_frac"],
                attention_frac_of_hbm=s["attention"]["frac_of_hbm"], weight_GB=s["weight_GB"], kv_GB=s["kv_GB"],
                graph_replay_ms_per_step=s["graph_replay_ms_per_step"])
     if r is not None:
@@ -555,7 +569,8 @@ def run_sweep(steps, warmup, peaks, rank=0):
             att_ms, n_prof = 0.0, 2
             for _ in range(n_prof):
                 step()
-                att_ms += sum(e["ms"] for e in hs.hspec_get_profile(drafter.handle) if e["name"] == "attn_partial")
+                prof = hs.hspec_get_profile(drafter.handle)
+                att_ms += sum(e["ms"] for e in prof if e["name"] == "attn_partial")
             hs.hspec_set_profiling(drafter.handle, False)
             att_ms /= n_prof
             a = workload_accounting(dict(cfg, k=k), ctx, B, k)
@@ -564,6 +579,8 @@ def run_sweep(steps, warmup, peaks, rank=0):
             cells.append(dict(
                 B=B, k=k, ms_per_step=round(ms, 4), draft_tokens_per_s=round(B * k / (ms * 1e-3), 1),
                 hbm_roofline_frac=round(hbm_ms / ms, 4), max_roofline_frac=round(max(hbm_ms, tensor_ms) / ms, 4),
+                serial_roofline_frac=round(serial_roofline_ms([(e["name"], e["flops"], e["bytes"]) for e in prof],
+                                                              a["kv_bytes"], peaks) / ms, 4),
                 attention_frac_of_hbm=round(a["kv_bytes"] / (att_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 4) if att_ms > 0 else None,
                 kv_GB_read=round(a["kv_bytes"] / 1e9, 3),
                 drafter_kv_GB_avoided=round(a["drafter_kv_bytes_avoided"] / 1e9, 3),
@@ -768,6 +785,7 @@ def main_ours(args):
         "clocks": head["clocks"],
         "roofline": s["roofline"], "rooflines": s["rooflines"],
         "step": {k: s[k] for k in ("hbm_roofline_ms", "hbm_roofline_frac", "tensor_roofline_ms", "max_roofline_frac",
+                                   "serial_roofline_ms", "serial_roofline_frac",
                                    "weight_GB", "kv_GB", "drafter_kv_GB_avoided", "ms_per_step_profiled",
                                    "graph_replay_ms_per_step")},
         "attention": s["attention"], "gemm": s["gemm"], "kernels": kernel_table(head),

@@ -143,6 +143,27 @@ __device__ __forceinline__ void tmem_wait_ld32(uint32_t* r) {
                :
                : "memory");
 }
+// two fp32 operations in one instruction (sm_100 packed forms): halves the issue slots of the scale-and-subtract and of
+// the row-sum adds around the exponentials
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // 2^x by the special-function unit alone (flush-to-zero form: no range fix-up code around it)
 __device__ __forceinline__ float ex2_ftz(float x) {
   float y;
@@ -343,7 +364,7 @@ __device__ __forceinline__ void produce_operand(const AttnTcArgs& a, const CUten
 
 // Persistent: one CTA per SM walks the work list (items item_at(0), item_at(1), ...).  All ring and buffer indices
 // count tiles across items (gt): K slot = gt % NSK, V slot = gt % NSV, S / P buffer = gt % NSB.
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(352, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnTcArgs a,
                const int* __restrict__ count, const int4* __restrict__ items) {
   pdl_wait();
@@ -403,14 +424,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
     produce_operand(a, is_v ? &tmV : &tmK, is_v ? a.v_pool : a.k_pool, is_v ? a.vb : a.kb, sKV + (is_v ? NSK * KV_BYTES : 0),
                     is_v ? bars->v_full : bars->k_full, is_v ? bars->v_empty : bars->k_empty, abort_flag, items, n_items, lane,
                     is_v ? NSV : NSK);
-  } else if (warp == 9 || warp == 11) {
-    // ================================================================= MMA issuers: warp 9 the scores, warp 11 the P V products
-    // Two threads, because an issuing thread is held while the tensor pipe's queue is full: with one thread, a P that
-    // became ready while the scores two tiles ahead were being issued waited behind them, and the scores waited behind
-    // every P.  The pipe runs one thread's MMAs in issue order but not two threads', so the score thread waits for the
-    // COMPLETION of the P V product that last read the buffer it is about to overwrite (the barrier that frees that
-    // tile's V slot: same index, same phase, since both rings have three slots).
-    static_assert(NSB == NSV, "the score thread reuses the V ring's release barriers");
+  } else if (warp == 9) {
+    // ================================================================= MMA issuer
     if (lane == 0) {
       // fp32 accumulate, bf16 x bf16, M = 128, N = 128; scores: A = Q, B = K tile, both K-major in shared memory;
       // P V: A = P from tensor memory, B = V tile (MN-major)
@@ -423,76 +438,106 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
 #else
 #define MCLK(i)
 #endif
-      int4 w_next = items[item_at(0)];
-      if (warp == 9) {
-        // S = Q K^T of tile gt into S buffer gt % NSB, as far ahead of the softmax warps as the three buffers, the K
-        // ring and the Q tile allow; this runs across item boundaries (the softmax warps put the next item's Q tile in
-        // place while they work on this item's last tile: every score product of the item has finished by then).
-        for (; item_at(int(n)) < n_items && ok; ++n) {
-          const Item wi = unpack_item(w_next);
-          if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
-          const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
+      // Two cursors walk this CTA's tiles in the same order.  The P V cursor (item n, global tile gt) follows the softmax
+      // warps.  The score cursor (item n_s, tile t_s of T_s, global tile gts) runs up to two tiles ahead of it, ACROSS
+      // item boundaries: the softmax warps put the next item's Q tile in place while they work on this item's last tile
+      // (every score product of the item has finished by then), so the next item's first scores are computed while this
+      // item's last P V product and its read-out are still under way.
+      // S = Q K^T of tile gts into S buffer gts % NSB.  The buffer last held P of tile gts - NSB, whose P V product this
+      // thread issued earlier; the tensor pipe runs one thread's MMAs in issue order.
+      uint32_t gts = 0, n_s = 0;
+      int t_s = 0;
+      int4 ws_next = items[item_at(0)];
+      bool s_valid = true;
+      int T_s;
+      {
+        const Item w0 = unpack_item(ws_next);
+        T_s = make_range(w0.ctx, a.window, a.chunk, w0.c, a.k).T;
+        if (item_at(1) < n_items) ws_next = items[item_at(1)];
+      }
+      // returns 1 = issued, 0 = the item's Q tile is not there yet (only when it may come back later), -1 = timed out
+      auto issue_s = [&](bool must) -> int {
+        if (t_s == 0) {
+          const uint32_t qb = smem_u32(&bars->q_ready);
           MCLK(0)
-          if (!mbar_wait(smem_u32(&bars->q_ready), n & 1)) { ok = false; break; }      // this item's Q tile is in place
+          if (must) { if (!mbar_wait(qb, n_s & 1)) return -1; }
+          else if (!mbar_test(qb, n_s & 1)) return 0;
           MCLK(4)
-          for (int t = 0; t < g.T && ok; ++t, ++gt) {
-            const int s = gt % NSK;
-            MCLK(0)
-            if (!mbar_wait(smem_u32(&bars->k_full[s]), (gt / NSK) & 1)) { ok = false; break; }
-            MCLK(1)
-            // the buffer last held P of tile gt - NSB: its P V product must be complete
-            if (gt >= uint32_t(NSB) && !mbar_wait(smem_u32(&bars->v_empty[gt % NSV]), ((gt / NSV) - 1) & 1)) { ok = false; break; }
-            MCLK(2)
-            tc_fence_after();
-            const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
+          tc_fence_after();
+        }
+        const int s = gts % NSK;
+        MCLK(0)
+        if (!mbar_wait(smem_u32(&bars->k_full[s]), (gts / NSK) & 1)) return -1;
+        MCLK(1)
+        tc_fence_after();
+        const uint32_t kbase = smem_u32(sKV + s * KV_BYTES);
 #pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) {
-              const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
-              const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
-              umma_bf16(tmem_s0 + (gt % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
-            }
-            umma_commit(smem_u32(&bars->k_empty[s]));
-            umma_commit(smem_u32(&bars->s_ready[gt % NSB]));
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const uint64_t da = umma_desc_kmajor_sw128(smem_u32(sQ) + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+          const uint64_t db = umma_desc_kmajor_sw128(kbase + (ks >> 2) * KV_HALF) + uint64_t((ks & 3) * 2);
+          umma_bf16(tmem_s0 + (gts % NSB) * 128, da, db, id_qk, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(smem_u32(&bars->k_empty[s]));
+        umma_commit(smem_u32(&bars->s_ready[gts % NSB]));
+        ++gts;
+        if (++t_s == T_s) {                            // on to the next item (its descriptor was fetched an item ago)
+          t_s = 0;
+          ++n_s;
+          if (item_at(int(n_s)) < n_items) {
+            const Item wn = unpack_item(ws_next);
+            T_s = make_range(wn.ctx, a.window, a.chunk, wn.c, a.k).T;
+            if (item_at(int(n_s) + 1) < n_items) ws_next = items[item_at(int(n_s) + 1)];
+          } else {
+            s_valid = false;
           }
         }
-      } else {
-        for (; item_at(int(n)) < n_items && ok; ++n) {
-          const Item wi = unpack_item(w_next);
-          if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
-          const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
-          for (int t = 0; t < g.T && ok; ++t, ++gt) {
-            const int s = gt % NSV;
-            MCLK(0)
-            if (!mbar_wait(smem_u32(&bars->p_ready[gt % NSB]), (gt / NSB) & 1)) { ok = false; break; }
-            MCLK(2)
-            if (!mbar_wait(smem_u32(&bars->v_full[s]), (gt / NSV) & 1)) { ok = false; break; }
-            MCLK(3)
-            // the first P V product of an item overwrites O: the previous item's accumulator must have been read out
-            if (t == 0 && n > 0 && !mbar_wait(smem_u32(&bars->o_free), (n - 1) & 1)) { ok = false; break; }
-            MCLK(5)
-            tc_fence_after();
-            const uint32_t vbase = smem_u32(sKV + (NSK + s) * KV_BYTES);
-#pragma unroll
-            for (int ks = 0; ks < KT / 16; ++ks) {
-              // A = 16 keys of P = 8 TMEM columns; B = the same 16 keys (rows) of V
-              const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
-              umma_bf16_ts(tmem_o, tmem_s0 + (gt % NSB) * 128 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
-            }
-            umma_commit(smem_u32(&bars->v_empty[s]));
+        return 1;
+      };
+      int4 w_next = items[item_at(0)];
+      for (; item_at(int(n)) < n_items && ok; ++n) {
+        const Item wi = unpack_item(w_next);
+        if (item_at(int(n) + 1) < n_items) w_next = items[item_at(int(n) + 1)];
+        const Range g = make_range(wi.ctx, a.window, a.chunk, wi.c, a.k);
+        for (int t = 0; t < g.T && ok; ++t, ++gt) {
+          // the scores of this tile must be under way (the softmax warps wait for them); the next two are issued as soon
+          // as their K tile and, at an item's first tile, its Q tile are there
+          while (ok && s_valid && gts <= gt + 2) {
+            const int r = issue_s(gts <= gt);
+            if (r < 0) ok = false;
+            if (r <= 0) break;
           }
-          if (ok) umma_commit(smem_u32(&bars->o_done));
+          if (!ok) break;
+          const int s = gt % NSV;
+          MCLK(0)
+          if (!mbar_wait(smem_u32(&bars->p_ready[gt % NSB]), (gt / NSB) & 1)) { ok = false; break; }
+          MCLK(2)
+          if (!mbar_wait(smem_u32(&bars->v_full[s]), (gt / NSV) & 1)) { ok = false; break; }
+          MCLK(3)
+          // the first P V product of an item overwrites O: the previous item's accumulator must have been read out
+          if (t == 0 && n > 0 && !mbar_wait(smem_u32(&bars->o_free), (n - 1) & 1)) { ok = false; break; }
+          MCLK(5)
+          tc_fence_after();
+          const uint32_t vbase = smem_u32(sKV + (NSK + s) * KV_BYTES);
+#pragma unroll
+          for (int ks = 0; ks < KT / 16; ++ks) {
+            // A = 16 keys of P = 8 TMEM columns; B = the same 16 keys (rows) of V
+            const uint64_t db = umma_desc_mnmajor_sw128(vbase + ks * 2048);
+            umma_bf16_ts(tmem_o, tmem_s0 + (gt % NSB) * 128 + ks * 8, db, id_pv, (t > 0 || ks > 0) ? 1u : 0u);
+          }
+          umma_commit(smem_u32(&bars->v_empty[s]));
         }
+        if (ok) umma_commit(smem_u32(&bars->o_done));
       }
 #ifdef HSPEC_ATTN_TIMING
       MCLK(0)
       if (blockIdx.x == 0 || blockIdx.x == 147)
-        printf("cta %d mma warp %d: total %lld | issue %lld wait_k %lld wait_p_or_buffer %lld wait_v %lld wait_q %lld wait_ofree %lld\n",
-               blockIdx.x, warp, clock64() - m_start, mk[0], mk[1], mk[2], mk[3], mk[4], mk[5]);
+        printf("cta %d mma: total %lld | issue %lld wait_k %lld wait_p %lld wait_v %lld wait_q %lld wait_ofree %lld\n",
+               blockIdx.x, clock64() - m_start, mk[0], mk[1], mk[2], mk[3], mk[4], mk[5]);
 #endif
       if (!ok) {
         atomicExch(a.status, STATUS_TIMEOUT_MMA);
         *abort_flag = 1;
-        if (warp == 11) mbar_arrive(smem_u32(&bars->o_done));
+        mbar_arrive(smem_u32(&bars->o_done));
       }
     }
   } else {
@@ -649,16 +694,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ 
         TCLK(4)
         // ---- P = exp2(s * scale - m_ref) -> bf16 pairs -> this thread's 32 of the 64 P columns, which lie over the
         // first half of the S buffer (both threads of the row took their scores into registers before the exchange)
-        const float neg_m = -m_ref;
-        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint64_t scale2 = pack_f32x2(a.scale_log2, a.scale_log2), neg_m2 = pack_f32x2(-m_ref, -m_ref);
+        uint64_t ls2[2] = {0ull, 0ull};               // two packed accumulators = four row-sum chains
         uint32_t pw[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
-          const float p0 = ex2_ftz(fmaf(s[2 * e], a.scale_log2, neg_m));
-          const float p1 = ex2_ftz(fmaf(s[2 * e + 1], a.scale_log2, neg_m));
-          ls4[e & 1] += p0; ls4[2 + (e & 1)] += p1;
+          float x0, x1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(s[2 * e], s[2 * e + 1]), scale2, neg_m2), x0, x1);
+          const float p0 = ex2_ftz(x0), p1 = ex2_ftz(x1);
+          ls2[e & 1] = add_f32x2(ls2[e & 1], pack_f32x2(p0, p1));
           pw[e] = pack_bf16(p0, p1);
         }
+        float ls4[4];
+        unpack_f32x2(ls2[0], ls4[0], ls4[1]);
+        unpack_f32x2(ls2[1], ls4[2], ls4[3]);
         tmem_st32(t_s + hf * 32, pw);
         l_sum += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
         tmem_st_wait();
@@ -905,7 +954,7 @@ cudaError_t attention_tc_launch(const AttnCall& c, int max_chunks, cudaStream_t 
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   trk_begin(trk, "attn_partial");
-  launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(384), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
+  launch_pdl(attn_tc_kernel, dim3(n_sms), dim3(352), smem, stream, tmK, tmV, a, (const int*)count, (const int4*)items);
   trk_end(trk);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;

@@ -41,6 +41,15 @@ def test_peaks_fallback_and_file(tmp_path, monkeypatch):
     assert p["hbm_gbs"] > 1000 and p["bf16_tflops_sustained"] > 100 and p["source"] in ("measured", "fallback")
 
 
+def test_serial_roofline_sums_each_launch_at_its_own_bound():
+    peaks = dict(hbm_gbs=1000.0, bf16_tflops_sustained=100.0)
+    launches = [("gemm:proj_ds", 1e9, 2e9),          # streaming: 2 GB at 1 TB/s = 2 ms (its flops would take 0.01 ms)
+                ("gemm2:gate_up", 4e11, 1e8),        # tensor-bound: 4e11 flops at 100 TF/s = 4 ms (bytes 0.1 ms)
+                ("mamba_scan", 1e6, 5e8),            # 0.5 ms of state bytes
+                ("rmsnorm", 0.0, 9e9)]               # row-wise kernels are not counted
+    assert bench.serial_roofline_ms(launches, 1e9, peaks) == pytest.approx(2.0 + 4.0 + 0.5 + 1.0)
+
+
 def _worker(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
