@@ -647,9 +647,9 @@ def case_gemm(reps, M=2048, n_out=25600, K=5120):
           f"{2 * n_out * K / (min(us) * 1e-6) / 1e12:.2f} TB/s of weights, {2 * M * n_out * K / (min(us) * 1e-6) / 1e12:.0f} TFLOP/s")
 
 
-def case_scan(reps):
+def case_scan(reps, B=32, Di=8192):
     import paper_2609_24197_b200 as hs
-    B, k, Di, P, N, G = 32, 16, 8192, 64, 128, 4
+    k, P, N, G = 16, 64, 128, 4
     H = Di // P
     ld = 2 * Di + 2 * G * N + H
     zx = _randn((B * k, ld), 6, 1.0, torch.float32)
@@ -658,10 +658,39 @@ def case_scan(reps):
     dtb, Al, Ds = _randn((H,), 10, 1.0, torch.float32) - 4, torch.rand(H, device="cuda") * 2, torch.ones(H, device="cuda")
     y = torch.empty((B * k, Di), dtype=torch.float32, device="cuda")
     ws = torch.empty(hs.hspec_scan_workspace_bytes(B, k, Di, N, G), dtype=torch.uint8, device="cuda")
-    for _ in range(reps):
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    ev[0].record()
+    for i in range(reps):
         hs.hspec_op_mamba_scan(zx, None, s0, cw, cb, dtb, Al, Ds, y, B, k, Di, P, N, G, 4, ws)
+        ev[i + 1].record()
     torch.cuda.synchronize()
-    print(f"scan: B={B} H={H} S_init bytes per launch={B * H * P * N * 2}")
+    us = [round(ev[i].elapsed_time(ev[i + 1]) * 1e3, 1) for i in range(reps)]
+    print(f"scan: B={B} H={H} S_init bytes per launch={B * H * P * N * 2} activation bytes (z, xBC, dt in; y out)="
+          f"{B * k * (ld + Di) * 4} us per call (conv + cb + stream)={us}")
+
+
+def case_rowwise(reps, M=2048, D=5120, Hq=64, Hkv=8, dh=128, k=16):
+    """The row-wise kernels of a layer at the 32B-class shapes: RMSNorm over D, and per-head norm + RoPE of q, k, v."""
+    import paper_2609_24197_b200 as hs
+    x, w = _randn((M, D), 31, 1.0, torch.float32), 1 + _randn((D,), 32, 0.02, torch.float32)
+    y = torch.empty((M, D), dtype=torch.float16, device="cuda")
+    qkv = _randn((M, (Hq + 2 * Hkv) * dh), 33, 1.0, torch.float32)
+    qw, kw = 1 + _randn((dh,), 34, 0.1, torch.float32), 1 + _randn((dh,), 35, 0.1, torch.float32)
+    B = M // k
+    ctx = torch.randint(0, 32000, (B,), dtype=torch.int32, device="cuda")
+    q = torch.empty((M, Hq, dh), dtype=torch.bfloat16, device="cuda")
+    kb, vb = (torch.empty((M, Hkv, dh), dtype=torch.bfloat16, device="cuda") for _ in range(2))
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * reps + 1)]
+    ev[0].record()
+    for i in range(reps):
+        hs.hspec_op_rmsnorm(x, w, y, 1e-6)
+        ev[2 * i + 1].record()
+        hs.hspec_op_qk_norm_rope(qkv, qw, kw, ctx, q, kb, vb, B, k, Hq, Hkv, dh, 1e6, 1e-6, 1)
+        ev[2 * i + 2].record()
+    torch.cuda.synchronize()
+    us = [round(ev[i].elapsed_time(ev[i + 1]) * 1e3, 1) for i in range(2 * reps)]
+    print(f"rowwise: rmsnorm [{M} x {D}] fp32 -> fp16 ({M * D * 6} bytes) us={us[0::2]}; qk_norm_rope [{M} x {(Hq + 2 * Hkv) * dh}] "
+          f"fp32 -> bf16 ({M * (Hq + 2 * Hkv) * dh * 6} bytes) us={us[1::2]}")
 
 
 def case_overlap(reps):
@@ -716,6 +745,8 @@ CASES = {
     "gemm_skinny64": (case_gemm, dict(M=64, n_out=262144, K=5120)),                # Proj_dS at concurrency 64 (a fifth of it)
     "gemm_skinny128": (case_gemm, dict(M=128, n_out=262144, K=5120)),              # Proj_dS at concurrency 128 (a fifth of it; the 2-SM kernel)
     "scan": (case_scan, {}),
+    "scan32b": (case_scan, dict(B=128, Di=10240)),                                 # conc128_32b's layer
+    "rowwise": (case_rowwise, {}),
     "overlap": (case_overlap, {}),
 }
 

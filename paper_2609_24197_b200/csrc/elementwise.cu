@@ -3,6 +3,8 @@
 #include "common.cuh"
 #include "kernels.h"
 
+#include <cstdlib>
+
 namespace hspec {
 
 namespace {
@@ -130,6 +132,75 @@ __global__ void qk_norm_rope_kernel(const float* __restrict__ qkv, const float* 
   }
 }
 
+// Same operation, one CTA per row (dh a multiple of 4): the row's dh/2 sines and cosines are computed once into shared
+// memory and serve all Hq + Hkv heads (a warp per head recomputed them 72 times per row at the 32B-class shapes), a
+// warp takes every eighth head with 8-byte loads, the loads of ROPE_HB heads in flight together.  The arithmetic per
+// element is that of the kernel above.
+constexpr int ROPE_HB = 5;
+__global__ void __launch_bounds__(256)
+qk_norm_rope_row_kernel(const float* __restrict__ qkv, const float* __restrict__ qw, const float* __restrict__ kw,
+                        const float* __restrict__ inv_freq, const int32_t* __restrict__ ctx_lens,
+                        __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ kb, __nv_bfloat16* __restrict__ vb,
+                        int k, int Hq, int Hkv, int dh, float eps, int qk_norm) {
+  pdl_wait();
+  pdl_trigger();
+  __shared__ __align__(8) float cs_s[64], sn_s[64];
+  const int m = blockIdx.x, half = dh / 2, heads = Hq + 2 * Hkv;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const float pos = float(ctx_lens[m / k] + m % k);
+  for (int j = threadIdx.x; j < half; j += blockDim.x) sincosf(pos * inv_freq[j], &sn_s[j], &cs_s[j]);
+  __syncthreads();
+  const float* row = qkv + size_t(m) * heads * dh;
+  // dh <= 128: a lane's share of a head is one pair of rotation pairs, j = 2 lane and 2 lane + 1 (lanes past dh / 4
+  // hold zeros and store nothing, but take part in the warp reduction)
+  const int j2 = lane;
+  const bool act = j2 < half / 2;
+  for (int h0 = warp; h0 < heads; h0 += 8 * ROPE_HB) {
+    float2 a[ROPE_HB], b[ROPE_HB];
+#pragma unroll
+    for (int u = 0; u < ROPE_HB; ++u) {
+      const int hh = h0 + u * 8;
+      if (hh < heads && act) {
+        a[u] = *reinterpret_cast<const float2*>(row + size_t(hh) * dh + 2 * j2);
+        b[u] = *reinterpret_cast<const float2*>(row + size_t(hh) * dh + half + 2 * j2);
+      } else {
+        a[u] = b[u] = make_float2(0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < ROPE_HB; ++u) {
+      const int hh = h0 + u * 8;
+      if (hh >= heads) continue;                            // warp-uniform
+      if (hh >= Hq + Hkv) {                                 // values: plain conversion
+        if (act) {
+          __nv_bfloat16* dst = vb + (size_t(m) * Hkv + (hh - Hq - Hkv)) * dh;
+          *reinterpret_cast<__nv_bfloat162*>(dst + 2 * j2) = __floats2bfloat162_rn(a[u].x, a[u].y);
+          *reinterpret_cast<__nv_bfloat162*>(dst + half + 2 * j2) = __floats2bfloat162_rn(b[u].x, b[u].y);
+        }
+        continue;
+      }
+      const bool is_q = hh < Hq;
+      float inv = 1.f;
+      if (qk_norm) {
+        float ss = a[u].x * a[u].x + a[u].y * a[u].y + b[u].x * b[u].x + b[u].y * b[u].y;
+        for (int off = 16; off > 0; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        inv = rsqrtf(ss / float(dh) + eps);
+      }
+      if (!act) continue;
+      float v1x = a[u].x * inv, v1y = a[u].y * inv, v2x = b[u].x * inv, v2y = b[u].y * inv;
+      if (qk_norm) {
+        const float* w = is_q ? qw : kw;
+        const float2 wa = *reinterpret_cast<const float2*>(w + 2 * j2), wb = *reinterpret_cast<const float2*>(w + half + 2 * j2);
+        v1x *= wa.x; v1y *= wa.y; v2x *= wb.x; v2y *= wb.y;
+      }
+      const float2 cs = *reinterpret_cast<const float2*>(cs_s + 2 * j2), sn = *reinterpret_cast<const float2*>(sn_s + 2 * j2);
+      __nv_bfloat16* dst = is_q ? q + (size_t(m) * Hq + hh) * dh : kb + (size_t(m) * Hkv + (hh - Hq)) * dh;
+      *reinterpret_cast<__nv_bfloat162*>(dst + 2 * j2) = __floats2bfloat162_rn(v1x * cs.x - v2x * sn.x, v1y * cs.y - v2y * sn.y);
+      *reinterpret_cast<__nv_bfloat162*>(dst + half + 2 * j2) = __floats2bfloat162_rn(v2x * cs.x + v1x * sn.x, v2y * cs.y + v1y * sn.y);
+    }
+  }
+}
+
 // The comparison drafters' cache write (Sec. 2.2 "KV injection in block drafting"): one warp per (new position, head).
 // Key heads: optional RMSNorm over dh, rotate-half RoPE at the position, bf16, into the paged key pool; value heads:
 // bf16 into the paged value pool.  Row t belongs to request req[t] and sits at absolute position pos[t].
@@ -231,7 +302,7 @@ cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token,
 
 cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_16, int M, int n, float eps, cudaStream_t stream,
                            uint32_t* status, bool bf16_out) {
-  const int threads = n >= 2048 ? 512 : 256;
+  const int threads = n >= 2048 ? 512 : 256;            // (256 or 384 threads per row measured the same at n = 5120)
   cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, y_16, n, eps, status, bf16_out ? 1 : 0);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
@@ -242,6 +313,11 @@ cudaError_t qk_norm_rope_launch(const float* qkv, const float* qw, const float* 
   if (dh > 256 || (dh & 1)) return cudaErrorInvalidValue;
   const float* tab = rope_table(theta, dh);
   if (!tab) return cudaErrorMemoryAllocation;
+  if ((dh & 3) == 0 && dh <= 128) {
+    cudaError_t e = launch_pdl(qk_norm_rope_row_kernel, dim3(B * k), dim3(256), 0, stream, qkv, qw, kw, tab, ctx_lens,
+                               (__nv_bfloat16*)q, (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps, qk_norm);
+    return e != cudaSuccess ? e : cudaGetLastError();
+  }
   const int n_pairs = B * k * (Hq + 2 * Hkv);
   cudaError_t e = launch_pdl(qk_norm_rope_kernel, dim3((n_pairs + 7) / 8), dim3(256), 0, stream, qkv, qw, kw, tab, ctx_lens,
                              (__nv_bfloat16*)q, (__nv_bfloat16*)kb, (__nv_bfloat16*)vb, k, Hq, Hkv, dh, eps, qk_norm, n_pairs);

@@ -326,60 +326,118 @@ mamba_scan_mma_kernel(ScanArgs a) {
 // Three-kernel form of the fast path (used when the caller provides scratch): the small per-position
 // operands are prepared once per request and group, so the kernel that streams S_init has no
 // block-wide phases in front of its loads.
-//   scan_conv_kernel   causal depthwise conv + SiLU of every xBC channel (thread = channel, taps in registers);
+//   scan_conv_kernel   causal depthwise conv + SiLU of every xBC channel (thread = 4 channels x 4 positions);
 //                      C is also written as fp16 head + fp16 remainder for the tensor-core contraction
 //   scan_cb_kernel     CB[b, g, t, s] = C_t . B_s for s <= t
 //   mamba_scan_stream_kernel  one warp per head: everything it needs is fetched up front (cp.async for the
 //                      shared operands, 16-byte loads of S_init straight into the MMA fragments)
-__global__ void scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* __restrict__ c16) {
+constexpr int CONV_ROWS = 4;                                 // block positions per thread
+// thread = (VEC adjacent channels, group of four block positions): the filter reads raw inputs only, so the groups are
+// independent; a thread's seven (vector) loads are in flight together and it needs few registers.  VEC = 4 (16-byte
+// loads and stores) when every channel offset and row stride is a multiple of four, else 1.  (One thread per channel
+// walking all k rows held 72 registers, three blocks per SM, and reached 25 % of the DRAM peak with its warps waiting
+// on loads; one channel and four rows per thread was bound by the instruction issue, 85 %, most of it set-up.)
+template <int VEC>
+__global__ void __launch_bounds__(256)
+scan_conv_kernel(ScanArgs a, float* __restrict__ xact, __half* __restrict__ c16) {
   pdl_wait();
   pdl_trigger();
-  const int ch = blockIdx.x * blockDim.x + threadIdx.x;
-  const int b = blockIdx.y;
+  const int ch = (blockIdx.x * blockDim.x + threadIdx.x) * VEC;
+  const int n_grp = (a.k + CONV_ROWS - 1) / CONV_ROWS;
+  const int b = blockIdx.y / n_grp, i0 = (blockIdx.y % n_grp) * CONV_ROWS;
   if (ch >= a.d_xBC) return;
-  float w[4] = {0.f, 0.f, 0.f, 0.f};
-  for (int j = 0; j < a.d_conv; ++j) w[4 - a.d_conv + j] = a.conv_w[ch * a.d_conv + j];   // right-aligned taps
-  const float bias = a.conv_b[ch];
-  float h0 = 0.f, h1 = 0.f, h2 = 0.f;                        // the three rows before the current one (zero left context)
+  float w[VEC][4], bias[VEC];
+#pragma unroll
+  for (int v = 0; v < VEC; ++v) {
+    if (VEC == 4 && a.d_conv == 4) {                         // a channel's four taps in one 16-byte load
+      const float4 t = __ldg(reinterpret_cast<const float4*>(a.conv_w) + ch + v);
+      w[v][0] = t.x; w[v][1] = t.y; w[v][2] = t.z; w[v][3] = t.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[v][j] = (j >= 4 - a.d_conv) ? a.conv_w[(ch + v) * a.d_conv + j - (4 - a.d_conv)] : 0.f;   // right-aligned taps
+    }
+  }
+  if (VEC == 4) {
+    const float4 t = __ldg(reinterpret_cast<const float4*>(a.conv_b + ch));
+    bias[0] = t.x; bias[VEC > 1 ? 1 : 0] = t.y; bias[VEC > 1 ? 2 : 0] = t.z; bias[VEC > 1 ? 3 : 0] = t.w;
+  } else {
+    bias[0] = a.conv_b[ch];
+  }
   const size_t row0 = size_t(b) * a.k;
   const int GN = a.G * a.N;
   const int c_col = ch - a.Di - GN;                          // >= 0 for C channels
-  // eight rows' loads are issued together: the recurrence over rows is short, the load latency is not
-  for (int i0 = 0; i0 < a.k; i0 += 8) {
-    float in[8];
+  float in[CONV_ROWS + 3][VEC];                              // rows i0 - 3 .. i0 + 3 (zero left context before the block)
 #pragma unroll
-    for (int j = 0; j < 8; ++j) in[j] = (i0 + j < a.k) ? __ldcs(a.zxbcdt + (row0 + i0 + j) * a.ld_in + a.Di + ch) : 0.f;
+  for (int j = 0; j < CONV_ROWS + 3; ++j) {
+    const int i = i0 - 3 + j;
+    const bool ok = i >= 0 && i < a.k;
+    const float* src = a.zxbcdt + (row0 + (ok ? i : 0)) * a.ld_in + a.Di + ch;
+    if (VEC == 4) {
+      const float4 t = ok ? __ldg(reinterpret_cast<const float4*>(src)) : make_float4(0.f, 0.f, 0.f, 0.f);
+      in[j][0] = t.x; in[j][VEC > 1 ? 1 : 0] = t.y; in[j][VEC > 1 ? 2 : 0] = t.z; in[j][VEC > 1 ? 3 : 0] = t.w;
+    } else {
+      in[j][0] = ok ? __ldg(src) : 0.f;
+    }
+  }
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int i = i0 + j;
-      if (i >= a.k) break;
-      const float cur = in[j];
-      const float v = silu_f(bias + w[0] * h0 + w[1] * h1 + w[2] * h2 + w[3] * cur);
-      h0 = h1; h1 = h2; h2 = cur;
-      xact[(row0 + i) * a.d_xBC + ch] = v;
-      if (c_col >= 0) {
-        const __half hi = __float2half_rn(v);
-        c16[((row0 + i) * 2 + 0) * GN + c_col] = hi;
-        c16[((row0 + i) * 2 + 1) * GN + c_col] = __float2half_rn(v - __half2float(hi));
+  for (int r = 0; r < CONV_ROWS; ++r) {
+    const int i = i0 + r;
+    if (i >= a.k) break;
+    float o[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v)
+      o[v] = silu_f(bias[v] + w[v][0] * in[r][v] + w[v][1] * in[r + 1][v] + w[v][2] * in[r + 2][v] + w[v][3] * in[r + 3][v]);
+    float* dst = xact + (row0 + i) * a.d_xBC + ch;
+    if (VEC == 4) *reinterpret_cast<float4*>(dst) = make_float4(o[0], o[VEC > 1 ? 1 : 0], o[VEC > 1 ? 2 : 0], o[VEC > 1 ? 3 : 0]);
+    else dst[0] = o[0];
+    if (c_col >= 0) {
+      __half hi[VEC], lo[VEC];
+#pragma unroll
+      for (int v = 0; v < VEC; ++v) { hi[v] = __float2half_rn(o[v]); lo[v] = __float2half_rn(o[v] - __half2float(hi[v])); }
+      __half* d_hi = c16 + ((row0 + i) * 2 + 0) * GN + c_col;
+      __half* d_lo = c16 + ((row0 + i) * 2 + 1) * GN + c_col;
+      if (VEC == 4) {
+        *reinterpret_cast<uint2*>(d_hi) = *reinterpret_cast<const uint2*>(hi);
+        *reinterpret_cast<uint2*>(d_lo) = *reinterpret_cast<const uint2*>(lo);
+      } else {
+        d_hi[0] = hi[0];
+        d_lo[0] = lo[0];
       }
     }
   }
 }
 
-__global__ void scan_cb_kernel(ScanArgs a, const float* __restrict__ xact, float* __restrict__ cb) {
+// CB[b, g, t, s] = C_t . B_s for s <= t.  One block per (request, group): the block's B and C rows are staged in shared
+// memory (rows padded by four floats so that the 16-byte reads of a warp's threads spread over the banks), each thread
+// takes (t, s) pairs with float4 dot products in the order n = 0 .. N - 1 of the scalar loop it replaces (that loop read
+// both rows from global memory one float at a time and ran at the L1's limit).
+__global__ void __launch_bounds__(256)
+scan_cb_kernel(ScanArgs a, const float* __restrict__ xact, float* __restrict__ cb) {
   pdl_wait();
   pdl_trigger();
+  extern __shared__ __align__(16) float cb_sm[];
   const int g = blockIdx.x, b = blockIdx.y;
-  const int k = a.k, N = a.N;
+  const int k = a.k, N = a.N, ldr = N + 4;
   const size_t row0 = size_t(b) * k;
   const int GN = a.G * N;
+  float* Bs = cb_sm;                 // [k][N + 4]
+  float* Cs = cb_sm + k * ldr;       // [k][N + 4]
+  for (int idx = threadIdx.x; idx < 2 * k * (N / 4); idx += blockDim.x) {
+    const int which = idx / (k * (N / 4)), rem = idx % (k * (N / 4)), r = rem / (N / 4), c4 = rem % (N / 4);
+    const float4 v = *reinterpret_cast<const float4*>(xact + (row0 + r) * a.d_xBC + a.Di + which * GN + g * N + c4 * 4);
+    *reinterpret_cast<float4*>((which ? Cs : Bs) + r * ldr + c4 * 4) = v;
+  }
+  __syncthreads();
   for (int idx = threadIdx.x; idx < k * k; idx += blockDim.x) {
     const int t = idx / k, s2 = idx % k;
     float dot = 0.f;
     if (s2 <= t) {
-      const float* cr = xact + (row0 + t) * a.d_xBC + a.Di + GN + g * N;
-      const float* br = xact + (row0 + s2) * a.d_xBC + a.Di + g * N;
-      for (int n = 0; n < N; ++n) dot += cr[n] * br[n];
+      const float4* cr = reinterpret_cast<const float4*>(Cs + t * ldr);
+      const float4* br = reinterpret_cast<const float4*>(Bs + s2 * ldr);
+      for (int n4 = 0; n4 < N / 4; ++n4) {
+        const float4 c = cr[n4], bb = br[n4];
+        dot += c.x * bb.x; dot += c.y * bb.y; dot += c.z * bb.z; dot += c.w * bb.w;
+      }
     }
     cb[((size_t(b) * a.G + g) * KMAX + t) * KMAX + s2] = dot;
   }
@@ -392,14 +450,16 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   pdl_wait();
   pdl_trigger();
   constexpr int HPC = 4, NT = P / 8, KP = N / 32, ROWS = MT * 16;
+  constexpr int CS = 2 * N + 32;                               // halves per C row (hi | lo | 64 bytes of padding: the 16-byte
+                                                               // fragment reads of rows gq and gq + 1 then fall on different banks)
   extern __shared__ __align__(16) float sm[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h0 = blockIdx.x * HPC, b = blockIdx.y;
   const int hpg = a.H / a.G, g = h0 / hpg, k = a.k, GN = a.G * N;
   const int h = h0 + warp;
   const size_t row0 = size_t(b) * k;
-  __half* C16 = reinterpret_cast<__half*>(sm);                 // [ROWS][2][N]  (hi, lo), rows >= k zero
-  float* CB = sm + ROWS * N;                                   // [ROWS][ROWS]
+  __half* C16 = reinterpret_cast<__half*>(sm);                 // [ROWS][CS]  (hi, lo), rows >= k zero
+  float* CB = sm + ROWS * CS / 2;                                   // [ROWS][ROWS]
   float* xs = CB + ROWS * ROWS + warp * (ROWS * P);            // per warp [ROWS][P]
   float* Wh = CB + ROWS * ROWS + HPC * ROWS * P + warp * ROWS * (ROWS + 1);   // per warp [ROWS][ROWS+1]
 
@@ -417,7 +477,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   // ---- shared operands (C halves, CB) and this head's x rows: cp.async, zero fill for the padding rows
   for (int idx = tid; idx < ROWS * 2 * N / 8; idx += 128) {
     const int r = idx / (2 * N / 8), rest = idx % (2 * N / 8), half = rest / (N / 8), c8 = rest % (N / 8);
-    cp_async16(smem_u32(C16 + (r * 2 + half) * N + c8 * 8), c16 + ((row0 + min(r, k - 1)) * 2 + half) * GN + g * N + c8 * 8, r < k);
+    cp_async16(smem_u32(C16 + r * CS + half * N + c8 * 8), c16 + ((row0 + min(r, k - 1)) * 2 + half) * GN + g * N + c8 * 8, r < k);
   }
   for (int idx = tid; idx < ROWS * ROWS / 4; idx += 128) {
     const int r = idx / (ROWS / 4), c4 = idx % (ROWS / 4);
@@ -470,8 +530,8 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
       }
 #pragma unroll
       for (int mt = 0; mt < MT; ++mt) {
-        const __half* c0 = C16 + ((mt * 16 + gq) * 2) * N + kp * 32 + tq * 8;
-        const __half* c1 = C16 + ((mt * 16 + gq + 8) * 2) * N + kp * 32 + tq * 8;
+        const __half* c0 = C16 + (mt * 16 + gq) * CS + kp * 32 + tq * 8;
+        const __half* c1 = C16 + (mt * 16 + gq + 8) * CS + kp * 32 + tq * 8;
         const uint4 c_lo = *reinterpret_cast<const uint4*>(c0), c_hi = *reinterpret_cast<const uint4*>(c1);
         const uint4 r_lo = *reinterpret_cast<const uint4*>(c0 + N), r_hi = *reinterpret_cast<const uint4*>(c1 + N);
         const uint32_t a0[4] = {c_lo.x, c_hi.x, c_lo.y, c_hi.y}, a1[4] = {c_lo.z, c_hi.z, c_lo.w, c_hi.w};
@@ -526,7 +586,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
 template <int MT>
 size_t scan_stream_smem() {
   constexpr int P = 64, N = 128, HPC = 4, ROWS = MT * 16;
-  return sizeof(__half) * ROWS * 2 * N + sizeof(float) * (ROWS * ROWS + HPC * ROWS * P + HPC * ROWS * (ROWS + 1));
+  return sizeof(__half) * ROWS * (2 * N + 32) + sizeof(float) * (ROWS * ROWS + HPC * ROWS * P + HPC * ROWS * (ROWS + 1));
 }
 
 template <int MT>
@@ -562,10 +622,15 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
     float* cbw = xact + M * a.d_xBC;
     __half* c16 = reinterpret_cast<__half*>(cbw + size_t(c.B) * c.G * KMAX * KMAX);
     trk_begin(trk, "scan_conv", 0, double(M) * a.d_xBC * 8);
-    launch_pdl(scan_conv_kernel, dim3((a.d_xBC + 255) / 256, c.B), dim3(256), 0, stream, a, xact, c16);
+    const bool vec4 = a.Di % 4 == 0 && (c.G * c.N) % 4 == 0 && a.ld_in % 4 == 0 &&
+                      ((reinterpret_cast<uintptr_t>(a.zxbcdt) | reinterpret_cast<uintptr_t>(c.ws) | reinterpret_cast<uintptr_t>(a.conv_w) |
+                        reinterpret_cast<uintptr_t>(a.conv_b)) & 15) == 0;
+    const dim3 grid_c((a.d_xBC / (vec4 ? 4 : 1) + 255) / 256, c.B * ((c.k + CONV_ROWS - 1) / CONV_ROWS));
+    if (vec4) launch_pdl(scan_conv_kernel<4>, grid_c, dim3(256), 0, stream, a, xact, c16);
+    else launch_pdl(scan_conv_kernel<1>, grid_c, dim3(256), 0, stream, a, xact, c16);
     trk_end(trk);
     trk_begin(trk, "scan_cb", 0, 0);
-    launch_pdl(scan_cb_kernel, dim3(c.G, c.B), dim3(256), 0, stream, a, xact, (float*)cbw);
+    launch_pdl(scan_cb_kernel, dim3(c.G, c.B), dim3(256), size_t(2) * c.k * (c.N + 4) * sizeof(float), stream, a, xact, (float*)cbw);
     trk_end(trk);
     const size_t smem_s = two ? scan_stream_smem<2>() : scan_stream_smem<1>();
     static bool sset[2][MAX_DEVICES] = {};
