@@ -20,6 +20,15 @@ __global__ void embed_rows_kernel(const __nv_bfloat16* __restrict__ embed, const
   const int tok = (i == 0) ? last_token[b] : mask_id;
   const __nv_bfloat16* src = embed + size_t(tok) * D;
   float* dst = X + size_t(m) * D;
+  if ((D & 3) == 0 && ((reinterpret_cast<uintptr_t>(embed) | reinterpret_cast<uintptr_t>(X)) & 15) == 0) {
+    // four elements per thread and step: 8-byte loads, 16-byte stores
+    for (int d4 = threadIdx.x; d4 < D / 4; d4 += blockDim.x) {
+      const uint2 t = __ldg(reinterpret_cast<const uint2*>(src) + d4);
+      reinterpret_cast<float4*>(dst)[d4] = make_float4(__uint_as_float(t.x << 16), __uint_as_float(t.x & 0xffff0000u),
+                                                       __uint_as_float(t.y << 16), __uint_as_float(t.y & 0xffff0000u));
+    }
+    return;
+  }
   for (int d = threadIdx.x; d < D; d += blockDim.x) dst[d] = __bfloat162float(src[d]);
 }
 
@@ -63,6 +72,7 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
     for (int i = 0; i < 6; ++i) {
       const int d4 = threadIdx.x + i * blockDim.x;
       if (d4 < nv) {
+        // (fetching the gains together with the row, before the block-wide sum, measured slower: 27 against 23 us)
         const float4 g = reinterpret_cast<const float4*>(w)[d4];
         // (a normalised value is at most sqrt(n) |w|; the saturating convert still guards a huge gain or a NaN-free
         // overflow of x * inv)

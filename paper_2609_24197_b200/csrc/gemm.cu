@@ -305,37 +305,35 @@ __global__ void splitk_reduce_f32x4_kernel(const float* __restrict__ part, int M
 }
 
 // ids[m] = lowest index among the per-tile maxima (tiles are in ascending vocabulary order).
-__global__ void argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
-                                     int* __restrict__ ids, const int* __restrict__ id_map) {
+// The partials are [tile][row]: a block takes eight consecutive rows, thread (r = tid % 8, tid / 8) walks every 32nd
+// tile of row r, so that eight neighbouring threads read one 32-byte sector (a block per row read 4 bytes of every
+// sector it touched: 33 us for 19 MB at M = 2048, V = 152 064).
+__device__ __forceinline__ void argmax_take(float& v, int& idx, float ov, int oi) {
+  if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+}
+__global__ void __launch_bounds__(256)
+argmax_reduce_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int M,
+                     int* __restrict__ ids, const int* __restrict__ id_map) {
   pdl_wait();
   pdl_trigger();
-  const int m = blockIdx.x;
+  const int r = threadIdx.x & 7, m = blockIdx.x * 8 + r;
   float v = -INFINITY;
   int idx = 0x7fffffff;
-  for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
-    const float ov = pv[size_t(t) * M + m];
-    const int oi = pi[size_t(t) * M + m];
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  if (m < M) {
+    for (int t = threadIdx.x >> 3; t < n_tiles; t += 32) argmax_take(v, idx, pv[size_t(t) * M + m], pi[size_t(t) * M + m]);
   }
-  __shared__ float sv[32];
-  __shared__ int si[32];
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-  }
-  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = v; si[threadIdx.x >> 5] = idx; }
+  // lanes r, r + 8, r + 16, r + 24 of a warp hold the same row
+  for (int off = 8; off < 32; off <<= 1)
+    argmax_take(v, idx, __shfl_xor_sync(0xffffffffu, v, off), __shfl_xor_sync(0xffffffffu, idx, off));
+  __shared__ float sv[8][8];
+  __shared__ int si[8][8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane < 8) { sv[warp][lane] = v; si[warp][lane] = idx; }
   __syncthreads();
-  if (threadIdx.x < 32) {
-    const int nw = blockDim.x >> 5;
-    v = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
-    idx = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-      const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-    }
-    if (threadIdx.x == 0) ids[m] = id_map ? id_map[idx] : idx;   // pruned drafter vocabulary: row index -> token id
+  if (threadIdx.x < 8 && m < M) {
+    v = sv[0][r]; idx = si[0][r];
+    for (int w = 1; w < 8; ++w) argmax_take(v, idx, sv[w][r], si[w][r]);
+    ids[m] = id_map ? id_map[idx] : idx;                    // pruned drafter vocabulary: row index -> token id
   }
 }
 
@@ -506,7 +504,7 @@ cudaError_t splitk_reduce_launch(const float* part, int splits, int M, int N, vo
 cudaError_t argmax_reduce_launch(const float* pv, const int* pi, int n_tiles, int M, int* ids, cudaStream_t stream,
                                  Tracker* trk, const int* id_map) {
   trk_begin(trk, "argmax_reduce", 0, double(n_tiles) * M * 8);
-  launch_pdl(argmax_reduce_kernel, dim3(M), dim3(256), 0, stream, pv, pi, n_tiles, M, ids, id_map);
+  launch_pdl(argmax_reduce_kernel, dim3((M + 7) / 8), dim3(256), 0, stream, pv, pi, n_tiles, M, ids, id_map);
   trk_end(trk);
   return cudaGetLastError();
 }
