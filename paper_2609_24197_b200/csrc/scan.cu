@@ -444,14 +444,17 @@ scan_cb_kernel(ScanArgs a, const float* __restrict__ xact, float* __restrict__ c
 }
 
 template <int P, int N, int MT>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, MT == 1 ? 4 : 3)
 mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __half* __restrict__ c16,
                          const float* __restrict__ cb) {
   pdl_wait();
   pdl_trigger();
-  constexpr int HPC = 4, NT = P / 8, KP = N / 32, ROWS = MT * 16;
-  constexpr int CS = 2 * N + 32;                               // halves per C row (hi | lo | 64 bytes of padding: the 16-byte
-                                                               // fragment reads of rows gq and gq + 1 then fall on different banks)
+  constexpr int HPC = 4, NT = P / 8, ROWS = MT * 16;
+  constexpr int XS = P + 8;                                    // floats per x row in shared memory (padded: the fragment reads
+                                                               // of rows tq and columns gq then fall on 32 different banks)
+  constexpr int CS = 2 * N + 8;                                // halves per C row (hi | lo | 16 bytes of padding: the 16-byte
+                                                               // fragment reads, 32 bytes apart along a row, of rows gq and gq + 1
+                                                               // then fall on different banks)
   extern __shared__ __align__(16) float sm[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h0 = blockIdx.x * HPC, b = blockIdx.y;
@@ -460,19 +463,18 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   const size_t row0 = size_t(b) * k;
   __half* C16 = reinterpret_cast<__half*>(sm);                 // [ROWS][CS]  (hi, lo), rows >= k zero
   float* CB = sm + ROWS * CS / 2;                                   // [ROWS][ROWS]
-  float* xs = CB + ROWS * ROWS + warp * (ROWS * P);            // per warp [ROWS][P]
-  float* Wh = CB + ROWS * ROWS + HPC * ROWS * P + warp * ROWS * (ROWS + 1);   // per warp [ROWS][ROWS+1]
+  float* xs = CB + ROWS * ROWS + warp * (ROWS * XS);           // per warp [ROWS][XS]
+  float* Wh = CB + ROWS * ROWS + HPC * ROWS * XS + warp * ROWS * (ROWS + 1);   // per warp [ROWS][ROWS+1]
 
   // ---- state fragments of the first two k-step pairs: issued before anything else
   const int gq = lane >> 2, tq = lane & 3;
   const __half* S = a.s_init ? a.s_init + (size_t(b) * a.H + h) * P * N : nullptr;
-  uint4 sv0[NT], sv1[NT];
+  // (32-byte loads: the four lanes of a row then cover a whole 128-byte line per instruction; with 16-byte loads every
+  // line was touched twice, and the state's loads were a quarter of the L1's work)
+  uint4 sv0[NT][2];
   if (S != nullptr) {
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      sv0[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + 0 * 32 + tq * 8));
-      sv1[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + 1 * 32 + tq * 8));
-    }
+    for (int j = 0; j < NT; ++j) ldg_nc_32B(S + size_t(j * 8 + gq) * N + tq * 16, sv0[j][0], sv0[j][1]);
   }
   // ---- shared operands (C halves, CB) and this head's x rows: cp.async, zero fill for the padding rows
   for (int idx = tid; idx < ROWS * 2 * N / 8; idx += 128) {
@@ -485,7 +487,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   }
   for (int idx = lane; idx < ROWS * P / 4; idx += 32) {
     const int r = idx / (P / 4), c4 = idx % (P / 4);
-    cp_async16(smem_u32(xs + r * P + c4 * 4), xact + (row0 + min(r, k - 1)) * a.d_xBC + h * P + c4 * 4, r < k);
+    cp_async16(smem_u32(xs + r * XS + c4 * 4), xact + (row0 + min(r, k - 1)) * a.d_xBC + h * P + c4 * 4, r < k);
   }
   cp_async_commit();
   // ---- dt, inclusive prefix sum of dt * A over the block positions (one warp shuffle scan per head)
@@ -503,11 +505,14 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
   }
   cp_async_wait<0>();
   __syncthreads();
-  // ---- W[t][s] = exp(c_t - c_s) dt_s CB[t][s]: lane s owns column s
-  for (int t = 0; t < k; ++t) {
-    const float ct = __shfl_sync(0xffffffffu, cum, t);
+  // ---- W[t][s] = exp(c_t - c_s) dt_s CB[t][s] for s <= t, plus the skip weight D on the diagonal: lane s owns
+  // column s; the rows past k are zero
+  const float Dh = a.Dskip[h];
+  for (int t = 0; t < ROWS; ++t) {
+    const float ct = __shfl_sync(0xffffffffu, cum, t & 31);
     float w = 0.f;
-    if (lane <= t) w = __expf(ct - cum) * dt * CB[t * ROWS + lane];
+    if (t < k && lane <= t) w = __expf(ct - cum) * dt * CB[t * ROWS + lane];
+    if (t < k && lane == t) w += Dh;
     if (lane < ROWS) Wh[t * (ROWS + 1) + lane] = w;
   }
   __syncwarp();
@@ -519,66 +524,90 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
     for (int j = 0; j < NT; ++j) { acc[mt][j][0] = acc[mt][j][1] = acc[mt][j][2] = acc[mt][j][3] = 0.f; }
   if (S != nullptr) {
 #pragma unroll
-    for (int kp = 0; kp < KP; ++kp) {
-      uint4 sv[NT];
-      if (kp >= 2) {
+    // the contraction index is permuted (the same way for C and for the state): within a chunk of 64, lane tq's 16
+    // consecutive elements serve four k-steps, four elements each
+    for (int kq = 0; kq < N / 64; ++kq) {
+      uint4 sv[NT][2];
+      if (kq >= 1) {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) sv[j] = __ldg(reinterpret_cast<const uint4*>(S + size_t(j * 8 + gq) * N + kp * 32 + tq * 8));
+        for (int j = 0; j < NT; ++j) ldg_nc_32B(S + size_t(j * 8 + gq) * N + kq * 64 + tq * 16, sv[j][0], sv[j][1]);
       } else {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) sv[j] = kp == 0 ? sv0[j] : sv1[j];
+        for (int j = 0; j < NT; ++j) { sv[j][0] = sv0[j][0]; sv[j][1] = sv0[j][1]; }
       }
 #pragma unroll
-      for (int mt = 0; mt < MT; ++mt) {
-        const __half* c0 = C16 + (mt * 16 + gq) * CS + kp * 32 + tq * 8;
-        const __half* c1 = C16 + (mt * 16 + gq + 8) * CS + kp * 32 + tq * 8;
-        const uint4 c_lo = *reinterpret_cast<const uint4*>(c0), c_hi = *reinterpret_cast<const uint4*>(c1);
-        const uint4 r_lo = *reinterpret_cast<const uint4*>(c0 + N), r_hi = *reinterpret_cast<const uint4*>(c1 + N);
-        const uint32_t a0[4] = {c_lo.x, c_hi.x, c_lo.y, c_hi.y}, a1[4] = {c_lo.z, c_hi.z, c_lo.w, c_hi.w};
-        const uint32_t e0[4] = {r_lo.x, r_hi.x, r_lo.y, r_hi.y}, e1[4] = {r_lo.z, r_hi.z, r_lo.w, r_hi.w};
+      for (int piece = 0; piece < 2; ++piece) {
 #pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          mma_f16_16816(acc[mt][j], a0, sv[j].x, sv[j].y);
-          mma_f16_16816(acc[mt][j], a1, sv[j].z, sv[j].w);
-          mma_f16_16816(acc[mt][j], e0, sv[j].x, sv[j].y);
-          mma_f16_16816(acc[mt][j], e1, sv[j].z, sv[j].w);
+        for (int mt = 0; mt < MT; ++mt) {
+          const __half* c0 = C16 + (mt * 16 + gq) * CS + kq * 64 + tq * 16 + piece * 8;
+          const __half* c1 = C16 + (mt * 16 + gq + 8) * CS + kq * 64 + tq * 16 + piece * 8;
+          const uint4 c_lo = *reinterpret_cast<const uint4*>(c0), c_hi = *reinterpret_cast<const uint4*>(c1);
+          const uint4 r_lo = *reinterpret_cast<const uint4*>(c0 + N), r_hi = *reinterpret_cast<const uint4*>(c1 + N);
+          const uint32_t a0[4] = {c_lo.x, c_hi.x, c_lo.y, c_hi.y}, a1[4] = {c_lo.z, c_hi.z, c_lo.w, c_hi.w};
+          const uint32_t e0[4] = {r_lo.x, r_hi.x, r_lo.y, r_hi.y}, e1[4] = {r_lo.z, r_hi.z, r_lo.w, r_hi.w};
+#pragma unroll
+          for (int j = 0; j < NT; ++j) {
+            mma_f16_16816(acc[mt][j], a0, sv[j][piece].x, sv[j][piece].y);
+            mma_f16_16816(acc[mt][j], a1, sv[j][piece].z, sv[j][piece].w);
+            mma_f16_16816(acc[mt][j], e0, sv[j][piece].x, sv[j][piece].y);
+            mma_f16_16816(acc[mt][j], e1, sv[j][piece].z, sv[j][piece].w);
+          }
         }
       }
     }
   }
-  // ---- epilogue: decay, intra-block term, D skip, gate
-  const float Dh = a.Dskip[h];
+  // ---- decay of the state term: row t of the accumulator times exp(c_t)
+#pragma unroll
+  for (int mt = 0; mt < MT; ++mt) {
+    const float d_lo = __expf(__shfl_sync(0xffffffffu, cum, (mt * 16 + gq) & 31));
+    const float d_hi = __expf(__shfl_sync(0xffffffffu, cum, (mt * 16 + gq + 8) & 31));
+#pragma unroll
+    for (int j = 0; j < NT; ++j) { acc[mt][j][0] *= d_lo; acc[mt][j][1] *= d_lo; acc[mt][j][2] *= d_hi; acc[mt][j][3] *= d_hi; }
+  }
+  // ---- intra-block term and D skip, y_t += sum_{s <= t} W[t][s] x_s, as a [ROWS x ROWS] x [ROWS x P] product on the
+  // tensor cores: tf32 operands keep fp32's range (W is a product of exponentials, dt and a 128-term dot product), and
+  // each operand is split in two tf32 parts, three products per k-step, for ~21 bits.  (The scalar form read x from
+  // shared memory once per (t, s) pair and thread, and the kernel ran at the L1's limit.)
+#pragma unroll
+  for (int ks = 0; ks < ROWS / 8; ++ks) {
+    uint32_t ah[MT][4], al[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+      const float* wr = Wh + (mt * 16 + gq) * (ROWS + 1) + ks * 8 + tq;
+      split_tf32(wr[0], ah[mt][0], al[mt][0]);
+      split_tf32(wr[8 * (ROWS + 1)], ah[mt][1], al[mt][1]);
+      split_tf32(wr[4], ah[mt][2], al[mt][2]);
+      split_tf32(wr[8 * (ROWS + 1) + 4], ah[mt][3], al[mt][3]);
+    }
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      uint32_t bh[2], bl[2];
+      split_tf32(xs[(ks * 8 + tq) * XS + j * 8 + gq], bh[0], bl[0]);
+      split_tf32(xs[(ks * 8 + tq + 4) * XS + j * 8 + gq], bh[1], bl[1]);
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        if (ks * 8 > mt * 16 + 15) continue;                   // W is lower triangular: nothing in this k-step for these rows
+        mma_tf32_1688(acc[mt][j], al[mt], bh[0], bh[1]);
+        mma_tf32_1688(acc[mt][j], ah[mt], bl[0], bl[1]);
+        mma_tf32_1688(acc[mt][j], ah[mt], bh[0], bh[1]);
+      }
+    }
+  }
+  // ---- gate and store
 #pragma unroll
   for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
       const int t = mt * 16 + gq + half * 8;
-      const float dec = __expf(__shfl_sync(0xffffffffu, cum, t & 31));
       if (t >= k) continue;
       const size_t row = row0 + t;
       float2 z[NT];
 #pragma unroll
       for (int j = 0; j < NT; ++j) z[j] = *reinterpret_cast<const float2*>(a.zxbcdt + row * a.ld_in + h * P + j * 8 + tq * 2);
-      float y[NT][2];
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        const float2 xv = *reinterpret_cast<const float2*>(xs + t * P + j * 8 + tq * 2);
-        y[j][0] = dec * acc[mt][j][half * 2] + Dh * xv.x;
-        y[j][1] = dec * acc[mt][j][half * 2 + 1] + Dh * xv.y;
-      }
-      for (int s2 = 0; s2 <= t; ++s2) {
-        const float w = Wh[t * (ROWS + 1) + s2];
-#pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          const float2 xv = *reinterpret_cast<const float2*>(xs + s2 * P + j * 8 + tq * 2);
-          y[j][0] += w * xv.x;
-          y[j][1] += w * xv.y;
-        }
-      }
 #pragma unroll
       for (int j = 0; j < NT; ++j)
         *reinterpret_cast<float2*>(a.y + row * a.Di + h * P + j * 8 + tq * 2) =
-            make_float2(y[j][0] * silu_f(z[j].x), y[j][1] * silu_f(z[j].y));
+            make_float2(acc[mt][j][half * 2] * silu_f(z[j].x), acc[mt][j][half * 2 + 1] * silu_f(z[j].y));
     }
   }
 }
@@ -586,7 +615,7 @@ mamba_scan_stream_kernel(ScanArgs a, const float* __restrict__ xact, const __hal
 template <int MT>
 size_t scan_stream_smem() {
   constexpr int P = 64, N = 128, HPC = 4, ROWS = MT * 16;
-  return sizeof(__half) * ROWS * (2 * N + 32) + sizeof(float) * (ROWS * ROWS + HPC * ROWS * P + HPC * ROWS * (ROWS + 1));
+  return sizeof(__half) * ROWS * (2 * N + 8) + sizeof(float) * (ROWS * ROWS + HPC * ROWS * (P + 8) + HPC * ROWS * (ROWS + 1));
 }
 
 template <int MT>
@@ -615,6 +644,7 @@ cudaError_t scan_launch(const ScanCall& c, cudaStream_t stream, Tracker* trk, st
   if (a.H % c.G) { if (err) *err = "scan: heads must divide into groups"; return cudaErrorInvalidValue; }
   // serving shapes: tensor-core path (needs 8-byte aligned rows for the float2 accesses)
   if (c.P == 64 && c.N == 128 && (a.H / c.G) % 4 == 0 && c.ld_in % 2 == 0 && c.Di % 4 == 0 && c.ws != nullptr &&
+      (reinterpret_cast<uintptr_t>(c.s_init) & 31) == 0 &&     // its 32-byte loads of the state
       c.ws_bytes >= scan_workspace_bytes(c.B, c.k, c.Di, c.N, c.G)) {
     const bool two = c.k > 16;
     const size_t M = size_t(c.B) * c.k;
