@@ -48,7 +48,9 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return r;
 }
 
-// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 (or bf16) out.
+// y = x / sqrt(mean(x^2) + eps) * w, one CTA per row, fp16 (or bf16) out.  VPT = 16-byte vectors a thread keeps in
+// registers between the two passes.
+template <int VPT>
 __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ w, void* __restrict__ y,
                                int n, float eps, uint32_t* status, int bf16_out) {
   pdl_wait();
@@ -56,20 +58,20 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
   __shared__ float red[32];
   const float* xr = x + size_t(blockIdx.x) * n;
   uint16_t* yr = reinterpret_cast<uint16_t*>(y) + size_t(blockIdx.x) * n;      // a row of 16-bit values, either type
-  if ((n & 3) == 0 && n <= 4 * 6 * int(blockDim.x)) {
+  if ((n & 3) == 0 && n <= 4 * VPT * int(blockDim.x)) {
     // 16-byte loads, the row stays in registers between the two passes
-    float4 v[6];
+    float4 v[VPT];
     const int nv = n >> 2;
     float ss = 0.f;
 #pragma unroll
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < VPT; ++i) {
       const int d4 = threadIdx.x + i * blockDim.x;
       v[i] = d4 < nv ? reinterpret_cast<const float4*>(xr)[d4] : make_float4(0.f, 0.f, 0.f, 0.f);
       ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
     }
     const float inv = rsqrtf(block_sum(ss, red) / float(n) + eps);
 #pragma unroll
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < VPT; ++i) {
       const int d4 = threadIdx.x + i * blockDim.x;
       if (d4 < nv) {
         // (fetching the gains together with the row, before the block-wide sum, measured slower: 27 against 23 us)
@@ -312,8 +314,10 @@ cudaError_t embed_rows_launch(const void* embed_bf16, const int32_t* last_token,
 
 cudaError_t rmsnorm_launch(const float* x, const float* w, void* y_16, int M, int n, float eps, cudaStream_t stream,
                            uint32_t* status, bool bf16_out) {
-  const int threads = n >= 2048 ? 512 : 256;            // (256 or 384 threads per row measured the same at n = 5120)
-  cudaError_t e = launch_pdl(rmsnorm_kernel, dim3(M), dim3(threads), 0, stream, x, w, y_16, n, eps, status, bf16_out ? 1 : 0);
+  // 256 threads with up to six vectors each as long as the row fits (n <= 6144), else 512: at n = 5120 the profiler
+  // timed 16.5-17.1 us with 256 threads, 18.1-19.5 with 512, 19.6-21.0 with 128 (twelve vectors each)
+  const int threads = n <= 4 * 6 * 256 ? 256 : 512;
+  cudaError_t e = launch_pdl(rmsnorm_kernel<6>, dim3(M), dim3(threads), 0, stream, x, w, y_16, n, eps, status, bf16_out ? 1 : 0);
   return e != cudaSuccess ? e : cudaGetLastError();
 }
 
