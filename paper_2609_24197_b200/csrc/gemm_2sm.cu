@@ -16,8 +16,8 @@
 // the MMA thread (wait for "full", commit to "empty") costs the tensor pipe about 150 clocks whatever the order of the
 // operations, so it is paid once per eight MMAs instead of once per four.
 //
-// Measurement builds (HSPEC_NVCC_FLAGS): -DHSPEC_GEMM2_NOLOAD (no operand is fetched), -DHSPEC_GEMM2_NOEPI (accumulators
-// are not read out), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time); HSPEC_GEMM2_KSUB=1 in the
+// Measurement builds (HSPEC_NVCC_FLAGS): -DHSPEC_GEMM2_NOLOAD (no operand is fetched), -DHSPEC_GEMM2_NOMMA (no MMA is
+// issued, stages are released unread), -DHSPEC_GEMM2_NOEPI (accumulators are not read out), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time); HSPEC_GEMM2_KSUB=1 in the
 // environment goes back to one k-step per stage.  On M = 2048, n_out = 25600, K = 5120, SM clocks per 256 x 256 x 16
 // instruction (the arithmetic needs 128): MMA issue alone, no barrier at all 128; one k-step per stage 167 alone and
 // 182 with loads and read-out; two k-steps per stage 146 and 160.
@@ -241,9 +241,13 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
           for (int sub = 0; sub < n_sub; ++sub) {
             const uint32_t sa = smem_u32(smem + size_t(s) * stage_bytes + size_t(sub) * sub_bytes);
             const uint64_t da = umma_desc_kmajor_sw128(sa), db = umma_desc_kmajor_sw128(sa + A_BYTES);
+#ifndef HSPEC_GEMM2_NOMMA                   // measurement build: stages are released unread (shows the load path's own rate)
 #pragma unroll
             for (int kk = 0; kk < TILE_K / 16; ++kk)
               umma_2sm(tmem_acc, da + uint64_t(kk * 2), db + uint64_t(kk * 2), idesc, (kt > kt_begin || sub > 0 || kk > 0) ? 1u : 0u);
+#else
+            (void)da; (void)db; (void)idesc;
+#endif
           }
           umma_commit_pair(smem_u32(&tail->empty[s]));
         }
