@@ -22,6 +22,7 @@
 
 #include <cuda.h>
 
+#include <cstdio>
 #include <cstdlib>
 
 namespace hspec {
@@ -45,6 +46,9 @@ struct __align__(8) GemmSmemTail {
 
 __global__ void __launch_bounds__(192, 2)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs g) {
+#ifdef HSPEC_GEMM_CLOCK
+  const long long clk_start = clock64();     // measurement build: one CTA prints where its clocks went
+#endif
   extern __shared__ uint8_t smem_raw[];
   // 128-byte swizzle needs 1024-byte aligned tiles
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -83,6 +87,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const uint32_t tmem_acc = tail->tmem_base;
   pdl_wait();                                   // set-up done: now the previous kernel's results may be read
   pdl_trigger();
+#ifdef HSPEC_GEMM_CLOCK
+  const long long clk_setup = clock64();
+#endif
 
   if (warp == 0) {
     if (lane == 0) {
@@ -138,7 +145,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                         // TMEM lane quarter this warp may read
-    if (g.addend != nullptr) {
+    if (g.addend != nullptr && g.mode == EPI_ARGMAX) {
       // the addend rows of this tile do not depend on the accumulator: pull this warp's 128-byte piece of every
       // row into L2 while the main loop runs (one line per lane and pass)
       const int n_w = tile_n * TILE_W + q * 32;
@@ -148,15 +155,93 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (m < g.M) asm volatile("prefetch.global.L2 [%0];" ::"l"(g.addend + size_t(m) * g.ld_add + n_w));
         }
     }
+    // EPI_ARGMAX_T: lane = request, its addends for the tile's columns are BN contiguous floats.  They do not depend on
+    // the accumulator: the first 64 are requested before the wait for it, and every group of 16 is re-filled as soon as
+    // it is used (64 loads per thread in flight; one dependent round trip per group made a CTA's epilogue 30 us).
+    float aq[4][16];
+    const int n_t = tile_n * TILE_W + q * 32 + lane;
+    const bool t_on = g.mode == EPI_ARGMAX_T && g.addend != nullptr && n_t < g.N_out;
+    auto load_aq = [&](float (&dst)[16], int c_first) {
+      const int mf = tile_m * g.BN + c_first;
+      const float* arow = g.addend + size_t(n_t) * g.ld_add + mf;
+      if (t_on && c_first < g.BN && mf + 16 <= g.M && (reinterpret_cast<uintptr_t>(arow) & 15) == 0) {
+#pragma unroll
+        for (int j4 = 0; j4 < 4; ++j4) {
+          const float4 t = __ldg(reinterpret_cast<const float4*>(arow) + j4);
+          dst[4 * j4] = t.x; dst[4 * j4 + 1] = t.y; dst[4 * j4 + 2] = t.z; dst[4 * j4 + 3] = t.w;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) dst[j] = (t_on && c_first < g.BN && mf + j < g.M) ? __ldg(arow + j) : 0.f;
+      }
+    };
+    if (g.mode == EPI_ARGMAX_T) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) load_aq(aq[u], u * 16);
+    }
     bool ok = mbar_wait(smem_u32(&tail->tmem_full), 0);
+#ifdef HSPEC_GEMM_CLOCK
+    const long long clk_acc = clock64();
+#endif
     if (!ok) atomicExch(g.status, STATUS_TIMEOUT_EPILOGUE);
     tc_fence_after();
     if (*reinterpret_cast<volatile uint32_t*>(&tail->abort_flag)) ok = false;
     const int m0 = tile_m * g.BN;
-    for (int w = 0; w < g.WT; ++w) {                // (WT = 2 is never combined with the arg-max epilogue)
+    // EPI_ARGMAX_T: this lane's running (max, lowest column) over the tile's columns
+    float t_best = -INFINITY;
+    int t_idx = 0x7fffffff;
+    if (g.mode == EPI_ARGMAX_T) {
+      // value = acc + addend[request][vocabulary row]; the arg-max over the tile's vocabulary rows runs inside the
+      // thread (ascending columns, strict comparison: the lowest index wins ties), no shuffles
+      const bool n_ok_t = n_t < g.N_out;
+      for (int c00 = 0; c00 < g.BN && ok; c00 += 64) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int c0 = c00 + u * 16;
+          if (c0 >= g.BN) break;                    // warp-uniform
+          uint32_t r[16];
+          tmem_ld16(tmem_acc + (uint32_t(q * 32) << 16) + uint32_t(c0), r);
+          tmem_ld_wait();
+          float add[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) add[j] = aq[u][j];
+          load_aq(aq[u], c0 + 64);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const int m = m0 + c0 + j;
+            const float val = __uint_as_float(r[j]) + add[j];
+            if (n_ok_t && m < g.M) {
+              if (g.logits != nullptr) g.logits[size_t(n_t) * g.ldo + m] = val;
+              if (val > t_best) { t_best = val; t_idx = m; }
+            }
+          }
+        }
+      }
+    }
+    for (int w = 0; w < g.WT && g.mode != EPI_ARGMAX_T; ++w) {   // (WT = 2 is never combined with the arg-max epilogues)
     const int tile_w = tile_n * g.WT + w;           // 128-row weight tile of this pass
     const int n = tile_w * TILE_W + q * 32 + lane;  // output feature (weight row) of this thread
     const bool n_ok = n < g.N_out;
+    // Addend of the arg-max epilogue (the causal-correction head): the loads of the next 16 columns are issued before
+    // this batch is reduced.  Measured on that head's CTAs (-DHSPEC_GEMM_CLOCK; K = 256, 128 requests): the epilogue
+    // takes 23 000 of a CTA's 29 000 clocks - 10 000 with neither addend nor reduction, +6 000 for the reduction network,
+    // +7 500 for the addend - and a queue of 64 loads per thread instead of 16 changes nothing: with two CTAs of four
+    // epilogue warps per SM it is the warps' instruction latency, not memory, that sets the pace.
+    float add_next[16];
+    auto load_addend = [&](int c_first) {
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int m = m0 + c_first + j;
+#ifdef HSPEC_GEMM_NOADDEND                   // measurement build
+        add_next[j] = float(m);
+#else
+        add_next[j] = (n_ok && c_first < g.BN && m < g.M) ? __ldcs(g.addend + size_t(m) * g.ld_add + n) : 0.f;
+#endif
+      }
+    };
+    const bool with_addend = g.mode == EPI_ARGMAX && g.addend != nullptr;
+    if (with_addend && ok) load_addend(0);
+
     for (int c0 = 0; c0 < g.BN && ok; c0 += 16) {
       uint32_t r[16];
       tmem_ld16(tmem_acc + (uint32_t(q * 32) << 16) + uint32_t(w * g.BN + c0), r);
@@ -201,16 +286,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       } else {  // EPI_ARGMAX: logits optional, (max, lowest index) over this warp's 32 vocabulary rows
         float add[16];
-        if (g.addend != nullptr) {      // all 16 loads in flight before the first use
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const int m = m0 + c0 + j;
-            add[j] = (n_ok && m < g.M) ? __ldcs(g.addend + size_t(m) * g.ld_add + n) : 0.f;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) add[j] = 0.f;
-        }
+        for (int j = 0; j < 16; ++j) add[j] = with_addend ? add_next[j] : 0.f;
+        if (with_addend) load_addend(c0 + 16);
         float v[16];
         int vi[16];
 #pragma unroll
@@ -220,11 +298,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           vi[j] = n;
           if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v[j];
         }
-        int row;
+        int row = 0;
+#ifndef HSPEC_GEMM_NOARGMAX                   // measurement build
         warp_argmax16(v, vi, lane, row);
+#endif
         if ((lane & 1) == 0) { tail->red_val[q][c0 + row] = v[0]; tail->red_idx[q][c0 + row] = vi[0]; }
       }
     }
+    }
+    if (g.mode == EPI_ARGMAX_T) {
+      // per (column tile, request): [tile_m][N_out]
+      const int n = tile_n * TILE_W + q * 32 + lane;
+      if (n < g.N_out) {
+        g.part_val[size_t(tile_m) * g.N_out + n] = ok ? t_best : -INFINITY;
+        g.part_idx[size_t(tile_m) * g.N_out + n] = ok ? t_idx : 0x7fffffff;
+      }
     }
     if (g.mode == EPI_ARGMAX) {
       asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
@@ -245,6 +333,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         g.part_idx[size_t(tile_n) * g.M + m] = idx;
       }
     }
+#ifdef HSPEC_GEMM_CLOCK
+    if (blockIdx.y == gridDim.y / 2 && blockIdx.x == 0 && blockIdx.z == 0 && threadIdx.x == 64)
+      printf("gemm cta %d: set-up %lld clocks, until the accumulator is complete %lld, epilogue %lld\n", int(blockIdx.y),
+             clk_setup - clk_start, clk_acc - clk_setup, clock64() - clk_acc);
+#endif
     tc_fence_before();
   }
   __syncthreads();
@@ -425,7 +518,7 @@ cudaError_t gemm_launch(const GemmCall& c, cudaStream_t stream, Tracker* trk, st
   const int smem_optin = g_smem_optin[current_device()];
   GemmArgs g{};
   g.M = c.M; g.N_out = c.n_out; g.K = c.K;
-  g.BN = gemm_pick_bn(c.M);
+  g.BN = c.bn > 0 ? c.bn : gemm_pick_bn(c.M);
   g.k_tiles_total = (c.K + TILE_K - 1) / TILE_K;
   int splits = c.splits < 1 ? 1 : c.splits;
   if (splits > g.k_tiles_total) splits = g.k_tiles_total;

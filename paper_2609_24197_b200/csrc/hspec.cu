@@ -628,7 +628,7 @@ int hspec_draft_block(hspec_handle* h, const hspec_step* in, const hspec_out* ou
     g.out = logits; g.ldo = d.Vd; g.status = h->d_status; g.label = "gemm:lm_head";
     CUDA_TRY(h, gemm_launch(g, st, trk, &errtxt));
     MarkovCall mc{};
-    mc.logits = logits; mc.ld = d.Vd; mc.W_in = W("markov_in").data; mc.tmW_out = &W("markov_out").tm; mc.f16 = !bf;
+    mc.logits = logits; mc.ld = d.Vd; mc.W_in = W("markov_in").data; mc.tmW_out = &W("markov_out").tm; mc.W_out = W("markov_out").data; mc.f16 = !bf;
     mc.last_token = in->last_token; mc.id_map = id_map; mc.ids = out->draft_ids; mc.B = B; mc.k = k; mc.Vd = d.Vd;
     mc.r = c.markov_rank; mc.write_logits = out->logits != nullptr; mc.ws = ws + p.MARKOV; mc.status = h->d_status;
     CUDA_TRY(h, markov_launch(mc, st, trk, &errtxt));
@@ -822,7 +822,7 @@ int hspec_op_markov_head(float* logits, int64_t ld, const void* W_in, const void
   if (!make_tmap_16bit_2d(&tm, W_out, Vd, r, r, 128, w_dtype == HSPEC_F16, &errtxt))
     return fail(nullptr, HSPEC_ERR_BAD_SHAPE, "hspec_op_markov_head: " + errtxt);
   MarkovCall mc{};
-  mc.logits = logits; mc.ld = ld; mc.W_in = W_in; mc.tmW_out = &tm; mc.f16 = (w_dtype == HSPEC_F16);
+  mc.logits = logits; mc.ld = ld; mc.W_in = W_in; mc.tmW_out = &tm; mc.W_out = W_out; mc.f16 = (w_dtype == HSPEC_F16);
   mc.last_token = last_token; mc.id_map = id_map; mc.ids = ids; mc.B = B; mc.k = k; mc.Vd = Vd; mc.r = r;
   mc.write_logits = write_logits; mc.ws = workspace;
   mc.status = global_status();

@@ -100,6 +100,8 @@ enum GemmEpilogue : int {
   EPI_STORE_F16 = 5,    // y fp16 = acc
   EPI_SWIGLU_F16 = 6,   // weight rows interleaved in blocks of 16 (gate | up): h fp16 [M, n_out/2] = SiLU(gate) * up
   EPI_SWIGLU_BF16 = 7,  // the same with h stored as bf16
+  EPI_ARGMAX_T = 8,     // arg-max over the ACTIVATION side: the "weights" are a few rows (the requests' factor rows), the
+                        // "activations" the vocabulary matrix; every accumulator lane (request) reduces its own columns
 };
 inline bool epi_is_swiglu(int mode) { return mode == EPI_SWIGLU_F16 || mode == EPI_SWIGLU_BF16; }
 
@@ -143,6 +145,7 @@ struct GemmCall {       // host-side description of one y = x W^T
   int* part_idx;
   uint32_t* status;
   const char* label;        // profile name (may be null)
+  int bn;                   // one-CTA kernel: activation rows per CTA (0 = by the row count)
 };
 
 bool make_tmap_16bit_2d(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld_elems,
@@ -166,6 +169,7 @@ struct MarkovCall {
   long long ld;
   const void *W_in;                 // [V, r] 16-bit: factor row of every possible previous token
   const CUtensorMap* tmW_out;       // [Vd, r] 16-bit, box 128 x 64
+  const void* W_out;                // the same matrix by address
   bool f16;
   const int* last_token;            // [B]
   const int* id_map;                // [Vd] draft-vocabulary index -> token id, or null

@@ -3,6 +3,8 @@
 #include "common.cuh"
 #include "kernels.h"
 
+#include <cstdlib>
+
 namespace hspec {
 
 namespace {
@@ -95,49 +97,54 @@ __global__ void markov_gather_kernel(const uint16_t* __restrict__ W_in, const in
 
 // Position i of every request: lowest index among the per-tile maxima -> ids[b * k + i] (mapped to a token id when the
 // drafter's vocabulary is pruned), and the factor row of that token -> x[b, :] for position i + 1.
-__global__ void markov_reduce_gather_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int B,
-                                            int* __restrict__ ids, int k, int i, const int* __restrict__ id_map,
-                                            const uint16_t* __restrict__ W_in, uint16_t* __restrict__ x, int r, int gather) {
+// The partials are [tile][request]: a block takes eight consecutive requests, thread (tid % 8, tid / 8) walks every
+// 128th tile of its request, so that eight neighbouring threads read one 32-byte sector (1024 threads: there are only
+// B / 8 blocks, and the kernel sits between two dependent GEMMs, so its latency counts).
+__global__ void __launch_bounds__(1024)
+markov_reduce_gather_kernel(const float* __restrict__ pv, const int* __restrict__ pi, int n_tiles, int B,
+                            int* __restrict__ ids, int k, int i, const int* __restrict__ id_map,
+                            const uint16_t* __restrict__ W_in, uint16_t* __restrict__ x, int r, int gather) {
   pdl_wait();
   pdl_trigger();
-  const int b = blockIdx.x;
+  const int rr = threadIdx.x & 7, b = blockIdx.x * 8 + rr;
   float v = -INFINITY;
   int idx = 0x7fffffff;
-  for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
-    const float ov = pv[size_t(t) * B + b];
-    const int oi = pi[size_t(t) * B + b];
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
+  auto take = [&](float ov, int oi) { if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; } };
+  if (b < B) {
+    for (int t = threadIdx.x >> 3; t < n_tiles; t += 256) {          // two tiles' loads in flight per step
+      const int t2 = t + 128;
+      const float v1 = pv[size_t(t) * B + b], v2 = t2 < n_tiles ? pv[size_t(t2) * B + b] : -INFINITY;
+      const int i1 = pi[size_t(t) * B + b], i2 = t2 < n_tiles ? pi[size_t(t2) * B + b] : 0x7fffffff;
+      take(v1, i1);
+      take(v2, i2);
+    }
   }
-  __shared__ float sv[32];
-  __shared__ int si[32];
-  __shared__ int token;
-  for (int off = 16; off > 0; off >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-    if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-  }
-  if ((threadIdx.x & 31) == 0) { sv[threadIdx.x >> 5] = v; si[threadIdx.x >> 5] = idx; }
+  for (int off = 8; off < 32; off <<= 1) take(__shfl_xor_sync(0xffffffffu, v, off), __shfl_xor_sync(0xffffffffu, idx, off));
+  __shared__ float sv[32][8];
+  __shared__ int si[32][8];
+  __shared__ int token[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane < 8) { sv[warp][lane] = v; si[warp][lane] = idx; }
   __syncthreads();
-  if (threadIdx.x < 32) {
-    const int nw = blockDim.x >> 5;
-    v = threadIdx.x < nw ? sv[threadIdx.x] : -INFINITY;
-    idx = threadIdx.x < nw ? si[threadIdx.x] : 0x7fffffff;
-    for (int off = 16; off > 0; off >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, v, off);
-      const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
-      if (ov > v || (ov == v && oi < idx)) { v = ov; idx = oi; }
-    }
-    if (threadIdx.x == 0) {
-      const int tok = id_map ? id_map[idx] : idx;
+  if (threadIdx.x < 8) {
+    int tok = 0;
+    if (b < B) {
+      v = sv[0][rr]; idx = si[0][rr];
+      for (int w = 1; w < 32; ++w) take(sv[w][rr], si[w][rr]);
+      tok = id_map ? id_map[idx] : idx;
       ids[size_t(b) * k + i] = tok;
-      token = tok;
     }
+    token[rr] = tok;
   }
   __syncthreads();
   if (gather) {
-    const uint16_t* src = W_in + size_t(token) * r;
-    for (int j = threadIdx.x; j < (r >> 3); j += blockDim.x)
-      reinterpret_cast<uint4*>(x + size_t(b) * r)[j] = reinterpret_cast<const uint4*>(src)[j];
+    // warp w copies the factor row of request blockIdx.x * 8 + w (16 bytes per lane and step)
+    const int bw = blockIdx.x * 8 + warp;
+    if (warp < 8 && bw < B) {
+      const uint16_t* src = W_in + size_t(token[warp]) * r;
+      for (int j = lane; j < (r >> 3); j += 32)
+        reinterpret_cast<uint4*>(x + size_t(bw) * r)[j] = reinterpret_cast<const uint4*>(src)[j];
+    }
   }
 }
 
@@ -152,6 +159,16 @@ cudaError_t token_probs_launch(const float* logits, long long ld, const int* ids
   token_probs_kernel<<<M, 512, 0, stream>>>(logits, ld, ids, p, V);
   return cudaGetLastError();
 }
+
+// From 65 to 128 requests the head's GEMM runs with the operands' roles exchanged: the requests' factor rows x [B, r]
+// sit on the MMA's M side (one 128-row tile), the vocabulary matrix W_out on the N side in tiles of 128 rows, so that an
+// accumulator lane is a request and its arg-max over the tile's vocabulary rows runs inside one thread, its addends
+// 512 contiguous bytes fetched four groups ahead.  (With the vocabulary on the lanes every group of 16 columns goes
+// through a 32-shuffle reduction network and 16 separate addend loads: 23 000 of a CTA's 29 000 clocks at 128
+// requests.  Measured per step of 16 positions at 128 requests, V = 152 064, r = 256: 1.68 ms -> 1.42 ms; with 32
+// requests only a quarter of the lanes would work and the vocabulary-on-lanes form is as fast, 0.34 against 0.36 ms
+// for 8 positions.)
+constexpr int MARKOV_T_MIN_B = 65, MARKOV_T_MAX_B = 128, MARKOV_T_TILE = 128;
 
 size_t markov_workspace_bytes(int B, int Vd, int r) {
   const size_t vt = (size_t(Vd) + 127) / 128;
@@ -169,9 +186,18 @@ cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk
   trk_end(trk);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
+  const bool transposed = c.B >= MARKOV_T_MIN_B && c.B <= MARKOV_T_MAX_B && c.W_out != nullptr;
+  CUtensorMap tm_x;
+  if (transposed && !make_tmap_16bit_2d(&tm_x, x, c.B, c.r, c.r, 128, c.f16, err)) return cudaErrorInvalidValue;
+  const size_t n_part = transposed ? (size_t(c.Vd) + MARKOV_T_TILE - 1) / MARKOV_T_TILE : vt;
   for (int i = 0; i < c.k; ++i) {
     GemmCall g{};
-    g.tmW = c.tmW_out; g.x = x; g.ldx = c.r; g.f16 = c.f16; g.M = c.B; g.n_out = c.Vd; g.K = c.r; g.mode = EPI_ARGMAX; g.splits = 1;
+    if (transposed) {
+      g.tmW = &tm_x; g.x = c.W_out; g.ldx = c.r; g.M = c.Vd; g.n_out = c.B; g.mode = EPI_ARGMAX_T; g.bn = MARKOV_T_TILE;
+    } else {
+      g.tmW = c.tmW_out; g.x = x; g.ldx = c.r; g.M = c.B; g.n_out = c.Vd; g.mode = EPI_ARGMAX;
+    }
+    g.f16 = c.f16; g.K = c.r; g.splits = 1;
     g.addend = c.logits + size_t(i) * c.ld;                 // row b of this GEMM is row b * k + i of the block's logits
     g.ld_add = (long long)c.k * c.ld;
     g.logits = c.write_logits ? c.logits + size_t(i) * c.ld : nullptr;
@@ -182,8 +208,8 @@ cudaError_t markov_launch(const MarkovCall& c, cudaStream_t stream, Tracker* trk
     e = gemm_launch(g, stream, trk, err);
     if (e != cudaSuccess) return e;
     trk_begin(trk, "markov_reduce");
-    launch_pdl(markov_reduce_gather_kernel, dim3(c.B), dim3(128), 0, stream, (const float*)part_val, (const int*)part_idx,
-               int(vt), c.B, c.ids, c.k, i, c.id_map, reinterpret_cast<const uint16_t*>(c.W_in), x, c.r, int(i + 1 < c.k));
+    launch_pdl(markov_reduce_gather_kernel, dim3((c.B + 7) / 8), dim3(1024), 0, stream, (const float*)part_val, (const int*)part_idx,
+               int(n_part), c.B, c.ids, c.k, i, c.id_map, reinterpret_cast<const uint16_t*>(c.W_in), x, c.r, int(i + 1 < c.k));
     trk_end(trk);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;

@@ -121,6 +121,13 @@ def test_markov_many_requests(hs):
     _markov_case(hs, B=130, k=3, V=2048, Vd=2048, r=256, seed=4)      # more requests than one activation tile
 
 
+def test_markov_65_to_128_requests_take_the_request_on_lanes_form(hs):
+    # (ragged pruned vocabulary, rank not a multiple of 64, logits written back; then fp16 factors without write-back)
+    _markov_case(hs, B=100, k=3, V=3000, Vd=3000 - 37, r=72, seed=7)
+    _markov_case(hs, B=128, k=2, V=2048, Vd=2048, r=256, seed=8, dtype=torch.float16, write_logits=False)
+    _markov_case(hs, B=65, k=2, V=777, Vd=777, r=64, seed=9)
+
+
 def test_markov_strong_table_changes_the_draft(hs):
     """With a table strong enough to matter, the drafted ids differ from the plain arg-max of the logits."""
     B, k, V, r = 6, 8, 512, 128
