@@ -476,7 +476,9 @@ void gemm2_pick(int M, int n_out, int K, int mode, int* bnt_out, int* splits_out
       if (s > 1 && kps * (s - 1) >= k_tiles) continue;         // an empty last slice
       double cost = double(full_waves) * (k_tiles * kstep + 1500.0);
       if (tail > 0) cost += kps * kstep + 1500.0;
-      if (s > 1) cost += (double(s + 2) * tail * bnt * 256 * 4.0 / 4.0e6 + 4.0) * 455.0;
+      // (the pass that sums the slices: its bytes at 4 TB/s plus 2 us; with 4, 8, 12 or 20 us fewer launches are sliced and
+      // the 256-row steps get slower, 1.93 -> 1.95 / 2.02 / 2.07 / 2.10 ms at paper_8b; no difference at 2048 rows)
+      if (s > 1) cost += (double(s + 2) * tail * bnt * 256 * 4.0 / 4.0e6 + 2.0) * 455.0;
       if (cost < best_cost) { best_cost = cost; best_bnt = bnt; best_s = s; }
     }
   }
