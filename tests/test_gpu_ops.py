@@ -153,7 +153,11 @@ def test_swiglu(hs):
     assert_bf16_close(h.float().cpu().numpy(), O.silu(g[:, :F]) * g[:, F:], "swiglu", ulps=0.5)
 
 
-@pytest.mark.parametrize("dh,Hq,Hkv,theta,qk_norm", [(64, 4, 2, 1e4, 1), (128, 8, 2, 1e6, 1), (128, 4, 4, 1e6, 0)])
+# (dh <= 128 and a multiple of 4: the row-per-block kernel, also with lanes past dh / 4 idle and with more heads than one
+# pass of its eight warps takes; other head sizes: the warp-per-head kernel)
+@pytest.mark.parametrize("dh,Hq,Hkv,theta,qk_norm", [(64, 4, 2, 1e4, 1), (128, 8, 2, 1e6, 1), (128, 4, 4, 1e6, 0),
+                                                      (96, 4, 4, 1e4, 1), (128, 64, 8, 1e6, 1), (256, 4, 2, 1e4, 1),
+                                                      (66, 2, 1, 1e4, 1)])
 def test_qk_norm_rope(hs, dh, Hq, Hkv, theta, qk_norm):
     B, k = 3, 5
     ctx = torch.tensor([0, 2047, 32760], dtype=torch.int32, device="cuda")
@@ -182,12 +186,20 @@ def test_qk_norm_rope(hs, dh, Hq, Hkv, theta, qk_norm):
     (2, 1, 128, 64, 128, 1, False, False), (2, 32, 192, 64, 4, 1, False, False), (2, 7, 128, 32, 24, 2, False, True),
     (2, 32, 512, 64, 128, 2, False, False), (3, 11, 1024, 64, 128, 4, True, True),
 ])
-@pytest.mark.parametrize("with_scratch", [False, True])
+@pytest.mark.parametrize("with_scratch", [False, True, "in_8_mod_16"])
 def test_mamba_scan(hs, B, k, Di, P, N, G, dtr, zero_state, with_scratch):
     H, d_conv = Di // P, 4
     d_xBC = Di + 2 * G * N
     ld = Di + d_xBC + (0 if dtr else H)
     zx = _randn((B * k, ld), 31, 1.0)
+    if with_scratch == "in_8_mod_16":
+        # the in-projection's output at an address that is 8 but not 16 bytes aligned: the conv kernel's scalar form
+        if ld % 2:
+            pytest.skip("needs an even row pitch")
+        base = torch.empty(B * k * ld + 2, dtype=torch.float32, device="cuda")
+        base[2:].view(B * k, ld).copy_(zx)
+        zx = base[2:].view(B * k, ld)
+        assert zx.data_ptr() % 16 == 8
     dt_raw = _randn((B * k, H), 32, 1.0) if dtr else None
     s_init = None if zero_state else _randn((B, H, P, N), 33, 1.5, torch.float16)
     conv_w = (torch.rand((d_xBC, d_conv), device="cuda", generator=torch.Generator(device="cuda").manual_seed(34)) - 0.5)
