@@ -18,7 +18,7 @@
 // stages only: 1 291 against 1 331 TFLOP/s on M = 2048, n_out = 25600, K = 5120.)
 //
 // Measurement builds (HSPEC_NVCC_FLAGS): -DHSPEC_GEMM2_NOLOAD (no operand is fetched), -DHSPEC_GEMM2_NOMMA (no MMA is
-// issued, stages are released unread), -DHSPEC_GEMM2_NOEPI (accumulators are not read out), -DHSPEC_GEMM2_NOSTORE (read out, not stored), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time); HSPEC_GEMM2_KSUB=1 in the
+// issued, stages are released unread), -DHSPEC_GEMM2_NOEPI (accumulators are not read out), -DHSPEC_GEMM2_NOSTORE (read out, not stored), -DHSPEC_GEMM2_NOARGMAX (LM-head epilogue without its reduction network), -DHSPEC_GEMM2_CLOCK (CTA 0 prints its SM clock count and the wall time); HSPEC_GEMM2_KSUB=1 in the
 // environment goes back to one k-step per stage.  On M = 2048, n_out = 25600, K = 5120, SM clocks per 256 x 256 x 16
 // instruction (the arithmetic needs 128): MMA issue alone, no barrier at all 128; one k-step per stage 167 alone and
 // 182 with loads and read-out; two k-steps per stage 146 and 160.
@@ -348,8 +348,12 @@ gemm_2sm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             vi[j] = n;
             if (g.logits != nullptr && n_ok && m < g.M) g.logits[size_t(m) * g.ldo + n] = v[j];
           }
-          int row;
+          // (The network costs the LM head 4 % - 2.34 -> 2.24 ms per step without it - mostly as clock under the power cap.
+          // One redux.sync maximum + ballot per column instead of the shuffle rounds: 2.56 ms.)
+          int row = 0;
+#ifndef HSPEC_GEMM2_NOARGMAX                 // measurement build: no reduction network (ids are wrong)
           warp_argmax16(v, vi, lane, row);
+#endif
           if ((lane & 1) == 0) { tail->red_val[q][c0 + row] = v[0]; tail->red_idx[q][c0 + row] = vi[0]; }
         }
       }
